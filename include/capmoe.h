@@ -1,0 +1,199 @@
+/* capmoe - capacity-aware Mixture-of-Experts layer forward on one NVIDIA B200 (sm_100a).
+ *
+ * One MoE layer (Eq. 1-2 of "Capacity-Aware Inference: Mitigating the Straggler Effect in
+ * Mixture of Experts") with the paper's two capacity rules, as six stream-ordered stages:
+ *
+ *   capmoe_route          router GEMM, softmax, per-token top-k, expert load   (Eq. 1, Eq. 3)
+ *   capmoe_token_drop     Capacity-Aware Token Drop                           (Eq. 7-10, Algorithm 1)
+ *   capmoe_expanded_drop  Capacity-Aware Expanded Drop                        (Algorithm 2)
+ *   capmoe_permute        gather kept tokens into expert-major rows
+ *   capmoe_grouped_ffn    SwiGLU expert FFN over the per-expert row segments  (E_i(x) of Eq. 2)
+ *   capmoe_combine        gate-weighted sum back to token order               (Eq. 2)
+ *
+ * Conventions, unless an entry point says otherwise
+ *   - Pointers named in the argument lists are DEVICE pointers owned by the caller; the library
+ *     allocates no device memory, keeps no per-call state and never synchronises the stream.
+ *     `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - All tensors are dense, row-major, 16-byte aligned.  dtype selects the storage type of the
+ *     activations and weights (CAPMOE_F32 or CAPMOE_BF16); logits, scores and gate weights are
+ *     always fp32; accumulation is always fp32.
+ *   - The return value is the only error channel (a capmoe_status as int).  Arguments are
+ *     validated before anything is launched; on a non-zero return nothing was enqueued, except
+ *     CAPMOE_ECUDA which reports a failed launch or driver call.
+ *   - Every output is a deterministic function of the inputs (positions come from ordered
+ *     prefix scans, integer atomics only where the result is order-independent).
+ *   - Notation follows the paper: N tokens, hidden size d, E experts, k experts per token,
+ *     capacity factor gamma, capacity C, D (virtual) expert-parallel devices with m = E/D
+ *     experts each, F the expert FFN width, A the number of kept (token, expert) assignments.
+ */
+#ifndef CAPMOE_H_
+#define CAPMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CAPMOE_OK = 0,
+  CAPMOE_EINVAL = 1,       /* null / misaligned pointer, negative size, k > E, E % D != 0 ... */
+  CAPMOE_EUNSUPPORTED = 2, /* well-formed request with no kernel (dtype, row size not 16-byte) */
+  CAPMOE_EWORKSPACE = 3,   /* workspace smaller than capmoe_*_workspace_bytes reports        */
+  CAPMOE_ECUDA = 4,        /* a CUDA call failed; see capmoe_last_cuda_error                   */
+  CAPMOE_ETIMEOUT = 5      /* a bounded device-side wait ran out (read from dev_status)       */
+} capmoe_status;
+
+typedef enum { CAPMOE_F32 = 0, CAPMOE_BF16 = 1 } capmoe_dtype;
+typedef enum { CAPMOE_CAP_CEIL = 0, CAPMOE_CAP_FLOOR = 1 } capmoe_round;
+
+/* ---------------------------------------------------------------- host-only helpers */
+
+/* Expert capacity C = gamma * N_bar with N_bar = N*k/E (Eq. 3; "Token Drop" paragraph),
+ * evaluated as (gamma*(N*k))/E in double as Algorithm 1 does, rounded up (CAPMOE_CAP_CEIL,
+ * default) or down (CAPMOE_CAP_FLOOR, the listing's int()), clamped to [0, N].  gamma = +inf
+ * gives C = N, i.e. the layer without capacity limits.  Host pointer out. */
+int capmoe_capacity(int64_t N, int E, int k, double gamma, int round, int64_t* C);
+
+/* Upper bound on A (rows of the permuted matrix) known before routing:
+ * min(E*C, N*k) for Token Drop, min(E*C, N*(k+E/D)) for Expanded Drop.  Host pointer out. */
+int capmoe_max_rows(int64_t N, int E, int k, int D, int64_t C, int expanded, int64_t* A_max);
+
+/* Scratch needed by capmoe_token_drop (expanded = 0) / capmoe_expanded_drop (expanded = 1). */
+int capmoe_drop_workspace_bytes(int64_t N, int E, int k, int D, int expanded, size_t* bytes);
+
+const char* capmoe_status_str(int status);
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+const char* capmoe_last_cuda_error(void);
+/* Number of kernels this library has launched in this process (all threads). */
+uint64_t capmoe_launch_count(void);
+/* 1 if grouped_ffn would take the tcgen05/TMA tensor-core path for this shape, else 0. */
+int capmoe_ffn_uses_tensor_cores(int d, int F, int dtype);
+
+/* ---------------------------------------------------------------- stage 1: router
+ * logits[t,e] = sum_j x[t,j]*w_router[e,j] + bias[e]; scores = softmax(logits) per token;
+ * top-k of the scores per token (Eq. 1; Algorithm 1, first three statements); load[e] = N_e,
+ * the number of tokens whose top-k holds e (Eq. 3's N_i).
+ *   x [N,d], w_router [E,d] in `dtype`; bias [E] fp32 or NULL.
+ *   out: logits [N,E] fp32, scores [N,E] fp32, topk_idx [N,k] int32 (score descending, ties to
+ *        the lower expert id), topk_score [N,k] fp32 (raw softmax values, not renormalised),
+ *        load [E] int32.
+ * The softmax is evaluated in binary32 in a fixed order (max; exp by range reduction and a
+ * degree-7 polynomial in fma form; left-to-right sum; IEEE division), so scores are a pure
+ * function of the fp32 logits.  logits_in, when not NULL, replaces the GEMM: the stage then
+ * starts from the caller's fp32 logits [N,E] (x and w_router may be NULL).
+ * Requires 1 <= k <= E <= 256, k <= 32. */
+int capmoe_route(const void* x, const void* w_router, const float* bias, const float* logits_in,
+                 int64_t N, int d, int E, int k, int dtype,
+                 float* logits, float* scores, int32_t* topk_idx, float* topk_score, int32_t* load,
+                 void* stream);
+
+/* ---------------------------------------------------------------- stage 2: Token Drop
+ * For every expert e, among the tokens whose top-k holds e keep the C with the highest score
+ * (all of them if N_e <= C); equal scores go to the lower token index (Eq. 7-10, Algorithm 1).
+ *   in : topk_score [N,k] fp32, topk_idx [N,k] int32, capacity C in [0,N].
+ *   out: keep_mask [N, ceil(E/64)] uint64, bit (e%64) of word e/64 set iff (t,e) is kept;
+ *        kept [E] int32 = min(N_e, C); expert_offsets [E+1] int32, exclusive prefix of kept
+ *        (expert_offsets[E] = A); slot_row [N,k] int32 = row of the permuted matrix that holds
+ *        top-k slot j of token t, or -1 if dropped.  Rows of expert e are
+ *        [expert_offsets[e], expert_offsets[e+1]) in ascending token index.
+ *   ws : capmoe_drop_workspace_bytes(N,E,k,0,0) bytes, contents undefined on entry and exit.
+ * C = N is the layer without dropping. */
+int capmoe_token_drop(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
+                      int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
+                      int32_t* slot_row, void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------- stage 3: Expanded Drop
+ * Token t is a candidate of its top-k experts and of all m = E/D experts of its home device
+ * h(t); all candidates of an expert compete on scores[t,e]; the expert keeps its C best, ties
+ * to the lower token index (Algorithm 2).  A token may end with more than k experts.
+ *   in : scores [N,E] fp32, topk_idx [N,k], C, D (E % D == 0), token_group [N] int32 with
+ *        h(t) in [0,D) or NULL for contiguous blocks h(t) = floor(t*D/N).
+ *   out: keep_mask, kept, expert_offsets as above; cand [E] int32 = candidates per expert;
+ *        slot_row [N, k+m] int32: slots 0..k-1 are the top-k slots, slot k+i is local expert
+ *        h(t)*m+i when it is not one of the token's top-k (else -1).
+ *   ws : capmoe_drop_workspace_bytes(N,E,k,D,1) bytes. */
+int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
+                         int64_t C, int D, const int32_t* token_group, uint64_t* keep_mask,
+                         int32_t* cand, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row,
+                         void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------- stage 4: permute
+ * x_perm[r] = x[t], perm_token[r] = t, perm_weight[r] = scores[t,e] for every kept (t,e) with
+ * r = its slot_row entry.  slots = k after Token Drop (pass D = 0) or k+E/D after Expanded Drop.
+ *   in : x [N,d] `dtype`, scores [N,E] fp32, topk_idx [N,k], token_group (as in stage 3),
+ *        slot_row [N,slots].
+ *   out: x_perm [A,d] `dtype`, perm_token [A] int32, perm_weight [A] fp32 (A rows written).
+ * Requires d*sizeof(elt) to be a multiple of 16. */
+int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
+                   const float* scores, const int32_t* topk_idx, const int32_t* token_group,
+                   const int32_t* slot_row, void* x_perm, int32_t* perm_token, float* perm_weight,
+                   void* stream);
+
+/* ---------------------------------------------------------------- stage 5: grouped SwiGLU FFN
+ * For every expert e and every row r in [expert_offsets[e], expert_offsets[e+1]):
+ *   h = silu(W_g[e] x_perm[r]) * (W_u[e] x_perm[r]),  y_perm[r] = W_d[e] h      (E_i(x) in Eq. 2).
+ *   in : x_perm [A_max,d], expert_offsets [E+1] (device), w_gate, w_up [E,F,d], w_down [E,d,F].
+ *   ws : h_ws [A_max,F] in `dtype` (the hidden activations; contents undefined afterwards).
+ *   out: y_perm [A_max,d] in `dtype`; rows >= expert_offsets[E] are left untouched.
+ * A_max is the allocated row count of x_perm / h_ws / y_perm (>= A).  No host-device sync:
+ * tiles are scheduled on the device from expert_offsets.
+ * D_straggler > 0 (E % D_straggler == 0) turns on straggler emulation: the experts of virtual
+ * device g run only on a fixed share floor(#SM/D) of the SMs, so the most loaded device sets
+ * the latency as under expert parallelism (Eq. 4, L proportional to max_i N_i).
+ * dev_status [1] int32 (device, may be NULL): set to CAPMOE_ETIMEOUT if a bounded wait inside
+ * the tensor-core kernel ran out; the caller zeroes it and reads it after synchronising.
+ * bf16 with d % 64 == 0 and F % 128 == 0 runs on tcgen05 tensor cores with TMA-fed tiles;
+ * everything else (fp32, odd shapes) runs a plain fp32-FMA kernel. */
+int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F,
+                       int dtype, const void* w_gate, const void* w_up, const void* w_down,
+                       void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
+                       int32_t* dev_status, void* stream);
+
+/* ---------------------------------------------------------------- stage 6: combine
+ * y[t] = sum over slots s with slot_row[t,s] >= 0 of perm_weight[row] * y_perm[row], added in
+ * ascending slot order in fp32, plus y_shared[t] (weight 1) when y_shared is not NULL; a token
+ * with nothing kept gets y_shared[t] or zeros (Eq. 2 with the kept set in place of K).
+ *   in : y_perm [A,d] `dtype`, slot_row [N,slots], perm_weight [A] fp32, y_shared [N,d] or NULL.
+ *   out: y [N,d] `dtype`. */
+int capmoe_combine(const void* y_perm, const int32_t* slot_row, const float* perm_weight,
+                   int64_t N, int d, int slots, int dtype, const void* y_shared, void* y,
+                   void* stream);
+
+/* ---------------------------------------------------------------- whole layer
+ * Buffers for one layer forward.  Every pointer is a device pointer sized as noted. */
+typedef struct {
+  /* problem */
+  int64_t N; int d, E, k, F, D, dtype;
+  int mode;              /* 0 = no drop (C = N), 1 = Token Drop, 2 = Expanded Drop */
+  int64_t C;             /* capacity (ignored for mode 0) */
+  int straggler;         /* 0/1: run the FFN in straggler-emulation mode over D devices */
+  /* inputs */
+  const void* x; const void* w_router; const float* bias;
+  const void* w_gate; const void* w_up; const void* w_down;
+  const void* ws_gate; const void* ws_up; const void* ws_down; int F_shared; /* shared expert or NULL/0 */
+  /* outputs and intermediates */
+  float* logits; float* scores; int32_t* topk_idx; float* topk_score; int32_t* load;
+  uint64_t* keep_mask; int32_t* cand; int32_t* kept; int32_t* expert_offsets; int32_t* slot_row;
+  void* x_perm; int32_t* perm_token; float* perm_weight;
+  void* h_ws; void* y_perm; int64_t A_max;
+  void* hs_ws; void* y_shared;  /* shared expert scratch: [N,F_shared], [N,d] */
+  const int32_t* one_segment;   /* [2] int32 holding {0, N}: the shared expert's single row segment */
+  void* y;
+  void* drop_ws; size_t drop_ws_bytes;
+  int32_t* dev_status;
+} capmoe_layer;
+
+/* Runs the stages above in order on `stream` (route, drop, permute, FFN, [shared FFN], combine). */
+int capmoe_layer_forward(const capmoe_layer* L, void* stream);
+
+/* Same, with the activations on the HOST: copies x_host [N,d] (pinned) to L->x, runs the layer,
+ * copies L->y to y_host [N,d] (pinned), all on `stream`; weights stay resident on the device.
+ * L->x is used as the device staging buffer and must be writable. */
+int capmoe_layer_forward_host(const capmoe_layer* L, const void* x_host, void* y_host, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAPMOE_H_ */

@@ -1,0 +1,321 @@
+"""ctypes binding of libcapmoe.so: same names as the C ABI, argument marshalling only.
+
+torch is used for device memory and streams; every step of the layer runs inside the CUDA
+library.  If the shared library is missing or cannot be loaded, every call raises: there is
+no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libcapmoe.so")
+_lib = None
+
+OK, EINVAL, EUNSUPPORTED, EWORKSPACE, ECUDA, ETIMEOUT = range(6)
+F32, BF16 = 0, 1
+MODE_NODROP, MODE_TOKEN_DROP, MODE_EXPANDED_DROP = 0, 1, 2
+MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2}
+
+EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_drop_workspace_bytes", "capmoe_status_str",
+           "capmoe_last_cuda_error", "capmoe_launch_count", "capmoe_ffn_uses_tensor_cores", "capmoe_route",
+           "capmoe_token_drop", "capmoe_expanded_drop", "capmoe_permute", "capmoe_grouped_ffn",
+           "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host"]
+
+
+class CapmoeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().capmoe_status_str(status).decode()
+        if status == ECUDA:
+            msg += " (" + lib().capmoe_last_cuda_error().decode() + ")"
+        super().__init__(f"{where}: {msg} [status {status}]")
+
+
+class _Layer(ctypes.Structure):
+    _fields_ = [
+        ("N", ctypes.c_int64), ("d", ctypes.c_int), ("E", ctypes.c_int), ("k", ctypes.c_int),
+        ("F", ctypes.c_int), ("D", ctypes.c_int), ("dtype", ctypes.c_int),
+        ("mode", ctypes.c_int), ("C", ctypes.c_int64), ("straggler", ctypes.c_int),
+        ("x", ctypes.c_void_p), ("w_router", ctypes.c_void_p), ("bias", ctypes.c_void_p),
+        ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p), ("w_down", ctypes.c_void_p),
+        ("ws_gate", ctypes.c_void_p), ("ws_up", ctypes.c_void_p), ("ws_down", ctypes.c_void_p),
+        ("F_shared", ctypes.c_int),
+        ("logits", ctypes.c_void_p), ("scores", ctypes.c_void_p), ("topk_idx", ctypes.c_void_p),
+        ("topk_score", ctypes.c_void_p), ("load", ctypes.c_void_p),
+        ("keep_mask", ctypes.c_void_p), ("cand", ctypes.c_void_p), ("kept", ctypes.c_void_p),
+        ("expert_offsets", ctypes.c_void_p), ("slot_row", ctypes.c_void_p),
+        ("x_perm", ctypes.c_void_p), ("perm_token", ctypes.c_void_p), ("perm_weight", ctypes.c_void_p),
+        ("h_ws", ctypes.c_void_p), ("y_perm", ctypes.c_void_p), ("A_max", ctypes.c_int64),
+        ("hs_ws", ctypes.c_void_p), ("y_shared", ctypes.c_void_p), ("one_segment", ctypes.c_void_p),
+        ("y", ctypes.c_void_p),
+        ("drop_ws", ctypes.c_void_p), ("drop_ws_bytes", ctypes.c_size_t),
+        ("dev_status", ctypes.c_void_p),
+    ]
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_05066_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.capmoe_status_str.restype = ctypes.c_char_p
+        L.capmoe_last_cuda_error.restype = ctypes.c_char_p
+        L.capmoe_launch_count.restype = ctypes.c_uint64
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.is_contiguous(), "capmoe tensors must be contiguous"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dt(t_or_dtype) -> int:
+    dt = t_or_dtype.dtype if isinstance(t_or_dtype, torch.Tensor) else t_or_dtype
+    if dt == torch.float32:
+        return F32
+    if dt == torch.bfloat16:
+        return BF16
+    raise CapmoeError(EUNSUPPORTED, f"dtype {dt}")
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise CapmoeError(rc, where)
+
+
+def _i64(v):
+    return ctypes.c_int64(int(v))
+
+
+# ----------------------------------------------------------------------------- host helpers
+def capacity(N: int, E: int, k: int, gamma: float, round_mode: str = "ceil") -> int:
+    out = ctypes.c_int64(0)
+    _check(lib().capmoe_capacity(_i64(N), int(E), int(k), ctypes.c_double(gamma),
+                                 0 if round_mode == "ceil" else 1, ctypes.byref(out)), "capmoe_capacity")
+    return out.value
+
+
+def max_rows(N: int, E: int, k: int, D: int, C: int, expanded: bool) -> int:
+    out = ctypes.c_int64(0)
+    _check(lib().capmoe_max_rows(_i64(N), int(E), int(k), int(D), _i64(C), int(bool(expanded)),
+                                 ctypes.byref(out)), "capmoe_max_rows")
+    return out.value
+
+
+def drop_workspace_bytes(N: int, E: int, k: int, D: int, expanded: bool) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().capmoe_drop_workspace_bytes(_i64(N), int(E), int(k), int(D), int(bool(expanded)),
+                                             ctypes.byref(out)), "capmoe_drop_workspace_bytes")
+    return out.value
+
+
+def launch_count() -> int:
+    return int(lib().capmoe_launch_count())
+
+
+def ffn_uses_tensor_cores(d: int, F: int, dtype) -> bool:
+    return bool(lib().capmoe_ffn_uses_tensor_cores(int(d), int(F), _dt(dtype)))
+
+
+# ----------------------------------------------------------------------------- stages
+def route(x, w_router, bias, k: int, logits_in=None, stream=None):
+    """-> dict(logits, scores, topk_idx, topk_score, load)"""
+    if logits_in is not None:
+        N, E = logits_in.shape
+        d, dev, dt = 0, logits_in.device, F32
+    else:
+        N, d = x.shape
+        E = w_router.shape[0]
+        dev, dt = x.device, _dt(x)
+    f32 = dict(device=dev, dtype=torch.float32)
+    i32 = dict(device=dev, dtype=torch.int32)
+    out = dict(logits=torch.empty((N, E), **f32), scores=torch.empty((N, E), **f32),
+               topk_idx=torch.empty((N, k), **i32), topk_score=torch.empty((N, k), **f32),
+               load=torch.empty((E,), **i32))
+    _check(lib().capmoe_route(_ptr(x), _ptr(w_router), _ptr(bias), _ptr(logits_in), _i64(N), int(d), int(E),
+                              int(k), dt, _ptr(out["logits"]), _ptr(out["scores"]), _ptr(out["topk_idx"]),
+                              _ptr(out["topk_score"]), _ptr(out["load"]), _stream(stream)), "capmoe_route")
+    return out
+
+
+def token_drop(topk_score, topk_idx, E: int, C: int, ws=None, stream=None):
+    """-> dict(keep_mask, kept, offsets, slot_row)"""
+    N, k = topk_idx.shape
+    dev = topk_idx.device
+    W = (E + 63) // 64
+    if ws is None:
+        ws = torch.empty((drop_workspace_bytes(N, E, k, 0, False),), device=dev, dtype=torch.uint8)
+    out = dict(keep_mask=torch.empty((N, W), device=dev, dtype=torch.int64),
+               kept=torch.empty((E,), device=dev, dtype=torch.int32),
+               offsets=torch.empty((E + 1,), device=dev, dtype=torch.int32),
+               slot_row=torch.empty((N, k), device=dev, dtype=torch.int32))
+    _check(lib().capmoe_token_drop(_ptr(topk_score), _ptr(topk_idx), _i64(N), int(E), int(k), _i64(C),
+                                   _ptr(out["keep_mask"]), _ptr(out["kept"]), _ptr(out["offsets"]),
+                                   _ptr(out["slot_row"]), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                                   _stream(stream)), "capmoe_token_drop")
+    return out
+
+
+def expanded_drop(scores, topk_idx, C: int, D: int, token_group=None, ws=None, stream=None):
+    """-> dict(keep_mask, cand, kept, offsets, slot_row)"""
+    N, E = scores.shape
+    k = topk_idx.shape[1]
+    dev = scores.device
+    if D < 1 or E % D != 0:
+        raise CapmoeError(EINVAL, "capmoe_expanded_drop: E % D != 0")
+    m = E // D
+    W = (E + 63) // 64
+    if ws is None:
+        ws = torch.empty((drop_workspace_bytes(N, E, k, D, True),), device=dev, dtype=torch.uint8)
+    out = dict(keep_mask=torch.empty((N, W), device=dev, dtype=torch.int64),
+               cand=torch.empty((E,), device=dev, dtype=torch.int32),
+               kept=torch.empty((E,), device=dev, dtype=torch.int32),
+               offsets=torch.empty((E + 1,), device=dev, dtype=torch.int32),
+               slot_row=torch.empty((N, k + m), device=dev, dtype=torch.int32))
+    _check(lib().capmoe_expanded_drop(_ptr(scores), _ptr(topk_idx), _i64(N), int(E), int(k), _i64(C), int(D),
+                                      _ptr(token_group), _ptr(out["keep_mask"]), _ptr(out["cand"]),
+                                      _ptr(out["kept"]), _ptr(out["offsets"]), _ptr(out["slot_row"]), _ptr(ws),
+                                      ctypes.c_size_t(ws.numel()), _stream(stream)), "capmoe_expanded_drop")
+    return out
+
+
+def permute(x, scores, topk_idx, slot_row, A_max: int, D: int = 0, token_group=None, stream=None):
+    """-> dict(x_perm [A_max,d], perm_token [A_max], perm_weight [A_max]); rows >= A are left unwritten"""
+    N, d = x.shape
+    E = scores.shape[1]
+    k = topk_idx.shape[1]
+    slots = slot_row.shape[1]
+    dev = x.device
+    out = dict(x_perm=torch.zeros((A_max, d), device=dev, dtype=x.dtype),
+               perm_token=torch.full((A_max,), -1, device=dev, dtype=torch.int32),
+               perm_weight=torch.zeros((A_max,), device=dev, dtype=torch.float32))
+    _check(lib().capmoe_permute(_ptr(x), _i64(N), int(d), int(E), int(k), int(slots), int(D), _dt(x),
+                                _ptr(scores), _ptr(topk_idx), _ptr(token_group), _ptr(slot_row),
+                                _ptr(out["x_perm"]), _ptr(out["perm_token"]), _ptr(out["perm_weight"]),
+                                _stream(stream)), "capmoe_permute")
+    return out
+
+
+def grouped_ffn(x_perm, offsets, w_gate, w_up, w_down, D_straggler: int = 0, h_ws=None, y_perm=None,
+                dev_status=None, stream=None):
+    """-> y_perm [A_max, d]"""
+    A_max, d = x_perm.shape
+    E, F, _ = w_gate.shape
+    dev = x_perm.device
+    if h_ws is None:
+        h_ws = torch.empty((A_max, F), device=dev, dtype=x_perm.dtype)
+    if y_perm is None:
+        y_perm = torch.zeros((A_max, d), device=dev, dtype=x_perm.dtype)
+    _check(lib().capmoe_grouped_ffn(_ptr(x_perm), _ptr(offsets), int(E), int(d), int(F), _dt(x_perm),
+                                    _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(h_ws), _ptr(y_perm),
+                                    _i64(A_max), int(D_straggler), _ptr(dev_status), _stream(stream)),
+           "capmoe_grouped_ffn")
+    return y_perm
+
+
+def combine(y_perm, slot_row, perm_weight, y_shared=None, y=None, stream=None):
+    """-> y [N, d]"""
+    N, slots = slot_row.shape
+    d = y_perm.shape[1]
+    if y is None:
+        y = torch.empty((N, d), device=slot_row.device, dtype=y_perm.dtype)
+    _check(lib().capmoe_combine(_ptr(y_perm), _ptr(slot_row), _ptr(perm_weight), _i64(N), int(d), int(slots),
+                                _dt(y_perm), _ptr(y_shared), _ptr(y), _stream(stream)), "capmoe_combine")
+    return y
+
+
+# ----------------------------------------------------------------------------- whole layer
+class MoELayer:
+    """Device buffers for one layer plus the C struct that names them.  `forward()` enqueues
+    capmoe_layer_forward; `forward_host()` enqueues the host-buffer variant."""
+
+    def __init__(self, x, w_router, bias, w_gate, w_up, w_down, k: int, D: int, mode: str, gamma: float = 1.0,
+                 straggler: bool = False, shared=None, round_mode: str = "ceil", C: Optional[int] = None):
+        dev = x.device
+        N, d = x.shape
+        E, F, _ = w_gate.shape
+        self.N, self.d, self.E, self.k, self.F, self.D = N, d, E, k, F, D
+        self.mode = mode
+        m = E // D
+        expanded = mode == "expanded_drop"
+        if C is None:
+            C = N if mode == "nodrop" else capacity(N, E, k, gamma, round_mode)
+        self.C = C
+        self.slots = k + m if expanded else k
+        A_max = max_rows(N, E, k, D, C, expanded)
+        self.A_max = A_max
+        W = (E + 63) // 64
+        f32 = dict(device=dev, dtype=torch.float32)
+        i32 = dict(device=dev, dtype=torch.int32)
+        act = dict(device=dev, dtype=x.dtype)
+        t = self.t = {}
+        t["x"], t["w_router"], t["bias"] = x, w_router, bias
+        t["w_gate"], t["w_up"], t["w_down"] = w_gate, w_up, w_down
+        t["logits"] = torch.empty((N, E), **f32)
+        t["scores"] = torch.empty((N, E), **f32)
+        t["topk_idx"] = torch.empty((N, k), **i32)
+        t["topk_score"] = torch.empty((N, k), **f32)
+        t["load"] = torch.empty((E,), **i32)
+        t["keep_mask"] = torch.empty((N, W), device=dev, dtype=torch.int64)
+        t["cand"] = torch.zeros((E,), **i32)
+        t["kept"] = torch.empty((E,), **i32)
+        t["expert_offsets"] = torch.empty((E + 1,), **i32)
+        t["slot_row"] = torch.empty((N, self.slots), **i32)
+        t["x_perm"] = torch.zeros((max(A_max, 1), d), **act)
+        t["perm_token"] = torch.full((max(A_max, 1),), -1, **i32)
+        t["perm_weight"] = torch.zeros((max(A_max, 1),), **f32)
+        t["h_ws"] = torch.empty((max(A_max, 1), F), **act)
+        t["y_perm"] = torch.zeros((max(A_max, 1), d), **act)
+        t["y"] = torch.empty((N, d), **act)
+        t["drop_ws"] = torch.empty((drop_workspace_bytes(N, E, k, D, expanded),), device=dev, dtype=torch.uint8)
+        t["dev_status"] = torch.zeros((1,), **i32)
+        F_shared = 0
+        if shared is not None:
+            t["ws_gate"], t["ws_up"], t["ws_down"] = shared
+            F_shared = shared[0].shape[-2]
+            t["hs_ws"] = torch.empty((N, F_shared), **act)
+            t["y_shared"] = torch.empty((N, d), **act)
+            t["one_segment"] = torch.tensor([0, N], **i32)
+        L = self.c = _Layer()
+        L.N, L.d, L.E, L.k, L.F, L.D, L.dtype = N, d, E, k, F, D, _dt(x)
+        L.mode, L.C, L.straggler = MODES[mode], C, int(bool(straggler))
+        L.F_shared, L.A_max = F_shared, A_max
+        L.drop_ws_bytes = t["drop_ws"].numel()
+        for name, _typ in _Layer._fields_:
+            if name in t:
+                assert t[name].is_contiguous()
+                setattr(L, name, t[name].data_ptr())
+
+    def forward(self, stream=None):
+        _check(lib().capmoe_layer_forward(ctypes.byref(self.c), _stream(stream)), "capmoe_layer_forward")
+        return self.t["y"]
+
+    def forward_host(self, x_host: torch.Tensor, y_host: torch.Tensor, stream=None):
+        assert x_host.is_pinned() and y_host.is_pinned() and x_host.is_contiguous() and y_host.is_contiguous()
+        _check(lib().capmoe_layer_forward_host(ctypes.byref(self.c), ctypes.c_void_p(x_host.data_ptr()),
+                                               ctypes.c_void_p(y_host.data_ptr()), _stream(stream)),
+               "capmoe_layer_forward_host")
+        return y_host
+
+    def check_device_status(self):
+        s = int(self.t["dev_status"].item())
+        if s != OK:
+            raise CapmoeError(s, "device status")

@@ -1,0 +1,167 @@
+// Host side of the C ABI: helpers, the FFN dispatcher and the whole-layer entry points.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace capmoe {
+
+static std::atomic<uint64_t> g_launches{0};
+static thread_local char g_cuda_err[256] = "";
+
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+int note_cuda(cudaError_t err) {
+  if (err == cudaSuccess) return CAPMOE_OK;
+  std::snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", cudaGetErrorName(err), cudaGetErrorString(err));
+  return CAPMOE_ECUDA;
+}
+
+int check_launch() {
+  count_launch(1);
+  return note_cuda(cudaPeekAtLastError());
+}
+
+int sm_count() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+// defined in ffn_simt.cu / ffn_tc.cu
+int ffn_simt(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
+             const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
+             int64_t A_max, cudaStream_t st);
+bool ffn_tc_supported(int d, int F, int dtype);
+int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
+           const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
+           int32_t* dev_status, cudaStream_t st);
+
+}  // namespace capmoe
+
+using namespace capmoe;
+
+extern "C" int capmoe_capacity(int64_t N, int E, int k, double gamma, int round, int64_t* C) {
+  if (!C || N < 0 || E < 1 || k < 1 || k > E || !(gamma >= 0.0)) return CAPMOE_EINVAL;
+  if (round != CAPMOE_CAP_CEIL && round != CAPMOE_CAP_FLOOR) return CAPMOE_EINVAL;
+  double c;
+  if (std::isinf(gamma)) {
+    c = (double)N;
+  } else {
+    const double v = (gamma * (double)(N * (int64_t)k)) / (double)E;
+    c = round == CAPMOE_CAP_FLOOR ? std::floor(v) : std::ceil(v);
+  }
+  if (c > (double)N) c = (double)N;
+  if (c < 0.0) c = 0.0;
+  *C = (int64_t)c;
+  return CAPMOE_OK;
+}
+
+extern "C" int capmoe_max_rows(int64_t N, int E, int k, int D, int64_t C, int expanded, int64_t* A_max) {
+  if (!A_max || N < 0 || E < 1 || k < 1 || k > E || C < 0) return CAPMOE_EINVAL;
+  if (expanded && (D < 1 || E % D != 0)) return CAPMOE_EINVAL;
+  const int64_t cands = N * (int64_t)(expanded ? k + E / D : k);
+  const int64_t cap = (int64_t)E * (C > N ? N : C);
+  *A_max = cands < cap ? cands : cap;
+  return CAPMOE_OK;
+}
+
+extern "C" const char* capmoe_status_str(int status) {
+  switch (status) {
+    case CAPMOE_OK: return "ok";
+    case CAPMOE_EINVAL: return "invalid argument";
+    case CAPMOE_EUNSUPPORTED: return "unsupported dtype or shape";
+    case CAPMOE_EWORKSPACE: return "workspace too small";
+    case CAPMOE_ECUDA: return "CUDA error";
+    case CAPMOE_ETIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+extern "C" const char* capmoe_last_cuda_error(void) { return g_cuda_err; }
+extern "C" uint64_t capmoe_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+extern "C" int capmoe_ffn_uses_tensor_cores(int d, int F, int dtype) { return ffn_tc_supported(d, F, dtype) ? 1 : 0; }
+
+extern "C" int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F,
+                                  int dtype, const void* w_gate, const void* w_up, const void* w_down,
+                                  void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
+                                  int32_t* dev_status, void* stream) {
+  if (E < 1 || d < 1 || F < 1 || A_max < 0 || D_straggler < 0) return CAPMOE_EINVAL;
+  if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
+  if (D_straggler > 0 && E % D_straggler != 0) return CAPMOE_EINVAL;
+  if (E > 256) return CAPMOE_EUNSUPPORTED;
+  if (!expert_offsets) return CAPMOE_EINVAL;
+  if (A_max == 0) return CAPMOE_OK;
+  if (!x_perm || !w_gate || !w_up || !w_down || !h_ws || !y_perm) return CAPMOE_EINVAL;
+  if (!aligned16(x_perm) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) || !aligned16(h_ws) ||
+      !aligned16(y_perm))
+    return CAPMOE_EINVAL;
+  if (ffn_tc_supported(d, F, dtype))
+    return ffn_tc(x_perm, expert_offsets, E, d, F, w_gate, w_up, w_down, h_ws, y_perm, A_max, D_straggler,
+                  dev_status, as_stream(stream));
+  if (D_straggler > 0) return CAPMOE_EUNSUPPORTED;   // SM partitioning exists only in the tensor-core kernel
+  return ffn_simt(x_perm, expert_offsets, E, d, F, dtype, w_gate, w_up, w_down, h_ws, y_perm, A_max,
+                  as_stream(stream));
+}
+
+extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
+  if (!L) return CAPMOE_EINVAL;
+  if (L->mode < 0 || L->mode > 2) return CAPMOE_EINVAL;
+  int rc = capmoe_route(L->x, L->w_router, L->bias, nullptr, L->N, L->d, L->E, L->k, L->dtype, L->logits,
+                        L->scores, L->topk_idx, L->topk_score, L->load, stream);
+  if (rc != CAPMOE_OK) return rc;
+  int slots, Dp;
+  if (L->mode == 2) {
+    if (L->D < 1 || L->E % L->D != 0) return CAPMOE_EINVAL;
+    rc = capmoe_expanded_drop(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, nullptr, L->keep_mask,
+                              L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes,
+                              stream);
+    slots = L->k + L->E / L->D;
+    Dp = L->D;
+  } else {
+    rc = capmoe_token_drop(L->topk_score, L->topk_idx, L->N, L->E, L->k, L->mode == 0 ? L->N : L->C,
+                           L->keep_mask, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes,
+                           stream);
+    slots = L->k;
+    Dp = 0;
+  }
+  if (rc != CAPMOE_OK) return rc;
+  rc = capmoe_permute(L->x, L->N, L->d, L->E, L->k, slots, Dp, L->dtype, L->scores, L->topk_idx, nullptr,
+                      L->slot_row, L->x_perm, L->perm_token, L->perm_weight, stream);
+  if (rc != CAPMOE_OK) return rc;
+  rc = capmoe_grouped_ffn(L->x_perm, L->expert_offsets, L->E, L->d, L->F, L->dtype, L->w_gate, L->w_up,
+                          L->w_down, L->h_ws, L->y_perm, L->A_max, L->straggler ? L->D : 0, L->dev_status,
+                          stream);
+  if (rc != CAPMOE_OK) return rc;
+  const void* y_shared = nullptr;
+  if (L->F_shared > 0) {
+    if (!L->ws_gate || !L->ws_up || !L->ws_down || !L->hs_ws || !L->y_shared || !L->one_segment)
+      return CAPMOE_EINVAL;
+    rc = capmoe_grouped_ffn(L->x, L->one_segment, 1, L->d, L->F_shared, L->dtype, L->ws_gate, L->ws_up,
+                            L->ws_down, L->hs_ws, L->y_shared, L->N, 0, L->dev_status, stream);
+    if (rc != CAPMOE_OK) return rc;
+    y_shared = L->y_shared;
+  }
+  return capmoe_combine(L->y_perm, L->slot_row, L->perm_weight, L->N, L->d, slots, L->dtype, y_shared, L->y,
+                        stream);
+}
+
+extern "C" int capmoe_layer_forward_host(const capmoe_layer* L, const void* x_host, void* y_host, void* stream) {
+  if (!L || !x_host || !y_host) return CAPMOE_EINVAL;
+  const size_t bytes = (size_t)L->N * L->d * elt_size(L->dtype);
+  cudaStream_t st = as_stream(stream);
+  cudaError_t err = cudaMemcpyAsync(const_cast<void*>(L->x), x_host, bytes, cudaMemcpyHostToDevice, st);
+  if (err != cudaSuccess) return note_cuda(err);
+  int rc = capmoe_layer_forward(L, stream);
+  if (rc != CAPMOE_OK) return rc;
+  err = cudaMemcpyAsync(y_host, L->y, bytes, cudaMemcpyDeviceToHost, st);
+  return note_cuda(err);
+}

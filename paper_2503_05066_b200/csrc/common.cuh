@@ -1,0 +1,36 @@
+// Internal helpers of the capmoe CUDA library (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "capmoe.h"
+
+namespace capmoe {
+
+// Bookkeeping shared by the translation units (defined in api.cu).
+void count_launch(int n = 1);
+int note_cuda(cudaError_t err);            // records the text, returns CAPMOE_ECUDA or CAPMOE_OK
+int check_launch();                        // cudaPeekAtLastError -> status, counts one launch
+int sm_count();                            // SMs of the current device (cached per device)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t elt_size(int dtype) { return dtype == CAPMOE_F32 ? 4 : 2; }
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Home device of token t: explicit table, or contiguous blocks floor(t*D/N).
+__device__ __forceinline__ int home_group(int64_t t, int64_t N, int D, const int32_t* token_group) {
+  return token_group ? token_group[t] : (int)((t * (int64_t)D) / N);
+}
+
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_float(float v);
+template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) {
+  return __float2bfloat16_rn(v);
+}
+
+}  // namespace capmoe

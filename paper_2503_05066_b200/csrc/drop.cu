@@ -1,0 +1,328 @@
+// Stages 2 and 3: Capacity-Aware Token Drop (Eq. 7-10, Algorithm 1) and Expanded Drop
+// (Algorithm 2).  Both reduce to: per expert, list the candidate tokens in token order, find
+// the C-th largest score with a shared-memory radix select over the float bit patterns
+// (non-negative floats order like unsigned integers), and keep everything above it plus the
+// first (C - #above) candidates equal to it, in token order.
+#include "common.cuh"
+
+namespace capmoe {
+namespace {
+
+constexpr int CNT_THREADS = 256;
+constexpr int SEL_THREADS = 1024;
+constexpr int SEL_WARPS = SEL_THREADS / 32;
+constexpr int RADIX_BINS = 2048;     // 11 + 11 + 10 bits
+
+struct DropWs {
+  int32_t* cand;      // [E]   candidate counts (Token Drop only; Expanded Drop uses the caller's)
+  uint32_t* key;      // [cap] score bits of each candidate, expert-major, token order inside
+  int32_t* tok;       // [cap]
+  int32_t* slot;      // [cap]
+};
+
+inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+inline size_t ws_bytes_needed(int64_t N, int E, int k, int D, int expanded) {
+  int64_t cap = N * (int64_t)(expanded ? k + E / D : k);
+  return align256(sizeof(int32_t) * 256) + 3 * align256(sizeof(int32_t) * (size_t)cap);
+}
+
+inline DropWs carve(void* ws, int64_t N, int E, int k, int D, int expanded) {
+  int64_t cap = N * (int64_t)(expanded ? k + E / D : k);
+  char* p = (char*)ws;
+  DropWs w;
+  w.cand = (int32_t*)p; p += align256(sizeof(int32_t) * 256);
+  w.key = (uint32_t*)p; p += align256(sizeof(int32_t) * (size_t)cap);
+  w.tok = (int32_t*)p;  p += align256(sizeof(int32_t) * (size_t)cap);
+  w.slot = (int32_t*)p;
+  return w;
+}
+
+// Candidates per expert: |{t : e in topk(t)}| (+ |{t : h(t) = e/m, e not in topk(t)}| when EXPANDED).
+template <bool EXPANDED>
+__global__ void __launch_bounds__(CNT_THREADS)
+k_count_candidates(const int32_t* __restrict__ topk_idx, int64_t N, int E, int k, int D,
+                   const int32_t* __restrict__ token_group, int32_t* __restrict__ cand) {
+  extern __shared__ int hist[];
+  for (int i = threadIdx.x; i < E; i += CNT_THREADS) hist[i] = 0;
+  __syncthreads();
+  const int64_t t = (int64_t)blockIdx.x * CNT_THREADS + threadIdx.x;
+  if (t < N) {
+    const int32_t* row = topk_idx + t * k;
+    for (int j = 0; j < k; ++j) atomicAdd(&hist[row[j]], 1);
+    if (EXPANDED) {
+      const int m = E / D;
+      const int g = home_group(t, N, D, token_group);
+      for (int i = 0; i < m; ++i) {
+        const int e = g * m + i;
+        bool in = false;
+        for (int j = 0; j < k; ++j) in |= (row[j] == e);
+        if (!in) atomicAdd(&hist[e], 1);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < E; i += CNT_THREADS)
+    if (hist[i]) atomicAdd(&cand[i], hist[i]);
+}
+
+// Exclusive prefix sum over the block (SEL_THREADS threads).  total = sum of all v.
+__device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t* sh /*[SEL_WARPS+1]*/, uint32_t& total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  uint32_t incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) sh[wid] = incl;
+  __syncthreads();
+  if (wid == 0) {
+    uint32_t w = sh[lane];                       // SEL_WARPS == 32
+    uint32_t wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      uint32_t n = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += n;
+    }
+    sh[lane] = wi - w;
+    if (lane == 31) sh[SEL_WARPS] = wi;
+  }
+  __syncthreads();
+  const uint32_t res = incl - v + sh[wid];
+  total = sh[SEL_WARPS];
+  __syncthreads();                               // sh may be reused right away
+  return res;
+}
+
+// Among `nbins` histogram bins ordered from the highest digit down, find the bin that holds the
+// rank-th largest element (rank >= 1).  Result in out[0] = bin, out[1] = rank inside that bin.
+__device__ __forceinline__ void find_bin(const int* hist, int nbins, uint32_t rank, uint32_t* scan_sh,
+                                         uint32_t* out) {
+  const int p0 = 2 * threadIdx.x, p1 = p0 + 1;
+  const uint32_t h0 = p0 < nbins ? (uint32_t)hist[nbins - 1 - p0] : 0u;
+  const uint32_t h1 = p1 < nbins ? (uint32_t)hist[nbins - 1 - p1] : 0u;
+  uint32_t total;
+  const uint32_t before = block_scan(h0 + h1, scan_sh, total);
+  if (before < rank && rank <= before + h0) {
+    out[0] = (uint32_t)(nbins - 1 - p0); out[1] = rank - before;
+  } else if (before + h0 < rank && rank <= before + h0 + h1) {
+    out[0] = (uint32_t)(nbins - 1 - p1); out[1] = rank - before - h0;
+  }
+  __syncthreads();
+}
+
+// One CTA per expert.
+template <bool EXPANDED>
+__global__ void __launch_bounds__(SEL_THREADS)
+k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop) or scores [N,E] (Expanded)
+         const int32_t* __restrict__ topk_idx, int64_t N, int E, int k, int64_t C, int D,
+         const int32_t* __restrict__ token_group, const int32_t* __restrict__ cand, DropWs ws,
+         unsigned long long* __restrict__ keep_mask, int32_t* __restrict__ kept,
+         int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
+  __shared__ int hist[RADIX_BINS];
+  __shared__ uint32_t scan_sh[SEL_WARPS + 1];
+  __shared__ uint32_t found[2];
+  const int e = blockIdx.x;
+  const int tid = threadIdx.x;
+  const int m = EXPANDED ? E / D : 1;
+  const int slots = EXPANDED ? k + m : k;
+  const int W = (E + 63) >> 6;
+
+  // candidate base (prefix of cand) and row offset (prefix of min(cand, C)) of this expert
+  uint32_t base, off, total;
+  {
+    uint32_t c = (tid < E) ? (uint32_t)cand[tid] : 0u;      // E <= 256 <= SEL_THREADS
+    uint32_t kc = c < (uint32_t)C ? c : (uint32_t)C;
+    uint32_t b = block_scan(c, scan_sh, total);
+    uint32_t o = block_scan(kc, scan_sh, total);
+    if (tid == e) { found[0] = b; found[1] = o; }
+    __syncthreads();
+    base = found[0]; off = found[1];
+    __syncthreads();
+  }
+  const uint32_t n = (uint32_t)cand[e];
+  const uint32_t keep_n = n < (uint32_t)C ? n : (uint32_t)C;
+  if (tid == 0) {
+    kept[e] = (int32_t)keep_n;
+    expert_offsets[e] = (int32_t)off;
+    if (e == E - 1) expert_offsets[E] = (int32_t)(off + keep_n);
+  }
+  const bool need_select = n > keep_n;
+  for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) hist[i] = 0;
+  __syncthreads();
+
+  // pass 1: list this expert's candidates in token order; first-level histogram on the way
+  uint32_t* wkey = ws.key + base;
+  int32_t* wtok = ws.tok + base;
+  int32_t* wslot = ws.slot + base;
+  uint32_t running = 0;
+  for (int64_t t0 = 0; t0 < N; t0 += SEL_THREADS) {
+    const int64_t t = t0 + tid;
+    int slot = -1;
+    uint32_t key = 0;
+    if (t < N) {
+      const int32_t* row = topk_idx + t * k;
+      for (int j = 0; j < k; ++j)
+        if (row[j] == e) slot = j;
+      if (EXPANDED) {
+        if (slot < 0 && home_group(t, N, D, token_group) == e / m) slot = k + (e % m);
+        if (slot >= 0) key = __float_as_uint(score_src[t * E + e]);
+      } else {
+        if (slot >= 0) key = __float_as_uint(score_src[t * k + slot]);
+      }
+    }
+    uint32_t tot;
+    const uint32_t pos = block_scan(slot >= 0 ? 1u : 0u, scan_sh, tot);
+    if (slot >= 0) {
+      const uint32_t p = running + pos;
+      wkey[p] = key; wtok[p] = (int32_t)t; wslot[p] = slot;
+      if (need_select) atomicAdd(&hist[key >> 21], 1);
+    }
+    running += tot;
+  }
+  __syncthreads();   // list and histogram complete (block-visible: same CTA wrote them)
+
+  if (!need_select) {
+    for (uint32_t i = tid; i < n; i += SEL_THREADS) {
+      const int32_t t = wtok[i];
+      slot_row[(int64_t)t * slots + wslot[i]] = (int32_t)(off + i);
+      atomicOr(&keep_mask[(int64_t)t * W + (e >> 6)], 1ull << (e & 63));
+    }
+    return;
+  }
+
+  // radix select of the C-th largest key: 11, 11, 10 bits
+  uint32_t rank = (uint32_t)C;          // C >= 1 here would be needed; C == 0 handled below
+  uint32_t tau = 0, need = 0;
+  if (C > 0) {
+    find_bin(hist, RADIX_BINS, rank, scan_sh, found);
+    const uint32_t b1 = found[0]; rank = found[1];
+    __syncthreads();
+    for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    for (uint32_t i = tid; i < n; i += SEL_THREADS) {
+      const uint32_t key = wkey[i];
+      if ((key >> 21) == b1) atomicAdd(&hist[(key >> 10) & 2047u], 1);
+    }
+    __syncthreads();
+    find_bin(hist, RADIX_BINS, rank, scan_sh, found);
+    const uint32_t b2 = found[0]; rank = found[1];
+    __syncthreads();
+    for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = (b1 << 11) | b2;
+    for (uint32_t i = tid; i < n; i += SEL_THREADS) {
+      const uint32_t key = wkey[i];
+      if ((key >> 10) == prefix) atomicAdd(&hist[key & 1023u], 1);
+    }
+    __syncthreads();
+    find_bin(hist, 1024, rank, scan_sh, found);
+    tau = (prefix << 10) | found[0];
+    need = found[1];                     // how many candidates equal to tau are kept
+    __syncthreads();
+  }
+
+  // ordered pass: keep key > tau, and the first `need` with key == tau
+  uint32_t run_gt = 0, run_eq = 0;
+  for (uint32_t i0 = 0; i0 < n; i0 += SEL_THREADS) {
+    const uint32_t i = i0 + tid;
+    uint32_t key = 0;
+    bool gt = false, eq = false;
+    if (i < n && C > 0) {
+      key = wkey[i];
+      gt = key > tau; eq = key == tau;
+    }
+    uint32_t tot;
+    const uint32_t packed = block_scan((gt ? 1u : 0u) | (eq ? 0x10000u : 0u), scan_sh, tot);
+    if (i < n) {
+      const uint32_t gt_before = run_gt + (packed & 0xffffu);
+      const uint32_t eq_before = run_eq + (packed >> 16);
+      const bool keep = gt || (eq && eq_before < need);
+      const int32_t t = wtok[i];
+      int32_t row = -1;
+      if (keep) {
+        row = (int32_t)(off + gt_before + (eq_before < need ? eq_before : need));
+        atomicOr(&keep_mask[(int64_t)t * W + (e >> 6)], 1ull << (e & 63));
+      }
+      slot_row[(int64_t)t * slots + wslot[i]] = row;
+    }
+    run_gt += tot & 0xffffu;
+    run_eq += tot >> 16;
+  }
+}
+
+template <bool EXPANDED>
+int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C, int D,
+             const int32_t* token_group, uint64_t* keep_mask, int32_t* cand_out, int32_t* kept,
+             int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr, size_t ws_bytes, cudaStream_t st) {
+  const int W = (E + 63) / 64;
+  const int slots = EXPANDED ? k + E / D : k;
+  cudaError_t err;
+  if (N == 0) {
+    if ((err = cudaMemsetAsync(kept, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
+    if ((err = cudaMemsetAsync(expert_offsets, 0, sizeof(int32_t) * (E + 1), st)) != cudaSuccess) return note_cuda(err);
+    if (cand_out && (err = cudaMemsetAsync(cand_out, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
+    return CAPMOE_OK;
+  }
+  if (ws_bytes < ws_bytes_needed(N, E, k, D, EXPANDED ? 1 : 0)) return CAPMOE_EWORKSPACE;
+  DropWs ws = carve(ws_ptr, N, E, k, D, EXPANDED ? 1 : 0);
+  int32_t* cand = cand_out ? cand_out : ws.cand;
+  if ((err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
+  if ((err = cudaMemsetAsync(keep_mask, 0, sizeof(uint64_t) * N * W, st)) != cudaSuccess) return note_cuda(err);
+  if (EXPANDED) {   // local-expert slots that are already top-k slots are never written: preset -1
+    if ((err = cudaMemsetAsync(slot_row, 0xff, sizeof(int32_t) * N * slots, st)) != cudaSuccess) return note_cuda(err);
+  }
+  k_count_candidates<EXPANDED><<<(unsigned)ceil_div(N, CNT_THREADS), CNT_THREADS, sizeof(int) * E, st>>>(
+      topk_idx, N, E, k, D, token_group, cand);
+  int rc = check_launch();
+  if (rc != CAPMOE_OK) return rc;
+  k_select<EXPANDED><<<E, SEL_THREADS, 0, st>>>(score_src, topk_idx, N, E, k, C, D, token_group, cand, ws,
+                                                 (unsigned long long*)keep_mask, kept, expert_offsets, slot_row);
+  return check_launch();
+}
+
+int validate(int64_t N, int E, int k, int64_t C) {
+  if (N < 0 || E < 1 || k < 1 || k > E || C < 0 || C > N) return CAPMOE_EINVAL;
+  if (E > 256 || k > 32) return CAPMOE_EUNSUPPORTED;
+  return CAPMOE_OK;
+}
+
+}  // namespace
+}  // namespace capmoe
+
+using namespace capmoe;
+
+extern "C" int capmoe_drop_workspace_bytes(int64_t N, int E, int k, int D, int expanded, size_t* bytes) {
+  if (!bytes || N < 0 || E < 1 || k < 1 || k > E) return CAPMOE_EINVAL;
+  if (expanded && (D < 1 || E % D != 0)) return CAPMOE_EINVAL;
+  if (N * (int64_t)(expanded ? k + E / D : k) >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  *bytes = ws_bytes_needed(N, E, k, expanded ? D : 1, expanded);
+  return CAPMOE_OK;
+}
+
+extern "C" int capmoe_token_drop(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
+                                 int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
+                                 int32_t* slot_row, void* ws, size_t ws_bytes, void* stream) {
+  int rc = validate(N, E, k, C);
+  if (rc != CAPMOE_OK) return rc;
+  if (!kept || !expert_offsets) return CAPMOE_EINVAL;
+  if (N > 0 && (!topk_score || !topk_idx || !keep_mask || !slot_row || !ws)) return CAPMOE_EINVAL;
+  if (N * (int64_t)k >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  return run_drop<false>(topk_score, topk_idx, N, E, k, C, 1, nullptr, keep_mask, nullptr, kept,
+                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream));
+}
+
+extern "C" int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
+                                    int64_t C, int D, const int32_t* token_group, uint64_t* keep_mask,
+                                    int32_t* cand, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row,
+                                    void* ws, size_t ws_bytes, void* stream) {
+  int rc = validate(N, E, k, C);
+  if (rc != CAPMOE_OK) return rc;
+  if (D < 1 || E % D != 0) return CAPMOE_EINVAL;
+  if (!kept || !expert_offsets || !cand) return CAPMOE_EINVAL;
+  if (N > 0 && (!scores || !topk_idx || !keep_mask || !slot_row || !ws)) return CAPMOE_EINVAL;
+  if (N * (int64_t)(k + E / D) >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  return run_drop<true>(scores, topk_idx, N, E, k, C, D, token_group, keep_mask, cand, kept, expert_offsets,
+                        slot_row, ws, ws_bytes, as_stream(stream));
+}
