@@ -31,6 +31,9 @@ def _stale(obj: str, src: str) -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "capmoe.h"), __file__]
+    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= max(os.path.getmtime(p) for p in deps):
+        return LIB                       # up to date (object files need not exist: only the .so travels)
     objdir = os.path.join(PKG, "build")
     os.makedirs(objdir, exist_ok=True)
     nvcc = _nvcc()

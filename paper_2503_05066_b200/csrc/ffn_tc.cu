@@ -1,7 +1,425 @@
-// placeholder until the tensor-core kernel lands
+// Stage 5, tensor-core path: grouped SwiGLU expert FFN in bf16 on tcgen05 (5th-generation
+// tensor cores) with TMA-fed shared-memory tiles and fp32 accumulators in tensor memory.
+//
+// Two persistent, warp-specialised kernels per layer:
+//   GEMM1  H[r, f]  = silu(x_perm[r,:] . W_g[e,f,:]) * (x_perm[r,:] . W_u[e,f,:])
+//   GEMM2  y_perm[r, j] = H[r,:] . W_d[e,j,:]
+// Both operands of both GEMMs are K-major (row-major activations, [out,in] weights), so every
+// tile is loaded by TMA with the 128-byte swizzle and consumed by tcgen05.mma straight from
+// shared memory.  One CTA per SM:
+//   warp 0      TMA producer (one lane): ring of STAGES {A 128x64, B 256x64} bf16 tiles
+//   warp 1      MMA issuer (one lane): 128 x 256 x 16 tcgen05.mma, accumulators ping-pong
+//               between two 256-column halves of the CTA's 512 TMEM columns
+//   warps 2-5   epilogue: tcgen05.ld the finished accumulator, SwiGLU / convert, 16-byte stores,
+//               overlapping the next tile's MMAs
+// GEMM1 puts 128 gate rows and 128 up rows of the same output columns into one 256-row B tile,
+// so one MMA yields both halves of the SwiGLU pair.  Tiles are enumerated on the device from
+// expert_offsets (no host synchronisation); within an expert the row-block index runs fastest
+// so that concurrently running CTAs share weight tiles through L2.  In straggler-emulation mode
+// the CTAs are split into D equal groups and group g only serves the experts of virtual device g.
+// Every mbarrier wait is bounded; on expiry the CTA raises a flag, all roles drain and the
+// kernel reports CAPMOE_ETIMEOUT through dev_status.
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace capmoe {
-bool ffn_tc_supported(int, int, int) { return false; }
-int ffn_tc(const void*, const int32_t*, int, int, int, const void*, const void*, const void*, void*, void*,
-           int64_t, int, int32_t*, cudaStream_t) { return CAPMOE_EUNSUPPORTED; }
+namespace {
+
+constexpr int BM = 128;              // rows per tile (TMEM lanes)
+constexpr int BK = 64;               // K elements per stage: 128 bytes of bf16 = one swizzle row
+constexpr int BNB = 256;             // B rows per stage = MMA N
+constexpr int UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;         // 16 KB
+constexpr int B_BYTES = BNB * BK * 2;        // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int TC_THREADS = 192;
+constexpr int MAX_E = 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                           2 * (MAX_E + 1) * 4;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the wait ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1; it < 0x40000000u; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 127u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 bytes apart,
+// 8-row groups 1024 bytes apart (stride byte offset), descriptor version 1 (Blackwell).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffffu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
+  d |= (uint64_t)1 << 46;                            // version
+  d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor, kind::f16: D = fp32, A = B = bf16, both K-major, M = 128, N = 256.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BNB >> 3) << 17) |
+                           ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp gets row (lane base + i).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+// ---------------------------------------------------------------- tile enumeration
+struct Tile { int e, row0, rows, n0; };
+
+// tile_start[e] = first tile of expert e; tiles of an expert: row block fastest, then column block.
+__device__ __forceinline__ bool locate_tile(int tile, int& cursor, const int* tile_start, const int* offs, int E,
+                                            int n_tile, Tile& t) {
+  while (cursor < E && tile >= tile_start[cursor + 1]) ++cursor;
+  if (cursor >= E) return false;
+  const int local = tile - tile_start[cursor];
+  const int cnt = offs[cursor + 1] - offs[cursor];
+  const int nmb = (cnt + BM - 1) / BM;
+  const int nb = local / nmb, mb = local - nb * nmb;
+  t.e = cursor;
+  t.row0 = offs[cursor] + mb * BM;
+  t.rows = min(BM, cnt - mb * BM);
+  t.n0 = nb * n_tile;
+  return true;
+}
+
+// SWIGLU = true : B tile = 128 rows of W_g + 128 rows of W_u, output columns n0..n0+127 of H
+// SWIGLU = false: B tile = 256 rows of W_d, output columns n0..n0+255 of y_perm
+template <bool SWIGLU>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+         const __grid_constant__ CUtensorMap map_b1, const int32_t* __restrict__ expert_offsets, int E,
+         int K /* reduction length */, int Nout /* output columns */, __nv_bfloat16* __restrict__ out,
+         int D_straggler, int32_t* __restrict__ dev_status) {
+  constexpr int N_TILE = SWIGLU ? 128 : 256;
+  extern __shared__ uint8_t smem_raw[];
+  // carve: tiles (1024-byte aligned), barriers, expert tables
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + STAGES * STAGE_BYTES);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* offs = reinterpret_cast<int*>(gen + STAGES * STAGE_BYTES + 256);
+  int* tile_start = offs + (MAX_E + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * STAGES + 2 + b); };
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 128); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = tid; i <= E; i += TC_THREADS) offs[i] = expert_offsets[i];
+  __syncthreads();
+  if (tid == 0) {
+    const int n_blocks = (Nout + N_TILE - 1) / N_TILE;
+    int acc = 0;
+    for (int e = 0; e < E; ++e) {
+      tile_start[e] = acc;
+      acc += ((offs[e + 1] - offs[e] + BM - 1) / BM) * n_blocks;
+    }
+    tile_start[E] = acc;
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // this CTA's share of the tile list
+  int tile_lo, tile_hi, stride, first;
+  if (D_straggler > 0) {
+    const int per = gridDim.x / D_straggler;            // CTAs per virtual device
+    const int g = blockIdx.x / per;
+    if (g >= D_straggler) { tile_lo = tile_hi = 0; first = 0; stride = 1; }
+    else {
+      const int m = E / D_straggler;
+      tile_lo = tile_start[g * m]; tile_hi = tile_start[(g + 1) * m];
+      first = tile_lo + (blockIdx.x - g * per); stride = per;
+    }
+  } else {
+    tile_lo = 0; tile_hi = tile_start[E]; first = blockIdx.x; stride = gridDim.x;
+  }
+  const int num_kb = (K + BK - 1) / BK;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int cursor = 0;
+      uint32_t kc = 0;
+      Tile t;
+      bool ok = true;
+      for (int tile = first; ok && tile < tile_hi; tile += stride) {
+        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, t)) break;
+        for (int kb = 0; kb < num_kb; ++kb, ++kc) {
+          const int s = kc % STAGES;
+          const uint32_t ph = (kc / STAGES) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          const uint32_t a_dst = tiles + (uint32_t)s * STAGE_BYTES;
+          const uint32_t b_dst = a_dst + A_BYTES;
+          tma_load_2d(a_dst, &map_a, kb * BK, t.row0, full_bar(s));
+          if (SWIGLU) {
+            tma_load_3d(b_dst, &map_b0, kb * BK, t.n0, t.e, full_bar(s));
+            tma_load_3d(b_dst + B_BYTES / 2, &map_b1, kb * BK, t.n0, t.e, full_bar(s));
+          } else {
+            tma_load_3d(b_dst, &map_b0, kb * BK, t.n0, t.e, full_bar(s));
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int cursor = 0;
+      uint32_t kc = 0, it = 0;
+      Tile t;
+      bool ok = true;
+      for (int tile = first; ok && tile < tile_hi; tile += stride, ++it) {
+        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, t)) break;
+        const uint32_t b = it & 1u, use = it >> 1;
+        if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + b * (uint32_t)BNB;
+        for (int kb = 0; kb < num_kb; ++kb, ++kc) {
+          const int s = kc % STAGES;
+          const uint32_t ph = (kc / STAGES) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = tiles + (uint32_t)s * STAGE_BYTES;
+          const uint64_t adesc = umma_desc(a_src);
+          const uint64_t bdesc = umma_desc(a_src + A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advance 32 bytes (16 bf16) inside the swizzled 128-byte row: +2 in 16-byte units
+            umma(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(empty_bar(s));                    // frees the stage when these MMAs have read it
+        }
+        if (ok) umma_commit(tfull_bar(b));              // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
+    const int row_in_tile = quarter * 32 + lane;
+    int cursor = 0;
+    uint32_t it = 0;
+    Tile t;
+    for (int tile = first; tile < tile_hi; tile += stride, ++it) {
+      if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, t)) break;
+      const uint32_t b = it & 1u, use = it >> 1;
+      bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
+      ready = __all_sync(0xffffffffu, ready);            // warp-uniform: tcgen05.ld below is .sync.aligned
+      if (!ready) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)BNB;
+      const bool row_ok = row_in_tile < t.rows;
+      __nv_bfloat16* orow = out + (int64_t)(t.row0 + row_in_tile) * Nout + t.n0;
+#pragma unroll 1
+      for (int c = 0; c < N_TILE; c += 32) {
+        uint32_t g[32];
+        uint32_t packed[16];
+        if (SWIGLU) {
+          uint32_t u[32];
+          tmem_ld32(taddr + (uint32_t)c, g);
+          tmem_ld32(taddr + (uint32_t)(128 + c), u);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float g0 = __uint_as_float(g[2 * j]), g1 = __uint_as_float(g[2 * j + 1]);
+            const float u0 = __uint_as_float(u[2 * j]), u1 = __uint_as_float(u[2 * j + 1]);
+            const float h0 = __fdividef(g0, 1.0f + __expf(-g0)) * u0;
+            const float h1 = __fdividef(g1, 1.0f + __expf(-g1)) * u1;
+            packed[j] = pack_bf16(h0, h1);
+          }
+        } else {
+          tmem_ld32(taddr + (uint32_t)c, g);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            packed[j] = pack_bf16(__uint_as_float(g[2 * j]), __uint_as_float(g[2 * j + 1]));
+        }
+        if (row_ok) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (t.n0 + c + v * 8 + 8 <= Nout)
+              *reinterpret_cast<uint4*>(orow + c + v * 8) =
+                  make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty_bar(b));
+    }
+  }
+
+  // ------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+  if (tid == 0 && *abort_flag && dev_status) atomicExch(dev_status, (int)CAPMOE_ETIMEOUT);
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// bf16 tensor [rows, cols] (2D) or [batch, rows, cols] (3D), cols contiguous; box = box_rows x 64 columns.
+bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t batch, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {cols, rows, batch};
+  cuuint64_t strides[2] = {cols * 2, cols * rows * 2};
+  cuuint32_t box[3] = {(cuuint32_t)BK, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const cuuint32_t rank = batch > 0 ? 3 : 2;
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool ffn_tc_supported(int d, int F, int dtype) {
+  return dtype == CAPMOE_BF16 && d % 64 == 0 && F % 64 == 0 && d >= 64 && F >= 64;
+}
+
+int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
+           const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
+           int32_t* dev_status, cudaStream_t st) {
+  if (E > MAX_E) return CAPMOE_EUNSUPPORTED;
+  alignas(64) CUtensorMap a1, bg, bu, a2, bd;
+  if (!make_map(&a1, x_perm, (uint64_t)d, (uint64_t)A_max, 0, BM) ||
+      !make_map(&bg, w_gate, (uint64_t)d, (uint64_t)F, (uint64_t)E, 128) ||
+      !make_map(&bu, w_up, (uint64_t)d, (uint64_t)F, (uint64_t)E, 128) ||
+      !make_map(&a2, h_ws, (uint64_t)F, (uint64_t)A_max, 0, BM) ||
+      !make_map(&bd, w_down, (uint64_t)F, (uint64_t)d, (uint64_t)E, 256))
+    return note_cuda(cudaErrorInvalidValue);
+  cudaError_t err = cudaFuncSetAttribute(k_ffn_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (err != cudaSuccess) return note_cuda(err);
+  err = cudaFuncSetAttribute(k_ffn_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (err != cudaSuccess) return note_cuda(err);
+  int grid = sm_count();
+  if (D_straggler > 0) {
+    if (grid < D_straggler) return CAPMOE_EUNSUPPORTED;
+    grid = (grid / D_straggler) * D_straggler;          // equal share of SMs per virtual device
+  }
+  k_ffn_tc<true><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a1, bg, bu, expert_offsets, E, d, F,
+                                                      (__nv_bfloat16*)h_ws, D_straggler, dev_status);
+  int rc = check_launch();
+  if (rc != CAPMOE_OK) return rc;
+  k_ffn_tc<false><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a2, bd, bd, expert_offsets, E, F, d,
+                                                       (__nv_bfloat16*)y_perm, D_straggler, dev_status);
+  return check_launch();
+}
+
+}  // namespace capmoe
