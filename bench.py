@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the capacity-aware MoE layer forward (one step = one layer forward over one
+batch of synthetic tokens: route -> drop -> permute -> grouped SwiGLU FFN -> combine).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config mixtral] [--mode expanded_drop]
+                    [--gamma 1.0] [--no-straggler] [--no-sweep] [--impl reference]
+
+Prints ONE JSON line.  `value` is tokens/s of the whole job with the inputs resident in HBM;
+`e2e` is the same metric through the host-buffer entry point (pinned host activations copied
+in and out inside the timed region); `roofline` is for the dominant kernel (the gate/up
+tcgen05 GEMM with the SwiGLU epilogue); `cpu_baseline` is the CPU checker timed on a bounded
+sample of the same workload; `modes` lists the other routing modes of the same workload
+(no-drop, Token Drop, Expanded Drop, with and without straggler emulation).
+With --impl reference the CPU checker itself is the timed program.
+Under torchrun (N > 1) each rank runs the same per-GPU workload (weak scaling, no collective on
+the data path); times are device times, max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "MoE-layer tokens/s at Mixtral shape"
+UNIT = "tokens/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 100 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.rows = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [s.strip() for s in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        # "under load": the upper half of the power samples
+        cut = statistics.median(power)
+        loaded = [s for s, p in zip(sm, power) if p >= cut] or sm
+        return {"sm_mhz": statistics.median(loaded), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+def _to_np(t):
+    import numpy as np
+    import torch
+    t = t.detach().cpu().contiguous()
+    return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+
+
+def cpu_oracle_run(cfg, inp, mode: str, gamma: float, budget_tokens: int):
+    """The CPU checker on a bounded sample: routing and the drop over all N tokens, the expert FFN
+    and the combine for `budget_tokens` tokens spread over the batch.  Returns (tokens/s, detail)."""
+    import numpy as np
+    import oracle
+    x, wr, b = _to_np(inp.x), _to_np(inp.w_router), inp.bias.numpy()
+    t0 = time.perf_counter()
+    logits = oracle.router_logits(x, wr, b, cfg.dtype)
+    scores = oracle.softmax(logits)
+    idx, _, load = oracle.topk(scores, cfg.k)
+    C = cfg.N if mode == "nodrop" else oracle.capacity(cfg.N, cfg.E, cfg.k, gamma)
+    if mode == "expanded_drop":
+        r = oracle.expanded_drop(scores, idx, C, cfg.D)
+        Dp = cfg.D
+    else:
+        r = oracle.token_drop(scores, idx, C)
+        Dp = 0
+    t_route = time.perf_counter() - t0
+    toks = np.linspace(0, cfg.N - 1, budget_tokens).astype(np.int32)
+    t1 = time.perf_counter()
+    oracle.layer_tokens(x, toks, scores, idx, r["slot_row"], Dp, _to_np(inp.w_gate), _to_np(inp.w_up),
+                        _to_np(inp.w_down), cfg.dtype)
+    t_ffn = time.perf_counter() - t1
+    per_token = t_route / cfg.N + t_ffn / budget_tokens
+    return 1.0 / per_token, dict(route_drop_s_full_N=t_route, ffn_combine_s_sample=t_ffn,
+                                 sample_tokens=int(budget_tokens), cores=oracle.num_threads())
+
+
+def run_reference(args, rank):
+    """--impl reference: the CPU checker as it stands, on the host cores."""
+    from paper_2503_05066_b200 import synth
+    if rank != 0:
+        return
+    cfg = synth.CONFIGS[args.config]
+    inp = synth.make_layer_inputs(cfg)
+    sample = args.ref_tokens or 64
+    vals = []
+    for i in range(args.warmup + args.steps):
+        v, detail = cpu_oracle_run(cfg, inp, args.mode, args.gamma, sample)
+        if i >= args.warmup:
+            vals.append(v)
+    v = statistics.mean(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cfg.N / v, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": _config_dict(cfg, args),
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": detail["cores"], "kind": "oracle",
+                         "sample": f"router+drop on all {cfg.N} tokens, expert FFN+combine on {sample} tokens "
+                                   "spread over the batch; per-token times added"},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def _config_dict(cfg, args):
+    return {"workload": f"{cfg.name}: N={cfg.N} d={cfg.d} E={cfg.E} k={cfg.k} F={cfg.F} D={cfg.D} {cfg.dtype}",
+            "mode": args.mode, "gamma": args.gamma, "straggler_emulation": bool(args.straggler),
+            "l2": "expert weights (%.2f GB) are larger than L2, no flush needed" %
+                  (3 * cfg.E * cfg.d * cfg.F * (2 if cfg.dtype == "bf16" else 4) / 1e9),
+            "inputs": "hidden N(0,1); router N(0,1/d) + per-expert bias (%s); experts N(0,0.02); seed %d"
+                      % (cfg.bias_kind, cfg.seed)}
+
+
+def time_layer(layer, steps, warmup, torch, events=None):
+    """ms per step (device time, CUDA events on the launching stream)."""
+    for _ in range(warmup):
+        layer.forward()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        if events is not None:
+            layer.set_stage_events(events[i])
+        layer.forward()
+    e1.record()
+    torch.cuda.synchronize()
+    layer.set_stage_events(None)
+    layer.check_device_status()
+    return e0.elapsed_time(e1) / steps
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", default="mixtral")
+    ap.add_argument("--mode", default="expanded_drop", choices=["nodrop", "token_drop", "expanded_drop"])
+    ap.add_argument("--gamma", type=float, default=1.0)
+    ap.add_argument("--no-straggler", dest="straggler", action="store_false")
+    ap.add_argument("--no-sweep", dest="sweep", action="store_false", help="skip the other modes")
+    ap.add_argument("--no-cpu", dest="cpu", action="store_false", help="skip the CPU baseline")
+    ap.add_argument("--impl", default="capmoe", choices=["capmoe", "reference"])
+    ap.add_argument("--ref-tokens", type=int, default=None,
+                    help="tokens in the CPU checker's FFN sample (default 1024 for cpu_baseline, 64 per step "
+                         "for --impl reference)")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "capmoe":
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2503_05066_b200 import capmoe, synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    capmoe.lib()
+    peaks = _peaks()
+
+    cfg = synth.CONFIGS[args.config].with_(seed=synth.CONFIGS[args.config].seed + rank)
+    if not cfg.straggler:
+        args.straggler = args.straggler and False
+    inp = synth.make_layer_inputs(cfg)
+    dev = torch.device("cuda", local_rank)
+    g = {k: getattr(inp, k).to(dev) for k in ("x", "w_router", "bias", "w_gate", "w_up", "w_down")}
+    shared = None if inp.shared is None else tuple(s.to(dev) for s in inp.shared)
+
+    def make(mode, gamma, straggler):
+        return capmoe.MoELayer(g["x"], g["w_router"], g["bias"], g["w_gate"], g["w_up"], g["w_down"], cfg.k,
+                               cfg.D, mode, gamma=gamma, straggler=straggler, shared=shared)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v: float) -> float:
+        if world == 1:
+            return v
+        t = torch.tensor([v], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ------------------------------------------------------------------ headline: K timed steps
+    layer = make(args.mode, args.gamma, args.straggler)
+    K = args.steps
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(capmoe.N_STAGE_EVENTS)] for _ in range(K)]
+    for evs in events:
+        for e in evs:
+            e.record()                                   # creates the handles
+    for _ in range(args.warmup):
+        layer.forward()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = capmoe.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K):
+        layer.set_stage_events(events[i])
+        layer.forward()
+    e1.record()
+    barrier()
+    launches = capmoe.launch_count() - launches0
+    clocks = sampler.stop()
+    layer.set_stage_events(None)
+    layer.check_device_status()
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / K)
+    value = world * cfg.N / (ms_step * 1e-3)
+
+    stage_ms = {}
+    for si, name in enumerate(capmoe.STAGE_NAMES):
+        stage_ms[name] = statistics.mean(events[i][si].elapsed_time(events[i][si + 1]) for i in range(K))
+    A = int(layer.t["expert_offsets"][-1].item())
+    kept = layer.t["kept"].cpu().tolist()
+    load = layer.t["load"].cpu().tolist()
+
+    # ------------------------------------------------------------------ roofline of the dominant kernel
+    elt = 2 if cfg.dtype == "bf16" else 4
+    gemm1_flops = 4.0 * A * cfg.d * cfg.F                # 2 * A * d * (2F)
+    gemm2_flops = 2.0 * A * cfg.d * cfg.F
+    t1 = stage_ms["ffn_gate_up"] * 1e-3
+    t2 = stage_ms["ffn_down"] * 1e-3
+    use_tc = capmoe.ffn_uses_tensor_cores(cfg.d, cfg.F, g["x"].dtype)
+    peak_tf = peaks["bf16_tflops_sustained"] if use_tc else None
+    roofline = {
+        "kernel": "k_ffn_tc<SWIGLU> (gate/up grouped GEMM + SwiGLU, tcgen05)" if use_tc else "k_grouped_gemm (fp32 FMA)",
+        "bound": "tensor" if use_tc else "alu",
+        "achieved": gemm1_flops / t1 / 1e12 if t1 > 0 else None, "peak": peak_tf, "unit": "TFLOP/s",
+        "frac": (gemm1_flops / t1 / 1e12 / peak_tf) if (t1 > 0 and peak_tf) else None,
+        "peak_source": peaks["source"] + " (sustained cuBLAS bf16: kernel timed inside a long step)",
+        "peak_burst": peaks["bf16_tflops"],
+        "flops_per_launch": gemm1_flops,
+        "traffic": None,
+        "down_gemm": {"achieved": gemm2_flops / t2 / 1e12 if t2 > 0 else None,
+                      "frac": (gemm2_flops / t2 / 1e12 / peak_tf) if (t2 > 0 and peak_tf) else None},
+    }
+    # HBM-bound stages: algorithmic bytes over stage time
+    n_kept_tok = int((layer.t["keep_mask"] != 0).any(dim=1).sum().item())
+    slots = layer.slots
+    hbm = {
+        "route": (cfg.N * cfg.d * elt + cfg.E * cfg.d * elt + 2 * 4 * cfg.N * cfg.E + 8 * cfg.N * cfg.k),
+        "permute": (n_kept_tok * cfg.d * elt + A * cfg.d * elt + 8 * A + 4 * cfg.N * slots),
+        "combine": (A * cfg.d * elt + cfg.N * cfg.d * elt + 4 * A + 4 * cfg.N * slots),
+    }
+    hbm_stages = {k: {"bytes": v, "GB/s": v / (stage_ms[k] * 1e-3) / 1e9,
+                      "frac_of_measured_copy": v / (stage_ms[k] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                  for k, v in hbm.items() if stage_ms[k] > 0}
+
+    # ------------------------------------------------------------------ e2e through the host-buffer entry point
+    xh = inp.x.clone().pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    for _ in range(2):
+        layer.forward_host(xh, yh)
+    barrier()
+    e0.record()
+    for _ in range(K):
+        layer.forward_host(xh, yh)
+    e1.record()
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1) / K)
+    nbytes = xh.numel() * xh.element_size()
+    e2e = {"value": world * cfg.N / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+           "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes}
+    del layer
+
+    # ------------------------------------------------------------------ the other modes of the same workload
+    modes = []
+    if args.sweep and rank == 0:
+        sweep_steps = max(3, min(K, 10))
+        nodrop_ms = {}
+        for strag in ([False, True] if cfg.straggler else [False]):
+            for mode, gam in [("nodrop", None)] + [(m, gm) for gm in cfg.gammas for m in ("token_drop", "expanded_drop")]:
+                lay = make(mode, 1.0 if gam is None else gam, strag)
+                ms = time_layer(lay, sweep_steps, 3, torch)
+                if mode == "nodrop":
+                    nodrop_ms[strag] = ms
+                a = int(lay.t["expert_offsets"][-1].item())
+                modes.append({"mode": mode, "gamma": gam, "straggler_emulation": strag, "ms_per_layer": ms,
+                              "tokens_per_s": cfg.N / (ms * 1e-3), "A": a, "A_over_Nk": a / (cfg.N * cfg.k),
+                              "speedup_vs_nodrop": nodrop_ms[strag] / ms})
+                del lay
+
+    # ------------------------------------------------------------------ CPU baseline (rank 0, N = 1 only)
+    cpu = None
+    if args.cpu and rank == 0 and world == 1:
+        v, detail = cpu_oracle_run(cfg, inp, args.mode, args.gamma, args.ref_tokens or 1024)
+        cpu = {"value": v, "unit": UNIT, "cores": detail["cores"], "kind": "oracle",
+               "sample": f"router+drop on all {cfg.N} tokens ({detail['route_drop_s_full_N']:.2f} s), expert "
+                         f"FFN+combine on {detail['sample_tokens']} tokens spread over the batch "
+                         f"({detail['ffn_combine_s_sample']:.2f} s); per-token times added"}
+
+    if rank == 0:
+        nbar = cfg.N * cfg.k / cfg.E
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": cfg.dtype, "data": "synthetic", "config": _config_dict(cfg, args),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu,
+            "stages_ms": stage_ms, "hbm_stages": hbm_stages,
+            "workload_stats": {"A": A, "C": int(layer_C(cfg, args, capmoe)), "max_load_over_mean": max(load) / nbar,
+                               "kept_fraction_of_Nk": A / (cfg.N * cfg.k), "kept_per_expert": kept,
+                               "load_per_expert": load},
+            "modes": modes,
+            "peaks": peaks,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def layer_C(cfg, args, capmoe):
+    return cfg.N if args.mode == "nodrop" else capmoe.capacity(cfg.N, cfg.E, cfg.k, args.gamma)
+
+
+if __name__ == "__main__":
+    main()

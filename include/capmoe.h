@@ -183,7 +183,13 @@ typedef struct {
   void* y;
   void* drop_ws; size_t drop_ws_bytes;
   int32_t* dev_status;
+  /* Optional stage timing.  NULL, or CAPMOE_N_STAGE_EVENTS cudaEvent_t handles (as void*) that the
+   * layer records on `stream`: [0] start, [1] after route, [2] after drop, [3] after permute,
+   * [4] after the gate/up GEMM + SwiGLU, [5] after the down GEMM, [6] after the shared expert,
+   * [7] after combine. */
+  void** stage_events;
 } capmoe_layer;
+#define CAPMOE_N_STAGE_EVENTS 8
 
 /* Runs the stages above in order on `stream` (route, drop, permute, FFN, [shared FFN], combine). */
 int capmoe_layer_forward(const capmoe_layer* L, void* stream);

@@ -57,7 +57,11 @@ class _Layer(ctypes.Structure):
         ("y", ctypes.c_void_p),
         ("drop_ws", ctypes.c_void_p), ("drop_ws_bytes", ctypes.c_size_t),
         ("dev_status", ctypes.c_void_p),
+        ("stage_events", ctypes.POINTER(ctypes.c_void_p)),
     ]
+
+N_STAGE_EVENTS = 8
+STAGE_NAMES = ["route", "drop", "permute", "ffn_gate_up", "ffn_down", "shared_ffn", "combine"]
 
 
 def lib():
@@ -303,6 +307,17 @@ class MoELayer:
             if name in t:
                 assert t[name].is_contiguous()
                 setattr(L, name, t[name].data_ptr())
+
+    def set_stage_events(self, events):
+        """events: None, or N_STAGE_EVENTS recorded torch.cuda.Event(enable_timing=True) objects."""
+        if events is None:
+            self.c.stage_events = ctypes.POINTER(ctypes.c_void_p)()
+            self._ev = None
+            return
+        assert len(events) == N_STAGE_EVENTS
+        arr = (ctypes.c_void_p * N_STAGE_EVENTS)(*[ctypes.c_void_p(e.cuda_event) for e in events])
+        self._ev = (arr, events)
+        self.c.stage_events = ctypes.cast(arr, ctypes.POINTER(ctypes.c_void_p))
 
     def forward(self, stream=None):
         _check(lib().capmoe_layer_forward(ctypes.byref(self.c), _stream(stream)), "capmoe_layer_forward")

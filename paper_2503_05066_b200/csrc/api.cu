@@ -39,11 +39,32 @@ int sm_count() {
 // defined in ffn_simt.cu / ffn_tc.cu
 int ffn_simt(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
              const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
-             int64_t A_max, cudaStream_t st);
+             int64_t A_max, cudaEvent_t mid, cudaStream_t st);
 bool ffn_tc_supported(int d, int F, int dtype);
 int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
            const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
-           int32_t* dev_status, cudaStream_t st);
+           int32_t* dev_status, cudaEvent_t mid, cudaStream_t st);
+
+static int grouped_ffn_impl(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
+                            const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
+                            int64_t A_max, int D_straggler, int32_t* dev_status, cudaEvent_t mid, void* stream) {
+  if (E < 1 || d < 1 || F < 1 || A_max < 0 || D_straggler < 0) return CAPMOE_EINVAL;
+  if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
+  if (D_straggler > 0 && E % D_straggler != 0) return CAPMOE_EINVAL;
+  if (E > 256) return CAPMOE_EUNSUPPORTED;
+  if (!expert_offsets) return CAPMOE_EINVAL;
+  if (A_max == 0) return CAPMOE_OK;
+  if (!x_perm || !w_gate || !w_up || !w_down || !h_ws || !y_perm) return CAPMOE_EINVAL;
+  if (!aligned16(x_perm) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) || !aligned16(h_ws) ||
+      !aligned16(y_perm))
+    return CAPMOE_EINVAL;
+  if (ffn_tc_supported(d, F, dtype))
+    return ffn_tc(x_perm, expert_offsets, E, d, F, w_gate, w_up, w_down, h_ws, y_perm, A_max, D_straggler,
+                  dev_status, mid, as_stream(stream));
+  if (D_straggler > 0) return CAPMOE_EUNSUPPORTED;   // SM partitioning exists only in the tensor-core kernel
+  return ffn_simt(x_perm, expert_offsets, E, d, F, dtype, w_gate, w_up, w_down, h_ws, y_perm, A_max, mid,
+                  as_stream(stream));
+}
 
 }  // namespace capmoe
 
@@ -94,30 +115,24 @@ extern "C" int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offs
                                   int dtype, const void* w_gate, const void* w_up, const void* w_down,
                                   void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
                                   int32_t* dev_status, void* stream) {
-  if (E < 1 || d < 1 || F < 1 || A_max < 0 || D_straggler < 0) return CAPMOE_EINVAL;
-  if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
-  if (D_straggler > 0 && E % D_straggler != 0) return CAPMOE_EINVAL;
-  if (E > 256) return CAPMOE_EUNSUPPORTED;
-  if (!expert_offsets) return CAPMOE_EINVAL;
-  if (A_max == 0) return CAPMOE_OK;
-  if (!x_perm || !w_gate || !w_up || !w_down || !h_ws || !y_perm) return CAPMOE_EINVAL;
-  if (!aligned16(x_perm) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) || !aligned16(h_ws) ||
-      !aligned16(y_perm))
-    return CAPMOE_EINVAL;
-  if (ffn_tc_supported(d, F, dtype))
-    return ffn_tc(x_perm, expert_offsets, E, d, F, w_gate, w_up, w_down, h_ws, y_perm, A_max, D_straggler,
-                  dev_status, as_stream(stream));
-  if (D_straggler > 0) return CAPMOE_EUNSUPPORTED;   // SM partitioning exists only in the tensor-core kernel
-  return ffn_simt(x_perm, expert_offsets, E, d, F, dtype, w_gate, w_up, w_down, h_ws, y_perm, A_max,
-                  as_stream(stream));
+  return grouped_ffn_impl(x_perm, expert_offsets, E, d, F, dtype, w_gate, w_up, w_down, h_ws, y_perm, A_max,
+                          D_straggler, dev_status, nullptr, stream);
 }
 
 extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if (!L) return CAPMOE_EINVAL;
   if (L->mode < 0 || L->mode > 2) return CAPMOE_EINVAL;
-  int rc = capmoe_route(L->x, L->w_router, L->bias, nullptr, L->N, L->d, L->E, L->k, L->dtype, L->logits,
-                        L->scores, L->topk_idx, L->topk_score, L->load, stream);
+  cudaStream_t st = as_stream(stream);
+  auto mark = [&](int i) -> int {
+    if (!L->stage_events) return CAPMOE_OK;
+    return note_cuda(cudaEventRecord((cudaEvent_t)L->stage_events[i], st));
+  };
+  int rc = mark(0);
   if (rc != CAPMOE_OK) return rc;
+  rc = capmoe_route(L->x, L->w_router, L->bias, nullptr, L->N, L->d, L->E, L->k, L->dtype, L->logits,
+                    L->scores, L->topk_idx, L->topk_score, L->load, stream);
+  if (rc != CAPMOE_OK) return rc;
+  if ((rc = mark(1)) != CAPMOE_OK) return rc;
   int slots, Dp;
   if (L->mode == 2) {
     if (L->D < 1 || L->E % L->D != 0) return CAPMOE_EINVAL;
@@ -134,24 +149,31 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
     Dp = 0;
   }
   if (rc != CAPMOE_OK) return rc;
+  if ((rc = mark(2)) != CAPMOE_OK) return rc;
   rc = capmoe_permute(L->x, L->N, L->d, L->E, L->k, slots, Dp, L->dtype, L->scores, L->topk_idx, nullptr,
                       L->slot_row, L->x_perm, L->perm_token, L->perm_weight, stream);
   if (rc != CAPMOE_OK) return rc;
-  rc = capmoe_grouped_ffn(L->x_perm, L->expert_offsets, L->E, L->d, L->F, L->dtype, L->w_gate, L->w_up,
-                          L->w_down, L->h_ws, L->y_perm, L->A_max, L->straggler ? L->D : 0, L->dev_status,
-                          stream);
+  if ((rc = mark(3)) != CAPMOE_OK) return rc;
+  rc = grouped_ffn_impl(L->x_perm, L->expert_offsets, L->E, L->d, L->F, L->dtype, L->w_gate, L->w_up, L->w_down,
+                        L->h_ws, L->y_perm, L->A_max, L->straggler ? L->D : 0, L->dev_status,
+                        L->stage_events ? (cudaEvent_t)L->stage_events[4] : nullptr, stream);
   if (rc != CAPMOE_OK) return rc;
+  if (L->A_max == 0 && (rc = mark(4)) != CAPMOE_OK) return rc;
+  if ((rc = mark(5)) != CAPMOE_OK) return rc;
   const void* y_shared = nullptr;
   if (L->F_shared > 0) {
     if (!L->ws_gate || !L->ws_up || !L->ws_down || !L->hs_ws || !L->y_shared || !L->one_segment)
       return CAPMOE_EINVAL;
-    rc = capmoe_grouped_ffn(L->x, L->one_segment, 1, L->d, L->F_shared, L->dtype, L->ws_gate, L->ws_up,
-                            L->ws_down, L->hs_ws, L->y_shared, L->N, 0, L->dev_status, stream);
+    rc = grouped_ffn_impl(L->x, L->one_segment, 1, L->d, L->F_shared, L->dtype, L->ws_gate, L->ws_up, L->ws_down,
+                          L->hs_ws, L->y_shared, L->N, 0, L->dev_status, nullptr, stream);
     if (rc != CAPMOE_OK) return rc;
     y_shared = L->y_shared;
   }
-  return capmoe_combine(L->y_perm, L->slot_row, L->perm_weight, L->N, L->d, slots, L->dtype, y_shared, L->y,
-                        stream);
+  if ((rc = mark(6)) != CAPMOE_OK) return rc;
+  rc = capmoe_combine(L->y_perm, L->slot_row, L->perm_weight, L->N, L->d, slots, L->dtype, y_shared, L->y,
+                      stream);
+  if (rc != CAPMOE_OK) return rc;
+  return mark(7);
 }
 
 extern "C" int capmoe_layer_forward_host(const capmoe_layer* L, const void* x_host, void* y_host, void* stream) {

@@ -101,13 +101,14 @@ k_grouped_gemm(const T* __restrict__ A, const int32_t* __restrict__ expert_offse
 
 template <typename T>
 int run(const T* x_perm, const int32_t* expert_offsets, int E, int d, int F, const T* wg, const T* wu,
-        const T* wd, T* h, T* y, int64_t A_max, cudaStream_t st) {
+        const T* wd, T* h, T* y, int64_t A_max, cudaEvent_t mid, cudaStream_t st) {
   const unsigned slots = (unsigned)(ceil_div(A_max, TS) + E);
   if (slots > 65535u) return CAPMOE_EUNSUPPORTED;
   k_grouped_gemm<T, true><<<dim3((unsigned)ceil_div(F, TS), slots), NT, 0, st>>>(x_perm, expert_offsets, E, d, F,
                                                                                 wg, wu, h);
   int rc = check_launch();
   if (rc != CAPMOE_OK) return rc;
+  if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
   k_grouped_gemm<T, false><<<dim3((unsigned)ceil_div(d, TS), slots), NT, 0, st>>>(h, expert_offsets, E, F, d, wd,
                                                                                  nullptr, y);
   return check_launch();
@@ -117,13 +118,13 @@ int run(const T* x_perm, const int32_t* expert_offsets, int E, int d, int F, con
 
 int ffn_simt(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
              const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
-             int64_t A_max, cudaStream_t st) {
+             int64_t A_max, cudaEvent_t mid, cudaStream_t st) {
   if (dtype == CAPMOE_F32)
     return run<float>((const float*)x_perm, expert_offsets, E, d, F, (const float*)w_gate, (const float*)w_up,
-                      (const float*)w_down, (float*)h_ws, (float*)y_perm, A_max, st);
+                      (const float*)w_down, (float*)h_ws, (float*)y_perm, A_max, mid, st);
   return run<__nv_bfloat16>((const __nv_bfloat16*)x_perm, expert_offsets, E, d, F, (const __nv_bfloat16*)w_gate,
                             (const __nv_bfloat16*)w_up, (const __nv_bfloat16*)w_down, (__nv_bfloat16*)h_ws,
-                            (__nv_bfloat16*)y_perm, A_max, st);
+                            (__nv_bfloat16*)y_perm, A_max, mid, st);
 }
 
 }  // namespace capmoe

@@ -395,7 +395,7 @@ bool ffn_tc_supported(int d, int F, int dtype) {
 
 int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
            const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
-           int32_t* dev_status, cudaStream_t st) {
+           int32_t* dev_status, cudaEvent_t mid, cudaStream_t st) {
   if (E > MAX_E) return CAPMOE_EUNSUPPORTED;
   alignas(64) CUtensorMap a1, bg, bu, a2, bd;
   if (!make_map(&a1, x_perm, (uint64_t)d, (uint64_t)A_max, 0, BM) ||
@@ -417,6 +417,7 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
                                                       (__nv_bfloat16*)h_ws, D_straggler, dev_status);
   int rc = check_launch();
   if (rc != CAPMOE_OK) return rc;
+  if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
   k_ffn_tc<false><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a2, bd, bd, expert_offsets, E, F, d,
                                                        (__nv_bfloat16*)y_perm, D_straggler, dev_status);
   return check_launch();
