@@ -104,6 +104,26 @@ int capmoe_token_drop(const float* topk_score, const int32_t* topk_idx, int64_t 
                       int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
                       int32_t* slot_row, void* ws, size_t ws_bytes, void* stream);
 
+/* Token Drop without caller-provided scratch.  The paper has no counterpart: this entry point
+ * exists for callers that can neither allocate device memory nor carve a workspace out of memory
+ * they own - a serving runtime whose memory pool is fixed at start-up, a host that forbids
+ * allocation after initialisation, or a language binding that only holds the input and output
+ * tensors.  Same inputs, outputs and results as capmoe_token_drop; the scratch is a fixed array in
+ * device memory that the library owns (about 12 MiB on every GPU that loads the library, held
+ * until the process exits).
+ *   - Limit: N*k <= CAPMOE_STATIC_DROP_MAX_PAIRS; larger calls return CAPMOE_EWORKSPACE and
+ *     launch nothing.
+ *   - It calls no cudaMalloc/cudaFree and no allocating library routine.  The first call on each
+ *     device looks up the array's device address (the device must be current); make that first
+ *     call outside of any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents: the
+ *     call clears the part that has to start at zero itself, but two calls that overlap on the
+ *     GPU (different streams, or several host threads) race on it.  Serialise them. */
+#define CAPMOE_STATIC_DROP_MAX_PAIRS (1 << 20)
+int capmoe_token_drop_static(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
+                             int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
+                             int32_t* slot_row, void* stream);
+
 /* ---------------------------------------------------------------- stage 3: Expanded Drop
  * Token t is a candidate of its top-k experts and of all m = E/D experts of its home device
  * h(t); all candidates of an expert compete on scores[t,e]; the expert keeps its C best, ties

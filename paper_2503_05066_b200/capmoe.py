@@ -25,7 +25,7 @@ MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2}
 
 EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_drop_workspace_bytes", "capmoe_status_str",
            "capmoe_last_cuda_error", "capmoe_launch_count", "capmoe_ffn_uses_tensor_cores", "capmoe_route",
-           "capmoe_token_drop", "capmoe_expanded_drop", "capmoe_permute", "capmoe_grouped_ffn",
+           "capmoe_token_drop", "capmoe_token_drop_static", "capmoe_expanded_drop", "capmoe_permute", "capmoe_grouped_ffn",
            "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host"]
 
 
@@ -175,6 +175,30 @@ def token_drop(topk_score, topk_idx, E: int, C: int, ws=None, stream=None):
                                    _ptr(out["keep_mask"]), _ptr(out["kept"]), _ptr(out["offsets"]),
                                    _ptr(out["slot_row"]), _ptr(ws), ctypes.c_size_t(ws.numel()),
                                    _stream(stream)), "capmoe_token_drop")
+    return out
+
+
+STATIC_DROP_MAX_PAIRS = 1 << 20
+
+
+def token_drop_static(topk_score, topk_idx, E: int, C: int, stream=None):
+    """Token Drop through the entry point that needs no workspace from the caller (the scratch
+    is a fixed array inside the library, shared by all calls on the device: do not overlap calls).
+    Limited to N*k <= STATIC_DROP_MAX_PAIRS.  -> dict(keep_mask, kept, offsets, slot_row)"""
+    N, k = topk_idx.shape
+    dev = topk_idx.device
+    W = (E + 63) // 64
+    out = dict(keep_mask=torch.empty((N, W), device=dev, dtype=torch.int64),
+               kept=torch.empty((E,), device=dev, dtype=torch.int32),
+               offsets=torch.empty((E + 1,), device=dev, dtype=torch.int32),
+               slot_row=torch.empty((N, k), device=dev, dtype=torch.int32))
+    rc = lib().capmoe_token_drop_static(_ptr(topk_score), _ptr(topk_idx), _i64(N), int(E), int(k), _i64(C),
+                                        _ptr(out["keep_mask"]), _ptr(out["kept"]), _ptr(out["offsets"]),
+                                        _ptr(out["slot_row"]), _stream(stream))
+    if rc == EWORKSPACE:
+        raise CapmoeError(rc, f"capmoe_token_drop_static: N*k = {N * k} exceeds the built-in scratch "
+                              f"({STATIC_DROP_MAX_PAIRS} pairs)")
+    _check(rc, "capmoe_token_drop_static")
     return out
 
 

@@ -3,6 +3,8 @@
 // the C-th largest score with a shared-memory radix select over the float bit patterns
 // (non-negative floats order like unsigned integers), and keep everything above it plus the
 // first (C - #above) candidates equal to it, in token order.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace capmoe {
@@ -325,4 +327,62 @@ extern "C" int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx
   if (N * (int64_t)(k + E / D) >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
   return run_drop<true>(scores, topk_idx, N, E, k, C, D, token_group, keep_mask, cand, kept, expert_offsets,
                         slot_row, ws, ws_bytes, as_stream(stream));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Token Drop for callers that cannot provide scratch memory (see capmoe_token_drop_static in the
+// header).  The scratch lives in a fixed array in device memory that belongs to the library.
+namespace capmoe {
+namespace {
+
+constexpr int64_t STATIC_MAX_PAIRS = CAPMOE_STATIC_DROP_MAX_PAIRS;
+// same layout as carve(): 256 counters, then three int32 lists of STATIC_MAX_PAIRS entries
+constexpr size_t STATIC_WS_BYTES = 256 * sizeof(int32_t) + 3 * sizeof(int32_t) * (size_t)STATIC_MAX_PAIRS;
+static_assert((sizeof(int32_t) * (size_t)STATIC_MAX_PAIRS) % 256 == 0, "lists must stay 256-byte aligned");
+
+static __device__ __align__(256) unsigned char g_static_drop_ws[STATIC_WS_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+static void* g_static_ws_addr[MAX_DEVICES];      // device address of the array, per device ordinal
+static bool g_static_ws_ready[MAX_DEVICES];
+static std::mutex g_static_ws_mutex;
+
+// In host code `g_static_drop_ws` is only a handle; the address a kernel can use has to be asked
+// for, once per device, while that device is current.
+int static_ws_for_current_device(void** out) {
+  int dev = -1;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return note_cuda(err);
+  if (dev < 0 || dev >= MAX_DEVICES) return CAPMOE_EUNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+  if (!g_static_ws_ready[dev]) {
+    void* p = nullptr;
+    err = cudaGetSymbolAddress(&p, g_static_drop_ws);
+    if (err != cudaSuccess) return note_cuda(err);
+    if (!p) return note_cuda(cudaErrorInvalidSymbol);
+    g_static_ws_addr[dev] = p;
+    g_static_ws_ready[dev] = true;
+  }
+  *out = g_static_ws_addr[dev];
+  return CAPMOE_OK;
+}
+
+}  // namespace
+}  // namespace capmoe
+
+extern "C" int capmoe_token_drop_static(const float* topk_score, const int32_t* topk_idx, int64_t N, int E,
+                                        int k, int64_t C, uint64_t* keep_mask, int32_t* kept,
+                                        int32_t* expert_offsets, int32_t* slot_row, void* stream) {
+  int rc = validate(N, E, k, C);
+  if (rc != CAPMOE_OK) return rc;
+  if (!kept || !expert_offsets) return CAPMOE_EINVAL;
+  if (N > 0 && (!topk_score || !topk_idx || !keep_mask || !slot_row)) return CAPMOE_EINVAL;
+  if (N * (int64_t)k > STATIC_MAX_PAIRS) return CAPMOE_EWORKSPACE;   // beyond the built-in scratch
+  void* ws = nullptr;
+  rc = static_ws_for_current_device(&ws);
+  if (rc != CAPMOE_OK) return rc;
+  // run_drop zeroes the candidate counters itself; the three lists are fully rewritten before
+  // they are read, so nothing else of the previous call's contents matters.
+  return run_drop<false>(topk_score, topk_idx, N, E, k, C, 1, nullptr, keep_mask, nullptr, kept,
+                         expert_offsets, slot_row, ws, STATIC_WS_BYTES, as_stream(stream));
 }
