@@ -88,30 +88,44 @@ k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row
   const int64_t t = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
   if (t >= N) return;
   const int32_t* sr = slot_row + t * slots;
-  for (int v0 = 0; v0 < row_vecs; v0 += 32) {
-    const int v = v0 + lane;
-    float acc[NV];
+  constexpr int VPL = 4;                               // 16-byte vectors per lane in flight per row
+  for (int v0 = 0; v0 < row_vecs; v0 += 32 * VPL) {
+    float acc[VPL][NV];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) acc[i] = 0.f;
-    if (y_shared && v < row_vecs) Vec16<T>::load(y_shared[t * row_vecs + v], acc);
+    for (int u = 0; u < VPL; ++u) {
+      const int v = v0 + u * 32 + lane;
+#pragma unroll
+      for (int i = 0; i < NV; ++i) acc[u][i] = 0.f;
+      if (y_shared && v < row_vecs) Vec16<T>::load(y_shared[t * row_vecs + v], acc[u]);
+    }
     for (int s0 = 0; s0 < slots; s0 += 32) {
       const int32_t mine = (s0 + lane < slots) ? sr[s0 + lane] : -1;
       const float wmine = mine >= 0 ? perm_weight[mine] : 0.f;
       unsigned rem = __ballot_sync(0xffffffffu, mine >= 0);
-      while (rem) {                                  // ascending slot order
+      while (rem) {                                    // ascending slot order
         const int b = __ffs(rem) - 1;
         rem &= rem - 1;
         const int32_t r = __shfl_sync(0xffffffffu, mine, b);
         const float wgt = __shfl_sync(0xffffffffu, wmine, b);
-        if (v < row_vecs) {
-          float f[NV];
-          Vec16<T>::load(y_perm[(int64_t)r * row_vecs + v], f);
+        const uint4* src = y_perm + (int64_t)r * row_vecs + v0 + lane;
+        uint4 raw[VPL];
 #pragma unroll
-          for (int i = 0; i < NV; ++i) acc[i] = fmaf(wgt, f[i], acc[i]);
+        for (int u = 0; u < VPL; ++u)                  // independent loads first, arithmetic after
+          raw[u] = (v0 + u * 32 + lane < row_vecs) ? __ldcs(src + u * 32) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < VPL; ++u) {
+          float f[NV];
+          Vec16<T>::load(raw[u], f);
+#pragma unroll
+          for (int i = 0; i < NV; ++i) acc[u][i] = fmaf(wgt, f[i], acc[u][i]);
         }
       }
     }
-    if (v < row_vecs) y[t * row_vecs + v] = Vec16<T>::store(acc);
+#pragma unroll
+    for (int u = 0; u < VPL; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < row_vecs) y[t * row_vecs + v] = Vec16<T>::store(acc[u]);
+    }
   }
 }
 

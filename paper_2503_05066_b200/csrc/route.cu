@@ -154,6 +154,129 @@ int launch_gemm(const T* x, const T* w, const float* bias, int64_t N, int d, int
   return check_launch();
 }
 
+// ---------------------------------------------------------------------------------------------
+// bf16 router GEMM, bandwidth-bound form.  The stage has to read X exactly once at HBM speed, so
+// X fragments go from global memory straight into tensor-core registers with 16-byte loads:
+// a CTA owns 16*MT tokens, its 8 warps split the d columns (split-K), each warp runs
+// mma.m16n8k16 (bf16 x bf16 -> fp32) over its column range and the 8 partial sums are added in
+// warp order through shared memory (a fixed order, so logits are reproducible).
+// The k index inside an MMA is only a summation index, so each thread takes its 8 consecutive
+// columns of X (one 16-byte load) as the k slots it owns in two MMAs, and loads the same 8
+// columns of W_r for its B fragment; no shared-memory staging or ldmatrix is needed.
+constexpr int RM_WARPS = 8;
+
+__device__ __forceinline__ void mma_bf16_16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int MT, int NT>
+__global__ void __launch_bounds__(RM_WARPS * 32)
+k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
+             const float* __restrict__ bias, int64_t N, int d, int E, float* __restrict__ logits) {
+  extern __shared__ float red[];                       // [RM_WARPS][16*MT][NT*8 + 1]
+  constexpr int ROWS = 16 * MT, EP = NT * 8, LD = EP + 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, q = lane & 3;
+  const int64_t t0 = (int64_t)blockIdx.x * ROWS;
+  const int kw = d / RM_WARPS;                         // columns per warp (multiple of 32)
+  const int kbeg = warp * kw;
+
+  float acc[MT][NT][4];
+#pragma unroll
+  for (int i = 0; i < MT; ++i)
+#pragma unroll
+    for (int j = 0; j < NT; ++j)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) acc[i][j][r] = 0.f;
+
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  const uint4* xrow[MT][2];
+#pragma unroll
+  for (int i = 0; i < MT; ++i) {
+    const int64_t ta = t0 + i * 16 + g, tb = ta + 8;
+    xrow[i][0] = ta < N ? reinterpret_cast<const uint4*>(x + ta * d + kbeg) + q : nullptr;
+    xrow[i][1] = tb < N ? reinterpret_cast<const uint4*>(x + tb * d + kbeg) + q : nullptr;
+  }
+  const uint4* wrow[NT];
+#pragma unroll
+  for (int j = 0; j < NT; ++j) {
+    const int e = j * 8 + g;
+    wrow[j] = e < E ? reinterpret_cast<const uint4*>(w + (int64_t)e * d + kbeg) + q : nullptr;
+  }
+
+  const int steps = kw / 32;                           // 32 columns (4 lanes x 8) per step
+#pragma unroll 4
+  for (int s = 0; s < steps; ++s) {
+    uint4 xa[MT], xb[MT];
+#pragma unroll
+    for (int i = 0; i < MT; ++i) {
+      xa[i] = xrow[i][0] ? __ldcs(xrow[i][0] + s * 4) : zero;       // streamed once: evict first
+      xb[i] = xrow[i][1] ? __ldcs(xrow[i][1] + s * 4) : zero;
+    }
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      const uint4 wv = wrow[j] ? __ldg(wrow[j] + s * 4) : zero;
+#pragma unroll
+      for (int i = 0; i < MT; ++i) {
+        mma_bf16_16816(acc[i][j], xa[i].x, xb[i].x, xa[i].y, xb[i].y, wv.x, wv.y);
+        mma_bf16_16816(acc[i][j], xa[i].z, xb[i].z, xa[i].w, xb[i].w, wv.z, wv.w);
+      }
+    }
+  }
+
+  // partial sums of this warp -> shared memory (accumulator layout: rows g, g+8; columns 2q, 2q+1)
+  float* mine = red + (size_t)warp * ROWS * LD;
+#pragma unroll
+  for (int i = 0; i < MT; ++i)
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      const int r0 = i * 16 + g, c0 = j * 8 + 2 * q;
+      mine[r0 * LD + c0] = acc[i][j][0];
+      mine[r0 * LD + c0 + 1] = acc[i][j][1];
+      mine[(r0 + 8) * LD + c0] = acc[i][j][2];
+      mine[(r0 + 8) * LD + c0 + 1] = acc[i][j][3];
+    }
+  __syncthreads();
+  for (int i = threadIdx.x; i < ROWS * E; i += RM_WARPS * 32) {
+    const int r = i / E, e = i - r * E;
+    const int64_t t = t0 + r;
+    if (t >= N) continue;
+    float sum = 0.f;
+#pragma unroll
+    for (int wv = 0; wv < RM_WARPS; ++wv) sum += red[((size_t)wv * ROWS + r) * LD + e];
+    logits[t * E + e] = sum + (bias ? bias[e] : 0.f);
+  }
+}
+
+bool router_mma_ok(int d, int E) { return d % (RM_WARPS * 32) == 0 && E <= 128; }
+
+template <int MT, int NT>
+int launch_router_mma_inst(const __nv_bfloat16* x, const __nv_bfloat16* w, const float* bias, int64_t N, int d,
+                           int E, float* logits, cudaStream_t st) {
+  const size_t smem = (size_t)RM_WARPS * 16 * MT * (NT * 8 + 1) * sizeof(float);
+  if (smem > 48 * 1024) {
+    cudaError_t e_ = cudaFuncSetAttribute(k_router_mma<MT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)smem);
+    if (e_ != cudaSuccess) return note_cuda(e_);
+  }
+  k_router_mma<MT, NT><<<(unsigned)ceil_div(N, 16 * MT), RM_WARPS * 32, smem, st>>>(x, w, bias, N, d, E, logits);
+  return check_launch();
+}
+
+int launch_router_mma(const __nv_bfloat16* x, const __nv_bfloat16* w, const float* bias, int64_t N, int d, int E,
+                      float* logits, cudaStream_t st) {
+  const int nt = (E + 7) / 8;
+  if (nt <= 1) return launch_router_mma_inst<1, 1>(x, w, bias, N, d, E, logits, st);
+  if (nt <= 2) return launch_router_mma_inst<1, 2>(x, w, bias, N, d, E, logits, st);
+  if (nt <= 4) return launch_router_mma_inst<2, 4>(x, w, bias, N, d, E, logits, st);
+  if (nt <= 8) return launch_router_mma_inst<2, 8>(x, w, bias, N, d, E, logits, st);
+  return launch_router_mma_inst<1, 16>(x, w, bias, N, d, E, logits, st);
+}
+
 }  // namespace
 }  // namespace capmoe
 
@@ -174,10 +297,14 @@ extern "C" int capmoe_route(const void* x, const void* w_router, const float* bi
   if (N == 0) return CAPMOE_OK;
   const float* lg = logits_in;
   if (!logits_in) {
-    int rc = dtype == CAPMOE_F32
-                 ? launch_gemm<float>((const float*)x, (const float*)w_router, bias, N, d, E, logits, st)
-                 : launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias,
-                                              N, d, E, logits, st);
+    int rc;
+    if (dtype == CAPMOE_F32)
+      rc = launch_gemm<float>((const float*)x, (const float*)w_router, bias, N, d, E, logits, st);
+    else if (router_mma_ok(d, E) && aligned16(x) && aligned16(w_router))
+      rc = launch_router_mma((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, N, d, E, logits, st);
+    else
+      rc = launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, N, d, E,
+                                      logits, st);
     if (rc != CAPMOE_OK) return rc;
     lg = logits;
   } else if (logits && logits != logits_in) {

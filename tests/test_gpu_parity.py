@@ -23,6 +23,17 @@ def cm():
     return capmoe
 
 
+_INPUT_CACHE = {}
+
+
+def cached_inputs(cfg):
+    """One set of inputs at a time (the Mixtral-shape weights are 2.8 GB on the host)."""
+    if cfg not in _INPUT_CACHE:
+        _INPUT_CACHE.clear()
+        _INPUT_CACHE[cfg] = synth.make_layer_inputs(cfg)
+    return _INPUT_CACHE[cfg]
+
+
 def dev(a):
     if isinstance(a, np.ndarray):
         a = torch.from_numpy(a)
@@ -208,7 +219,7 @@ def test_permute_and_combine(cm, dtype, d, mode):
 # ----------------------------------------------------------------------------- stage 5 and the layer
 def _layer_case(cm, cfg, mode, gamma, straggler=False, sample=None, std=0.02):
     """Run the CUDA layer, then the checker from the GPU's own fp32 logits; compare."""
-    inp = synth.make_layer_inputs(cfg)
+    inp = cached_inputs(cfg)
     wg, wu, wd = inp.w_gate, inp.w_up, inp.w_down
     shared = inp.shared
     layer = cm.MoELayer(dev(inp.x), dev(inp.w_router), dev(inp.bias), dev(wg), dev(wu), dev(wd), cfg.k, cfg.D,
