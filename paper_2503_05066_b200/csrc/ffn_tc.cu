@@ -30,14 +30,15 @@ constexpr int BM = 128;              // rows per tile (TMEM lanes)
 constexpr int BK = 64;               // K elements per stage: 128 bytes of bf16 = one swizzle row
 constexpr int BNB = 256;             // B rows per stage = MMA N
 constexpr int UMMA_K = 16;
-constexpr int STAGES = 4;
+constexpr int STAGES = 4;              // FFN ring depth (48 KB stages)
+constexpr int MAX_STAGES = 16;         // router ring depth limit (smaller stages, deeper ring)
 constexpr int A_BYTES = BM * BK * 2;         // 16 KB
 constexpr int B_BYTES = BNB * BK * 2;        // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TC_THREADS = 192;
 constexpr int MAX_E = 256;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
-                           2 * (MAX_E + 1) * 4;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/ +
+                           2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -106,16 +107,19 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor, kind::f16: D = fp32, A = B = bf16, both K-major, M = 128, N = 256.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BNB >> 3) << 17) |
-                           ((uint32_t)(BM >> 4) << 24);
+// Instruction descriptor, kind::f16: D = fp32, A = B = bf16, both K-major, M = 128, N = n_mma
+// (a multiple of 16 up to 256).
+__host__ __device__ constexpr uint32_t make_idesc(int n_mma) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
 
-__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                     uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -147,62 +151,81 @@ struct Tile { int e, row0, rows, n0; };
 
 // tile_start[e] = first tile of expert e; tiles of an expert: row block fastest, then column block.
 __device__ __forceinline__ bool locate_tile(int tile, int& cursor, const int* tile_start, const int* offs, int E,
-                                            int n_tile, Tile& t) {
+                                            int n_tile, int bm, Tile& t) {
   while (cursor < E && tile >= tile_start[cursor + 1]) ++cursor;
   if (cursor >= E) return false;
   const int local = tile - tile_start[cursor];
   const int cnt = offs[cursor + 1] - offs[cursor];
-  const int nmb = (cnt + BM - 1) / BM;
+  const int nmb = (cnt + bm - 1) / bm;
   const int nb = local / nmb, mb = local - nb * nmb;
   t.e = cursor;
-  t.row0 = offs[cursor] + mb * BM;
-  t.rows = min(BM, cnt - mb * BM);
+  t.row0 = offs[cursor] + mb * bm;
+  t.rows = min(bm, cnt - mb * bm);
   t.n0 = nb * n_tile;
   return true;
 }
 
-// SWIGLU = true : B tile = 128 rows of W_g + 128 rows of W_u, output columns n0..n0+127 of H
-// SWIGLU = false: B tile = 256 rows of W_d, output columns n0..n0+255 of y_perm
-template <bool SWIGLU>
+// MODE_GATE_UP: B tile = 128 rows of W_g + 128 rows of W_u, output columns n0..n0+127 of H (bf16)
+// MODE_DOWN   : B tile = 256 rows of W_d, output columns n0..n0+255 of y_perm (bf16)
+// MODE_ROUTER : one row segment [0, single_rows), B tile = all n_mma (>= Nout) rows of W_r,
+//               output = fp32 logits [rows, Nout] + bias  (Eq. 1's gate)
+enum { MODE_GATE_UP = 0, MODE_DOWN = 1, MODE_ROUTER = 2 };
+
+template <int MODE>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
          const __grid_constant__ CUtensorMap map_b1, const int32_t* __restrict__ expert_offsets, int E,
-         int K /* reduction length */, int Nout /* output columns */, __nv_bfloat16* __restrict__ out,
-         int D_straggler, int32_t* __restrict__ dev_status) {
+         int K /* reduction length */, int Nout /* output columns */, void* __restrict__ out_ptr,
+         int D_straggler, int32_t* __restrict__ dev_status, int n_mma, int single_rows,
+         const float* __restrict__ bias, int tile_rows /* rows per tile actually loaded (<= 128) */,
+         int n_stages, int stage_stride) {
+  constexpr bool SWIGLU = MODE == MODE_GATE_UP;
   constexpr int N_TILE = SWIGLU ? 128 : 256;
+  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(out_ptr);
+  const uint32_t idesc = make_idesc(n_mma);
+  // The MMA always spans 128 rows; with tile_rows < 128 (router, few tokens) only the first
+  // tile_rows rows of the A tile are loaded and stored, the rest of the accumulator is ignored.
+  const uint32_t a_bytes = (uint32_t)(tile_rows * BK * 2);
+  const uint32_t stage_tx = a_bytes + (uint32_t)(n_mma * BK * 2);
   extern __shared__ uint8_t smem_raw[];
   // carve: tiles (1024-byte aligned), barriers, expert tables
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (tiles - raw);
   uint64_t* bars = reinterpret_cast<uint64_t*>(gen + STAGES * STAGE_BYTES);
-  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  // bars[0..16) full, [16..32) empty, [32..34) tmem_full, [34..36) tmem_empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* offs = reinterpret_cast<int*>(gen + STAGES * STAGE_BYTES + 256);
+  int* offs = reinterpret_cast<int*>(gen + STAGES * STAGE_BYTES + 512);
   int* tile_start = offs + (MAX_E + 1);
+  float* bias_s = reinterpret_cast<float*>(tile_start + (MAX_E + 1) + 2);   // [256], router mode only
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * (uint32_t)s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(STAGES + s); };
-  auto tfull_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * STAGES + b); };
-  auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * STAGES + 2 + b); };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(MAX_STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 + b); };
 
   if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 128); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = tid; i <= E; i += TC_THREADS) offs[i] = expert_offsets[i];
+  if (MODE == MODE_ROUTER) {
+    if (tid == 0) { offs[0] = 0; offs[1] = single_rows; }
+    for (int i = tid; i < 256; i += TC_THREADS) bias_s[i] = (bias && i < Nout) ? bias[i] : 0.f;
+  } else {
+    for (int i = tid; i <= E; i += TC_THREADS) offs[i] = expert_offsets[i];
+  }
   __syncthreads();
   if (tid == 0) {
     const int n_blocks = (Nout + N_TILE - 1) / N_TILE;
     int acc = 0;
     for (int e = 0; e < E; ++e) {
       tile_start[e] = acc;
-      acc += ((offs[e + 1] - offs[e] + BM - 1) / BM) * n_blocks;
+      acc += ((offs[e + 1] - offs[e] + tile_rows - 1) / tile_rows) * n_blocks;
     }
     tile_start[E] = acc;
   }
@@ -241,20 +264,20 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       Tile t;
       bool ok = true;
       for (int tile = first; ok && tile < tile_hi; tile += stride) {
-        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, t)) break;
+        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
         for (int kb = 0; kb < num_kb; ++kb, ++kc) {
-          const int s = kc % STAGES;
-          const uint32_t ph = (kc / STAGES) & 1u;
+          const int s = (int)(kc % (uint32_t)n_stages);
+          const uint32_t ph = (kc / (uint32_t)n_stages) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(full_bar(s), STAGE_BYTES);
-          const uint32_t a_dst = tiles + (uint32_t)s * STAGE_BYTES;
-          const uint32_t b_dst = a_dst + A_BYTES;
+          mbar_expect_tx(full_bar(s), stage_tx);
+          const uint32_t a_dst = tiles + (uint32_t)s * (uint32_t)stage_stride;
+          const uint32_t b_dst = a_dst + a_bytes;
           tma_load_2d(a_dst, &map_a, kb * BK, t.row0, full_bar(s));
           if (SWIGLU) {
             tma_load_3d(b_dst, &map_b0, kb * BK, t.n0, t.e, full_bar(s));
             tma_load_3d(b_dst + B_BYTES / 2, &map_b1, kb * BK, t.n0, t.e, full_bar(s));
           } else {
-            tma_load_3d(b_dst, &map_b0, kb * BK, t.n0, t.e, full_bar(s));
+            tma_load_3d(b_dst, &map_b0, kb * BK, MODE == MODE_ROUTER ? 0 : t.n0, t.e, full_bar(s));
           }
         }
       }
@@ -267,23 +290,23 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       Tile t;
       bool ok = true;
       for (int tile = first; ok && tile < tile_hi; tile += stride, ++it) {
-        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, t)) break;
+        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
         const uint32_t b = it & 1u, use = it >> 1;
         if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + b * (uint32_t)BNB;
         for (int kb = 0; kb < num_kb; ++kb, ++kc) {
-          const int s = kc % STAGES;
-          const uint32_t ph = (kc / STAGES) & 1u;
+          const int s = (int)(kc % (uint32_t)n_stages);
+          const uint32_t ph = (kc / (uint32_t)n_stages) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_src = tiles + (uint32_t)s * STAGE_BYTES;
+          const uint32_t a_src = tiles + (uint32_t)s * (uint32_t)stage_stride;
           const uint64_t adesc = umma_desc(a_src);
-          const uint64_t bdesc = umma_desc(a_src + A_BYTES);
+          const uint64_t bdesc = umma_desc(a_src + a_bytes);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advance 32 bytes (16 bf16) inside the swizzled 128-byte row: +2 in 16-byte units
-            umma(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), (kb | k) != 0 ? 1u : 0u);
+            umma(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
           }
           umma_commit(empty_bar(s));                    // frees the stage when these MMAs have read it
         }
@@ -298,7 +321,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     uint32_t it = 0;
     Tile t;
     for (int tile = first; tile < tile_hi; tile += stride, ++it) {
-      if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, t)) break;
+      if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
       const uint32_t b = it & 1u, use = it >> 1;
       bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
       ready = __all_sync(0xffffffffu, ready);            // warp-uniform: tcgen05.ld below is .sync.aligned
@@ -306,6 +329,32 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)BNB;
       const bool row_ok = row_in_tile < t.rows;
+      if (MODE == MODE_ROUTER) {
+        float* lrow = reinterpret_cast<float*>(out_ptr) + (int64_t)(t.row0 + row_in_tile) * Nout;
+#pragma unroll 1
+        for (int c = 0; c < n_mma; c += 32) {
+          uint32_t g[32];
+          tmem_ld32(taddr + (uint32_t)c, g);
+          tmem_ld_wait();
+          float v[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(g[j]) + bias_s[c + j];
+          if (row_ok) {
+            if ((Nout & 3) == 0) {                       // rows are 16-byte aligned: vector stores
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                if (c + j < Nout) *reinterpret_cast<float4*>(lrow + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c + j < Nout) lrow[c + j] = v[j];
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(tempty_bar(b));
+        continue;
+      }
       __nv_bfloat16* orow = out + (int64_t)(t.row0 + row_in_tile) * Nout + t.n0;
 #pragma unroll 1
       for (int c = 0; c < N_TILE; c += 32) {
@@ -404,22 +453,55 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
       !make_map(&a2, h_ws, (uint64_t)F, (uint64_t)A_max, 0, BM) ||
       !make_map(&bd, w_down, (uint64_t)F, (uint64_t)d, (uint64_t)E, 256))
     return note_cuda(cudaErrorInvalidValue);
-  cudaError_t err = cudaFuncSetAttribute(k_ffn_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaError_t err = cudaFuncSetAttribute(k_ffn_tc<MODE_GATE_UP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         SMEM_BYTES);
   if (err != cudaSuccess) return note_cuda(err);
-  err = cudaFuncSetAttribute(k_ffn_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  err = cudaFuncSetAttribute(k_ffn_tc<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (err != cudaSuccess) return note_cuda(err);
   int grid = sm_count();
   if (D_straggler > 0) {
     if (grid < D_straggler) return CAPMOE_EUNSUPPORTED;
     grid = (grid / D_straggler) * D_straggler;          // equal share of SMs per virtual device
   }
-  k_ffn_tc<true><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a1, bg, bu, expert_offsets, E, d, F,
-                                                      (__nv_bfloat16*)h_ws, D_straggler, dev_status);
+  k_ffn_tc<MODE_GATE_UP><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a1, bg, bu, expert_offsets, E, d, F, h_ws,
+                                                              D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES);
   int rc = check_launch();
   if (rc != CAPMOE_OK) return rc;
   if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
-  k_ffn_tc<false><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a2, bd, bd, expert_offsets, E, F, d,
-                                                       (__nv_bfloat16*)y_perm, D_straggler, dev_status);
+  k_ffn_tc<MODE_DOWN><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a2, bd, bd, expert_offsets, E, F, d, y_perm,
+                                                           D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES);
+  return check_launch();
+}
+
+// Router logits on the same pipeline: logits[N,E] = x[N,d] . w_router[E,d]^T + bias, fp32 out.
+bool router_tc_supported(int64_t N, int d, int E) { return d % 64 == 0 && d >= 64 && E <= 256 && N < (1ll << 31); }
+
+int router_tc(const void* x, const void* w_router, const float* bias, int64_t N, int d, int E, float* logits,
+              cudaStream_t st) {
+  const int n_mma = (E + 15) / 16 * 16;
+  // The stage reads X once and is bound by HBM, so what matters is bytes in flight: use row tiles
+  // small enough that every SM gets one (the MMA still spans 128 rows; the unused rows cost
+  // nothing that is on the critical path) and as deep a ring as shared memory allows.
+  const int sms = sm_count();
+  const int tile_rows = N >= (int64_t)128 * sms ? 128 : (N >= (int64_t)64 * sms ? 64 : 32);
+  // A stage holds tile_rows rows of A followed by n_mma rows of B (both multiples of 1 KB).  The
+  // MMA reads 128 A rows whatever tile_rows is, so the last stage must leave room for that.
+  const int b_bytes = n_mma * BK * 2;
+  const int stage_stride = tile_rows * BK * 2 + b_bytes;
+  int n_stages = (STAGES * STAGE_BYTES - A_BYTES - b_bytes) / stage_stride + 1;
+  if (n_stages > MAX_STAGES) n_stages = MAX_STAGES;
+  if (n_stages > (STAGES * STAGE_BYTES) / stage_stride) n_stages = (STAGES * STAGE_BYTES) / stage_stride;
+  alignas(64) CUtensorMap ax, bw;
+  if (!make_map(&ax, x, (uint64_t)d, (uint64_t)N, 0, (uint32_t)tile_rows) ||
+      !make_map(&bw, w_router, (uint64_t)d, (uint64_t)E, 1, (uint32_t)n_mma))
+    return note_cuda(cudaErrorInvalidValue);
+  cudaError_t err = cudaFuncSetAttribute(k_ffn_tc<MODE_ROUTER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         SMEM_BYTES);
+  if (err != cudaSuccess) return note_cuda(err);
+  int grid = (int)ceil_div(N, tile_rows);
+  if (grid > sm_count()) grid = sm_count();
+  k_ffn_tc<MODE_ROUTER><<<grid, TC_THREADS, SMEM_BYTES, st>>>(ax, bw, bw, nullptr, 1, d, E, logits, 0, nullptr,
+                                                             n_mma, (int)N, bias, tile_rows, n_stages, stage_stride);
   return check_launch();
 }
 

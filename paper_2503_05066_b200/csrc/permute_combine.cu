@@ -1,48 +1,63 @@
 // Stage 4 (permute: gather kept tokens into expert-major rows) and stage 6 (combine: the
-// gate-weighted sum of Eq. 2 back in token order).  Pure data movement: one warp per token,
-// 16-byte accesses, each x row read once and written to every row that keeps it.
+// gate-weighted sum of Eq. 2 back in token order).  Pure data movement, bound by HBM.
+// Work unit = (token, 2 KB chunk of its row): one warp per unit, four 16-byte vectors per lane,
+// so that the number of units (N * row bytes / 2 KB) is many times the number of resident warps
+// and the last wave stays full.  Each x row is read once and written to every row that keeps it.
 #include "common.cuh"
 
 namespace capmoe {
 namespace {
 
-constexpr int PC_WARPS = 8;          // warps (tokens) per CTA
+constexpr int PC_WARPS = 8;          // warps (work units) per CTA
+constexpr int VPL = 4;               // 16-byte vectors per lane per unit
+constexpr int CHUNK_VECS = 32 * VPL; // vectors per unit (2 KB)
 constexpr int MAX_SLOTS = 288;       // k + m <= 32 + 256
 
 __global__ void __launch_bounds__(PC_WARPS * 32)
-k_permute(const uint4* __restrict__ x, int64_t N, int row_vecs /* 16-byte vectors per row */, int E, int k,
-          int slots, int D, const float* __restrict__ scores, const int32_t* __restrict__ topk_idx,
+k_permute(const uint4* __restrict__ x, int64_t N, int row_vecs /* 16-byte vectors per row */, int chunks, int E,
+          int k, int slots, int D, const float* __restrict__ scores, const int32_t* __restrict__ topk_idx,
           const int32_t* __restrict__ token_group, const int32_t* __restrict__ slot_row,
           uint4* __restrict__ x_perm, int32_t* __restrict__ perm_token, float* __restrict__ perm_weight) {
   const int lane = threadIdx.x & 31;
-  const int64_t t = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
+  const int64_t unit = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
+  const int64_t t = unit / chunks;
+  const int chunk = (int)(unit - t * chunks);
   if (t >= N) return;
-  const int m = D > 0 ? E / D : 0;
-  const int g = D > 0 ? home_group(t, N, D, token_group) : 0;
   const int32_t* sr = slot_row + t * slots;
-  // bookkeeping: lane s handles slot s (+32, +64, ...)
-  for (int s = lane; s < slots; s += 32) {
-    const int32_t r = sr[s];
-    if (r >= 0) {
-      const int e = s < k ? topk_idx[t * k + s] : g * m + (s - k);
-      perm_token[r] = (int32_t)t;
-      perm_weight[r] = scores[t * E + e];
+  if (chunk == 0) {                                    // bookkeeping once per token: lane s handles slot s, s+32, ...
+    const int m = D > 0 ? E / D : 0;
+    const int g = D > 0 ? home_group(t, N, D, token_group) : 0;
+    for (int s = lane; s < slots; s += 32) {
+      const int32_t r = sr[s];
+      if (r >= 0) {
+        const int e = s < k ? topk_idx[t * k + s] : g * m + (s - k);
+        perm_token[r] = (int32_t)t;
+        perm_weight[r] = scores[t * E + e];
+      }
     }
   }
-  const uint4* src = x + t * row_vecs;
+  const int v0 = chunk * CHUNK_VECS + lane;
+  const uint4* src = x + t * row_vecs + v0;
+  uint4 val[VPL];
+  bool loaded = false;
   for (int s0 = 0; s0 < slots; s0 += 32) {
     const int32_t mine = (s0 + lane < slots) ? sr[s0 + lane] : -1;
-    unsigned live = __ballot_sync(0xffffffffu, mine >= 0);
-    if (!live) continue;
-    for (int v = lane; v < row_vecs; v += 32) {
-      const uint4 val = src[v];
-      unsigned rem = live;
-      while (rem) {
-        const int b = __ffs(rem) - 1;
-        rem &= rem - 1;
-        const int32_t r = __shfl_sync(0xffffffffu, mine, b);
-        x_perm[(int64_t)r * row_vecs + v] = val;
-      }
+    unsigned rem = __ballot_sync(0xffffffffu, mine >= 0);
+    if (!rem) continue;
+    if (!loaded) {                                     // a token nobody keeps is never read
+#pragma unroll
+      for (int u = 0; u < VPL; ++u)
+        val[u] = (v0 + u * 32 < row_vecs) ? __ldcs(src + u * 32) : make_uint4(0u, 0u, 0u, 0u);
+      loaded = true;
+    }
+    while (rem) {
+      const int b = __ffs(rem) - 1;
+      rem &= rem - 1;
+      const int32_t r = __shfl_sync(0xffffffffu, mine, b);
+      uint4* dst = x_perm + (int64_t)r * row_vecs + v0;
+#pragma unroll
+      for (int u = 0; u < VPL; ++u)
+        if (v0 + u * 32 < row_vecs) dst[u * 32] = val[u];
     }
   }
 }
@@ -78,55 +93,67 @@ template <> struct Vec16<__nv_bfloat16> {
   }
 };
 
+// acc[u] += wgt * row[u] for the VPL vectors of one kept row
+template <typename T>
+__device__ __forceinline__ void axpy_row(float (*acc)[Vec16<T>::n], const uint4* raw, float wgt) {
+#pragma unroll
+  for (int u = 0; u < VPL; ++u) {
+    float f[Vec16<T>::n];
+    Vec16<T>::load(raw[u], f);
+#pragma unroll
+    for (int i = 0; i < Vec16<T>::n; ++i) acc[u][i] = fmaf(wgt, f[i], acc[u][i]);
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(PC_WARPS * 32)
 k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row,
-          const float* __restrict__ perm_weight, int64_t N, int row_vecs, int slots,
+          const float* __restrict__ perm_weight, int64_t N, int row_vecs, int chunks, int slots,
           const uint4* __restrict__ y_shared, uint4* __restrict__ y) {
   constexpr int NV = Vec16<T>::n;
   const int lane = threadIdx.x & 31;
-  const int64_t t = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
+  const int64_t unit = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
+  const int64_t t = unit / chunks;
+  const int chunk = (int)(unit - t * chunks);
   if (t >= N) return;
   const int32_t* sr = slot_row + t * slots;
-  constexpr int VPL = 4;                               // 16-byte vectors per lane in flight per row
-  for (int v0 = 0; v0 < row_vecs; v0 += 32 * VPL) {
-    float acc[VPL][NV];
+  const int v0 = chunk * CHUNK_VECS + lane;
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  float acc[VPL][NV];
 #pragma unroll
-    for (int u = 0; u < VPL; ++u) {
-      const int v = v0 + u * 32 + lane;
+  for (int u = 0; u < VPL; ++u) {
 #pragma unroll
-      for (int i = 0; i < NV; ++i) acc[u][i] = 0.f;
-      if (y_shared && v < row_vecs) Vec16<T>::load(y_shared[t * row_vecs + v], acc[u]);
-    }
-    for (int s0 = 0; s0 < slots; s0 += 32) {
-      const int32_t mine = (s0 + lane < slots) ? sr[s0 + lane] : -1;
-      const float wmine = mine >= 0 ? perm_weight[mine] : 0.f;
-      unsigned rem = __ballot_sync(0xffffffffu, mine >= 0);
-      while (rem) {                                    // ascending slot order
-        const int b = __ffs(rem) - 1;
-        rem &= rem - 1;
-        const int32_t r = __shfl_sync(0xffffffffu, mine, b);
-        const float wgt = __shfl_sync(0xffffffffu, wmine, b);
-        const uint4* src = y_perm + (int64_t)r * row_vecs + v0 + lane;
-        uint4 raw[VPL];
+    for (int i = 0; i < NV; ++i) acc[u][i] = 0.f;
+    if (y_shared && v0 + u * 32 < row_vecs) Vec16<T>::load(__ldcs(y_shared + t * row_vecs + v0 + u * 32), acc[u]);
+  }
+  for (int s0 = 0; s0 < slots; s0 += 32) {
+    const int32_t mine = (s0 + lane < slots) ? sr[s0 + lane] : -1;
+    const float wmine = mine >= 0 ? perm_weight[mine] : 0.f;
+    unsigned rem = __ballot_sync(0xffffffffu, mine >= 0);
+    while (rem) {                                      // ascending slot order, two kept rows per round
+      const int b0 = __ffs(rem) - 1;
+      rem &= rem - 1;
+      const bool two = rem != 0;
+      const int b1 = two ? __ffs(rem) - 1 : b0;
+      rem &= rem - 1;                                  // no-op when rem is already 0
+      const int32_t r0 = __shfl_sync(0xffffffffu, mine, b0), r1 = __shfl_sync(0xffffffffu, mine, b1);
+      const float w0 = __shfl_sync(0xffffffffu, wmine, b0), w1 = __shfl_sync(0xffffffffu, wmine, b1);
+      const uint4* p0 = y_perm + (int64_t)r0 * row_vecs + v0;
+      const uint4* p1 = y_perm + (int64_t)r1 * row_vecs + v0;
+      uint4 raw0[VPL], raw1[VPL];
 #pragma unroll
-        for (int u = 0; u < VPL; ++u)                  // independent loads first, arithmetic after
-          raw[u] = (v0 + u * 32 + lane < row_vecs) ? __ldcs(src + u * 32) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < VPL; ++u) {
-          float f[NV];
-          Vec16<T>::load(raw[u], f);
-#pragma unroll
-          for (int i = 0; i < NV; ++i) acc[u][i] = fmaf(wgt, f[i], acc[u][i]);
-        }
+      for (int u = 0; u < VPL; ++u) {                  // all loads first, arithmetic after
+        const bool in = v0 + u * 32 < row_vecs;
+        raw0[u] = in ? __ldcs(p0 + u * 32) : zero;
+        raw1[u] = (in && two) ? __ldcs(p1 + u * 32) : zero;
       }
-    }
-#pragma unroll
-    for (int u = 0; u < VPL; ++u) {
-      const int v = v0 + u * 32 + lane;
-      if (v < row_vecs) y[t * row_vecs + v] = Vec16<T>::store(acc[u]);
+      axpy_row<T>(acc, raw0, w0);
+      if (two) axpy_row<T>(acc, raw1, w1);
     }
   }
+#pragma unroll
+  for (int u = 0; u < VPL; ++u)
+    if (v0 + u * 32 < row_vecs) y[t * row_vecs + v0 + u * 32] = Vec16<T>::store(acc[u]);
 }
 
 }  // namespace
@@ -148,9 +175,12 @@ extern "C" int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int
   if (!x || !scores || !topk_idx || !slot_row || !x_perm || !perm_token || !perm_weight) return CAPMOE_EINVAL;
   if (!aligned16(x) || !aligned16(x_perm)) return CAPMOE_EINVAL;
   const int row_vecs = (int)((size_t)d * elt_size(dtype) / 16);
-  k_permute<<<(unsigned)ceil_div(N, PC_WARPS), PC_WARPS * 32, 0, as_stream(stream)>>>(
-      (const uint4*)x, N, row_vecs, E, k, slots, D, scores, topk_idx, token_group, slot_row, (uint4*)x_perm,
-      perm_token, perm_weight);
+  const int chunks = (row_vecs + CHUNK_VECS - 1) / CHUNK_VECS;
+  const int64_t blocks = ceil_div(N * chunks, PC_WARPS);
+  if (blocks > 0x7fffffff) return CAPMOE_EUNSUPPORTED;
+  k_permute<<<(unsigned)blocks, PC_WARPS * 32, 0, as_stream(stream)>>>(
+      (const uint4*)x, N, row_vecs, chunks, E, k, slots, D, scores, topk_idx, token_group, slot_row,
+      (uint4*)x_perm, perm_token, perm_weight);
   return check_launch();
 }
 
@@ -164,13 +194,16 @@ extern "C" int capmoe_combine(const void* y_perm, const int32_t* slot_row, const
   if (!slot_row || !y) return CAPMOE_EINVAL;       // y_perm / perm_weight may be NULL only if A == 0
   if (!aligned16(y_perm) || !aligned16(y) || !aligned16(y_shared)) return CAPMOE_EINVAL;
   const int row_vecs = (int)((size_t)d * elt_size(dtype) / 16);
-  const unsigned grid = (unsigned)ceil_div(N, PC_WARPS);
+  const int chunks = (row_vecs + CHUNK_VECS - 1) / CHUNK_VECS;
+  const int64_t blocks = ceil_div(N * chunks, PC_WARPS);
+  if (blocks > 0x7fffffff) return CAPMOE_EUNSUPPORTED;
   cudaStream_t st = as_stream(stream);
   if (dtype == CAPMOE_F32)
-    k_combine<float><<<grid, PC_WARPS * 32, 0, st>>>((const uint4*)y_perm, slot_row, perm_weight, N, row_vecs,
-                                                      slots, (const uint4*)y_shared, (uint4*)y);
+    k_combine<float><<<(unsigned)blocks, PC_WARPS * 32, 0, st>>>((const uint4*)y_perm, slot_row, perm_weight, N,
+                                                                row_vecs, chunks, slots, (const uint4*)y_shared,
+                                                                (uint4*)y);
   else
-    k_combine<__nv_bfloat16><<<grid, PC_WARPS * 32, 0, st>>>((const uint4*)y_perm, slot_row, perm_weight, N,
-                                                              row_vecs, slots, (const uint4*)y_shared, (uint4*)y);
+    k_combine<__nv_bfloat16><<<(unsigned)blocks, PC_WARPS * 32, 0, st>>>(
+        (const uint4*)y_perm, slot_row, perm_weight, N, row_vecs, chunks, slots, (const uint4*)y_shared, (uint4*)y);
   return check_launch();
 }

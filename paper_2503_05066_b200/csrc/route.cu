@@ -7,7 +7,6 @@ namespace {
 constexpr int RT_TOK = 32;     // tokens per CTA in the GEMM
 constexpr int RT_EG = 8;       // expert groups per CTA (threads = RT_TOK * RT_EG)
 constexpr int RT_BK = 64;      // K chunk
-constexpr int SM_TOK = 64;     // tokens per CTA in the softmax/top-k kernel
 
 // logits[t,e] = sum_j x[t,j] w[e,j] + bias[e], fp32 accumulate.  One CTA: RT_TOK tokens x all E
 // experts; thread (lane = token, group = tid/32) owns EPT experts of one token.
@@ -79,54 +78,94 @@ __device__ __forceinline__ float exp_fixed(float x) {
   return __uint_as_float(__float_as_uint(q) + ((unsigned)ni << 23));
 }
 
-// One thread per token: softmax over the E logits (left-to-right sum), top-k by repeated
-// arg-max (strict '>' keeps the lower expert id on equal scores), load histogram.
-__global__ void __launch_bounds__(SM_TOK)
-k_softmax_topk(const float* __restrict__ logits, int64_t N, int E, int k, float* __restrict__ scores,
-               int32_t* __restrict__ topk_idx, float* __restrict__ topk_score, int32_t* __restrict__ load) {
+// Softmax, top-k and load histogram.  One warp per token, EPL = ceil(E/32) experts per lane: the max is a shuffle reduction (exact), every lane evaluates exp for its
+// experts, ONE lane adds the E terms left to right (the order the scores are defined with),
+// every lane divides; top-k is k rounds of a warp arg-max on (score, lower expert id wins).
+constexpr int SW_WARPS = 8;
+
+template <int EPL>
+__global__ void __launch_bounds__(SW_WARPS * 32)
+k_softmax_topk_warp(const float* __restrict__ logits, int64_t N, int E, int k, float* __restrict__ scores,
+                    int32_t* __restrict__ topk_idx, float* __restrict__ topk_score, int32_t* __restrict__ load) {
   extern __shared__ float smem[];
-  const int ld = E + 1;
-  float* rows = smem;                                     // [SM_TOK][E+1]
-  int* hist = reinterpret_cast<int*>(smem + SM_TOK * ld); // [E]
-  const int tid = threadIdx.x;
-  const int64_t t0 = (int64_t)blockIdx.x * SM_TOK;
-  const int64_t nrow = min((int64_t)SM_TOK, N - t0);
-  for (int i = tid; i < E; i += SM_TOK) hist[i] = 0;
-  for (int64_t i = tid; i < nrow * E; i += SM_TOK) rows[(i / E) * ld + (i % E)] = logits[t0 * E + i];
+  float* prow = smem + (threadIdx.x >> 5) * (EPL * 32);       // this warp's E exponentials
+  int* hist = reinterpret_cast<int*>(smem + SW_WARPS * EPL * 32);
+  const int lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < E; i += SW_WARPS * 32) hist[i] = 0;
   __syncthreads();
-  float* row = rows + tid * ld;
-  if (tid < nrow) {
-    float mx = row[0];
-    for (int e = 1; e < E; ++e) mx = row[e] > mx ? row[e] : mx;
-    float sum = 0.f;
-    for (int e = 0; e < E; ++e) {
-      float p = exp_fixed(__fsub_rn(row[e], mx));
-      row[e] = p;
-      sum = __fadd_rn(sum, p);
+  const int64_t warps_total = (int64_t)gridDim.x * SW_WARPS;
+  for (int64_t t = (int64_t)blockIdx.x * SW_WARPS + (threadIdx.x >> 5); t < N; t += warps_total) {
+    const float* lrow = logits + t * E;
+    float v[EPL];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) {
+      const int e = lane + 32 * i;
+      v[i] = e < E ? lrow[e] : -INFINITY;
+      mx = v[i] > mx ? v[i] : mx;
     }
-    for (int e = 0; e < E; ++e) row[e] = __fdiv_rn(row[e], sum);
-  }
-  __syncthreads();
-  for (int64_t i = tid; i < nrow * E; i += SM_TOK) scores[t0 * E + i] = rows[(i / E) * ld + (i % E)];
-  __syncthreads();
-  if (tid < nrow) {
-    const int64_t t = t0 + tid;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float other = __shfl_xor_sync(0xffffffffu, mx, o);
+      mx = other > mx ? other : mx;
+    }
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) {
+      const int e = lane + 32 * i;
+      if (e < E) { v[i] = exp_fixed(__fsub_rn(v[i], mx)); prow[e] = v[i]; }
+    }
+    __syncwarp();
+    float sum = 0.f;
+    if (lane == 0)
+      for (int e = 0; e < E; ++e) sum = __fadd_rn(sum, prow[e]);
+    sum = __shfl_sync(0xffffffffu, sum, 0);
+    __syncwarp();                                              // prow is rewritten by the next token
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) {
+      const int e = lane + 32 * i;
+      if (e < E) { v[i] = __fdiv_rn(v[i], sum); scores[t * E + e] = v[i]; }
+      else v[i] = -1.f;                                        // never selected (scores are >= 0)
+    }
+    float my_score = 0.f;
+    int my_idx = 0;
     for (int j = 0; j < k; ++j) {
       float best = -1.f;
-      int be = 0;
-      for (int e = 0; e < E; ++e) {
-        float v = row[e];
-        if (v > best) { best = v; be = e; }
+      int be = 0x7fffffff;
+#pragma unroll
+      for (int i = 0; i < EPL; ++i)                            // ascending expert id inside the lane
+        if (v[i] > best) { best = v[i]; be = lane + 32 * i; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+        if (ob > best || (ob == best && oe < be)) { best = ob; be = oe; }
       }
-      row[be] = -2.f;                                     // taken (scores are >= 0)
-      topk_idx[t * k + j] = be;
-      topk_score[t * k + j] = best;
-      atomicAdd(&hist[be], 1);
+#pragma unroll
+      for (int i = 0; i < EPL; ++i)
+        if (be == lane + 32 * i) v[i] = -2.f;                  // taken
+      if (lane == j) { my_score = best; my_idx = be; }
+    }
+    if (lane < k) {
+      topk_idx[t * k + lane] = my_idx;
+      topk_score[t * k + lane] = my_score;
+      atomicAdd(&hist[my_idx], 1);
     }
   }
   __syncthreads();
-  for (int i = tid; i < E; i += SM_TOK)
+  for (int i = threadIdx.x; i < E; i += SW_WARPS * 32)
     if (hist[i]) atomicAdd(&load[i], hist[i]);
+}
+
+template <int EPL>
+int launch_softmax_warp(const float* lg, int64_t N, int E, int k, float* scores, int32_t* topk_idx,
+                        float* topk_score, int32_t* load, cudaStream_t st) {
+  const size_t smem = (size_t)SW_WARPS * EPL * 32 * sizeof(float) + (size_t)E * sizeof(int);
+  int64_t blocks = ceil_div(N, SW_WARPS);
+  const int64_t cap = (int64_t)sm_count() * 8;                 // resident CTAs; more tokens loop inside
+  if (blocks > cap) blocks = cap;
+  k_softmax_topk_warp<EPL><<<(unsigned)blocks, SW_WARPS * 32, smem, st>>>(lg, N, E, k, scores, topk_idx,
+                                                                          topk_score, load);
+  return check_launch();
 }
 
 template <typename T>
@@ -164,6 +203,12 @@ int launch_gemm(const T* x, const T* w, const float* bias, int64_t N, int d, int
 // columns of X (one 16-byte load) as the k slots it owns in two MMAs, and loads the same 8
 // columns of W_r for its B fragment; no shared-memory staging or ldmatrix is needed.
 constexpr int RM_WARPS = 8;
+}  // namespace
+// tcgen05 router GEMM (ffn_tc.cu): used when there are enough experts for the MMA work to matter
+bool router_tc_supported(int64_t N, int d, int E);
+int router_tc(const void* x, const void* w_router, const float* bias, int64_t N, int d, int E, float* logits,
+              cudaStream_t st);
+namespace {
 
 __device__ __forceinline__ void mma_bf16_16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -272,8 +317,11 @@ int launch_router_mma(const __nv_bfloat16* x, const __nv_bfloat16* w, const floa
   const int nt = (E + 7) / 8;
   if (nt <= 1) return launch_router_mma_inst<1, 1>(x, w, bias, N, d, E, logits, st);
   if (nt <= 2) return launch_router_mma_inst<1, 2>(x, w, bias, N, d, E, logits, st);
-  if (nt <= 4) return launch_router_mma_inst<2, 4>(x, w, bias, N, d, E, logits, st);
-  if (nt <= 8) return launch_router_mma_inst<2, 8>(x, w, bias, N, d, E, logits, st);
+  const bool wide = N >= (int64_t)32 * 2 * sm_count();      // enough tokens for 32-token CTAs to fill the GPU
+  if (nt <= 4) return wide ? launch_router_mma_inst<2, 4>(x, w, bias, N, d, E, logits, st)
+                           : launch_router_mma_inst<1, 4>(x, w, bias, N, d, E, logits, st);
+  if (nt <= 8) return wide ? launch_router_mma_inst<2, 8>(x, w, bias, N, d, E, logits, st)
+                           : launch_router_mma_inst<1, 8>(x, w, bias, N, d, E, logits, st);
   return launch_router_mma_inst<1, 16>(x, w, bias, N, d, E, logits, st);
 }
 
@@ -300,6 +348,8 @@ extern "C" int capmoe_route(const void* x, const void* w_router, const float* bi
     int rc;
     if (dtype == CAPMOE_F32)
       rc = launch_gemm<float>((const float*)x, (const float*)w_router, bias, N, d, E, logits, st);
+    else if (E > 16 && router_tc_supported(N, d, E) && aligned16(x) && aligned16(w_router))
+      rc = router_tc(x, w_router, bias, N, d, E, logits, st);
     else if (router_mma_ok(d, E) && aligned16(x) && aligned16(w_router))
       rc = launch_router_mma((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, N, d, E, logits, st);
     else
@@ -311,12 +361,9 @@ extern "C" int capmoe_route(const void* x, const void* w_router, const float* bi
     err = cudaMemcpyAsync(logits, logits_in, sizeof(float) * N * E, cudaMemcpyDeviceToDevice, st);
     if (err != cudaSuccess) return note_cuda(err);
   }
-  const size_t smem = (size_t)SM_TOK * (E + 1) * sizeof(float) + (size_t)E * sizeof(int);
-  if (smem > 48 * 1024) {
-    err = cudaFuncSetAttribute(k_softmax_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (err != cudaSuccess) return note_cuda(err);
-  }
-  k_softmax_topk<<<(unsigned)ceil_div(N, SM_TOK), SM_TOK, smem, st>>>(lg, N, E, k, scores, topk_idx,
-                                                                       topk_score, load);
-  return check_launch();
+  const int epl = (E + 31) / 32;
+  if (epl <= 1) return launch_softmax_warp<1>(lg, N, E, k, scores, topk_idx, topk_score, load, st);
+  if (epl <= 2) return launch_softmax_warp<2>(lg, N, E, k, scores, topk_idx, topk_score, load, st);
+  if (epl <= 4) return launch_softmax_warp<4>(lg, N, E, k, scores, topk_idx, topk_score, load, st);
+  return launch_softmax_warp<8>(lg, N, E, k, scores, topk_idx, topk_score, load, st);
 }
