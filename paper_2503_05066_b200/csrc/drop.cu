@@ -3,6 +3,14 @@
 // the C-th largest score with a shared-memory radix select over the float bit patterns
 // (non-negative floats order like unsigned integers), and keep everything above it plus the
 // first (C - #above) candidates equal to it, in token order.
+//
+// One small memset (the E candidate counters) and two launches:
+//   k_count_candidates  one CTA per 256 tokens: per-expert candidate counts (shared-memory
+//                       histogram, then integer atomics: the totals do not depend on order), and
+//                       the initial state of the outputs that k_select only touches sparsely
+//                       (keep_mask = 0, slot_row = -1 for Expanded Drop).
+//   k_select            one CTA per expert: prefix sums of the counts, ordered compaction,
+//                       radix select, ordered placement.
 #include <mutex>
 
 #include "common.cuh"
@@ -11,12 +19,16 @@ namespace capmoe {
 namespace {
 
 constexpr int CNT_THREADS = 256;
+constexpr int TPT = 4;                               // tokens (candidates) per thread per round in k_select
+constexpr int CNT_TOKENS = CNT_THREADS;              // tokens per counting CTA
 constexpr int SEL_THREADS = 1024;
 constexpr int SEL_WARPS = SEL_THREADS / 32;
-constexpr int RADIX_BINS = 2048;     // 11 + 11 + 10 bits
+constexpr int SEL_TOKENS = SEL_THREADS * TPT;        // tokens per compaction round
+constexpr int RADIX_BINS = 2048;                     // 11 + 11 + 10 bits
+constexpr int E_STRIDE = 256;                        // E <= 256
 
 struct DropWs {
-  int32_t* cand;      // [E]   candidate counts (Token Drop only; Expanded Drop uses the caller's)
+  int32_t* cand;      // [E_STRIDE] candidate counts (when the caller has no array for them)
   uint32_t* key;      // [cap] score bits of each candidate, expert-major, token order inside
   int32_t* tok;       // [cap]
   int32_t* slot;      // [cap]
@@ -25,35 +37,38 @@ struct DropWs {
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 inline size_t ws_bytes_needed(int64_t N, int E, int k, int D, int expanded) {
-  int64_t cap = N * (int64_t)(expanded ? k + E / D : k);
-  return align256(sizeof(int32_t) * 256) + 3 * align256(sizeof(int32_t) * (size_t)cap);
+  const int64_t cap = N * (int64_t)(expanded ? k + E / D : k);
+  return align256(sizeof(int32_t) * E_STRIDE) + 3 * align256(sizeof(int32_t) * (size_t)cap);
 }
 
 inline DropWs carve(void* ws, int64_t N, int E, int k, int D, int expanded) {
-  int64_t cap = N * (int64_t)(expanded ? k + E / D : k);
+  const int64_t cap = N * (int64_t)(expanded ? k + E / D : k);
   char* p = (char*)ws;
   DropWs w;
-  w.cand = (int32_t*)p; p += align256(sizeof(int32_t) * 256);
+  w.cand = (int32_t*)p; p += align256(sizeof(int32_t) * E_STRIDE);
   w.key = (uint32_t*)p; p += align256(sizeof(int32_t) * (size_t)cap);
   w.tok = (int32_t*)p;  p += align256(sizeof(int32_t) * (size_t)cap);
   w.slot = (int32_t*)p;
   return w;
 }
 
-// Candidates per expert: |{t : e in topk(t)}| (+ |{t : h(t) = e/m, e not in topk(t)}| when EXPANDED).
+// Candidates per expert among this CTA's tokens: |{t : e in topk(t)}| (+ |{t : h(t) = e/m, e not
+// in topk(t)}| when EXPANDED); plus the initial state of keep_mask / slot_row for these tokens.
 template <bool EXPANDED>
 __global__ void __launch_bounds__(CNT_THREADS)
 k_count_candidates(const int32_t* __restrict__ topk_idx, int64_t N, int E, int k, int D,
-                   const int32_t* __restrict__ token_group, int32_t* __restrict__ cand) {
+                   const int32_t* __restrict__ token_group, int32_t* __restrict__ cand,
+                   unsigned long long* __restrict__ keep_mask, int32_t* __restrict__ slot_row) {
   extern __shared__ int hist[];
   for (int i = threadIdx.x; i < E; i += CNT_THREADS) hist[i] = 0;
   __syncthreads();
-  const int64_t t = (int64_t)blockIdx.x * CNT_THREADS + threadIdx.x;
-  if (t < N) {
+  const int64_t t0 = (int64_t)blockIdx.x * CNT_TOKENS;
+  const int64_t t1 = min(N, t0 + CNT_TOKENS);
+  const int m = EXPANDED ? E / D : 1;
+  for (int64_t t = t0 + threadIdx.x; t < t1; t += CNT_THREADS) {
     const int32_t* row = topk_idx + t * k;
     for (int j = 0; j < k; ++j) atomicAdd(&hist[row[j]], 1);
     if (EXPANDED) {
-      const int m = E / D;
       const int g = home_group(t, N, D, token_group);
       for (int i = 0; i < m; ++i) {
         const int e = g * m + i;
@@ -62,6 +77,12 @@ k_count_candidates(const int32_t* __restrict__ topk_idx, int64_t N, int E, int k
         if (!in) atomicAdd(&hist[e], 1);
       }
     }
+  }
+  const int W = (E + 63) >> 6;
+  for (int64_t i = t0 * W + threadIdx.x; i < t1 * W; i += CNT_THREADS) keep_mask[i] = 0ull;
+  if (EXPANDED) {       // local-expert slots that are already top-k slots are never written again
+    const int slots = k + m;
+    for (int64_t i = t0 * slots + threadIdx.x; i < t1 * slots; i += CNT_THREADS) slot_row[i] = -1;
   }
   __syncthreads();
   for (int i = threadIdx.x; i < E; i += CNT_THREADS)
@@ -124,26 +145,25 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
          int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
   __shared__ int hist[RADIX_BINS];
   __shared__ uint32_t scan_sh[SEL_WARPS + 1];
-  __shared__ uint32_t found[2];
+  __shared__ uint32_t found[3];
   const int e = blockIdx.x;
   const int tid = threadIdx.x;
   const int m = EXPANDED ? E / D : 1;
   const int slots = EXPANDED ? k + m : k;
   const int W = (E + 63) >> 6;
 
-  // candidate base (prefix of cand) and row offset (prefix of min(cand, C)) of this expert
-  uint32_t base, off, total;
+  // candidate totals, candidate base (prefix of cand) and row offset (prefix of min(cand, C))
+  uint32_t base, off, n, total;
   {
-    uint32_t c = (tid < E) ? (uint32_t)cand[tid] : 0u;      // E <= 256 <= SEL_THREADS
-    uint32_t kc = c < (uint32_t)C ? c : (uint32_t)C;
-    uint32_t b = block_scan(c, scan_sh, total);
-    uint32_t o = block_scan(kc, scan_sh, total);
-    if (tid == e) { found[0] = b; found[1] = o; }
+    const uint32_t c = tid < E ? (uint32_t)cand[tid] : 0u;     // E <= 256 <= SEL_THREADS
+    const uint32_t kc = c < (uint32_t)C ? c : (uint32_t)C;
+    const uint32_t b = block_scan(c, scan_sh, total);
+    const uint32_t o = block_scan(kc, scan_sh, total);
+    if (tid == e) { found[0] = b; found[1] = o; found[2] = c; }
     __syncthreads();
-    base = found[0]; off = found[1];
+    base = found[0]; off = found[1]; n = found[2];
     __syncthreads();
   }
-  const uint32_t n = (uint32_t)cand[e];
   const uint32_t keep_n = n < (uint32_t)C ? n : (uint32_t)C;
   if (tid == 0) {
     kept[e] = (int32_t)keep_n;
@@ -154,34 +174,47 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
   for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) hist[i] = 0;
   __syncthreads();
 
-  // pass 1: list this expert's candidates in token order; first-level histogram on the way
+  // pass 1: list this expert's candidates in token order (each thread owns TPT consecutive
+  // tokens per round); first-level histogram on the way
   uint32_t* wkey = ws.key + base;
   int32_t* wtok = ws.tok + base;
   int32_t* wslot = ws.slot + base;
   uint32_t running = 0;
-  for (int64_t t0 = 0; t0 < N; t0 += SEL_THREADS) {
-    const int64_t t = t0 + tid;
-    int slot = -1;
-    uint32_t key = 0;
-    if (t < N) {
-      const int32_t* row = topk_idx + t * k;
-      for (int j = 0; j < k; ++j)
-        if (row[j] == e) slot = j;
-      if (EXPANDED) {
-        if (slot < 0 && home_group(t, N, D, token_group) == e / m) slot = k + (e % m);
-        if (slot >= 0) key = __float_as_uint(score_src[t * E + e]);
-      } else {
-        if (slot >= 0) key = __float_as_uint(score_src[t * k + slot]);
+  for (int64_t t0 = 0; t0 < N; t0 += SEL_TOKENS) {
+    // TPT sub-rounds of SEL_THREADS consecutive tokens each: all loads are issued before the
+    // first scan, so their latencies overlap; the scans then run in token order.
+    int slot[TPT];
+    uint32_t key[TPT];
+#pragma unroll
+    for (int u = 0; u < TPT; ++u) {
+      const int64_t t = t0 + (int64_t)u * SEL_THREADS + tid;
+      slot[u] = -1;
+      if (t < N) {
+        const int32_t* row = topk_idx + t * k;
+        for (int j = 0; j < k; ++j)
+          if (row[j] == e) slot[u] = j;
+        if (EXPANDED)
+          if (slot[u] < 0 && home_group(t, N, D, token_group) == e / m) slot[u] = k + (e % m);
       }
     }
-    uint32_t tot;
-    const uint32_t pos = block_scan(slot >= 0 ? 1u : 0u, scan_sh, tot);
-    if (slot >= 0) {
-      const uint32_t p = running + pos;
-      wkey[p] = key; wtok[p] = (int32_t)t; wslot[p] = slot;
-      if (need_select) atomicAdd(&hist[key >> 21], 1);
+#pragma unroll
+    for (int u = 0; u < TPT; ++u) {
+      const int64_t t = t0 + (int64_t)u * SEL_THREADS + tid;
+      key[u] = 0;
+      if (slot[u] >= 0)
+        key[u] = __float_as_uint(EXPANDED ? score_src[t * E + e] : score_src[t * k + slot[u]]);
     }
-    running += tot;
+#pragma unroll
+    for (int u = 0; u < TPT; ++u) {
+      if (t0 + (int64_t)u * SEL_THREADS >= N) break;           // uniform across the block
+      uint32_t tot;
+      const uint32_t p = running + block_scan(slot[u] >= 0 ? 1u : 0u, scan_sh, tot);
+      if (slot[u] >= 0) {
+        wkey[p] = key[u]; wtok[p] = (int32_t)(t0 + (int64_t)u * SEL_THREADS + tid); wslot[p] = slot[u];
+        if (need_select) atomicAdd(&hist[key[u] >> 21], 1);
+      }
+      running += tot;
+    }
   }
   __syncthreads();   // list and histogram complete (block-visible: same CTA wrote them)
 
@@ -194,8 +227,8 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
     return;
   }
 
-  // radix select of the C-th largest key: 11, 11, 10 bits
-  uint32_t rank = (uint32_t)C;          // C >= 1 here would be needed; C == 0 handled below
+  // radix select of the C-th largest key: 11, 11, 10 bits (C == 0 keeps nothing: no threshold)
+  uint32_t rank = (uint32_t)C;
   uint32_t tau = 0, need = 0;
   if (C > 0) {
     find_bin(hist, RADIX_BINS, rank, scan_sh, found);
@@ -204,8 +237,8 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
     for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) hist[i] = 0;
     __syncthreads();
     for (uint32_t i = tid; i < n; i += SEL_THREADS) {
-      const uint32_t key = wkey[i];
-      if ((key >> 21) == b1) atomicAdd(&hist[(key >> 10) & 2047u], 1);
+      const uint32_t kv = wkey[i];
+      if ((kv >> 21) == b1) atomicAdd(&hist[(kv >> 10) & 2047u], 1);
     }
     __syncthreads();
     find_bin(hist, RADIX_BINS, rank, scan_sh, found);
@@ -215,8 +248,8 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
     __syncthreads();
     const uint32_t prefix = (b1 << 11) | b2;
     for (uint32_t i = tid; i < n; i += SEL_THREADS) {
-      const uint32_t key = wkey[i];
-      if ((key >> 10) == prefix) atomicAdd(&hist[key & 1023u], 1);
+      const uint32_t kv = wkey[i];
+      if ((kv >> 10) == prefix) atomicAdd(&hist[kv & 1023u], 1);
     }
     __syncthreads();
     find_bin(hist, 1024, rank, scan_sh, found);
@@ -225,29 +258,38 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
     __syncthreads();
   }
 
-  // ordered pass: keep key > tau, and the first `need` with key == tau
+  // ordered pass (TPT consecutive candidates per thread): keep key > tau, and the first `need`
+  // with key == tau
   uint32_t run_gt = 0, run_eq = 0;
-  for (uint32_t i0 = 0; i0 < n; i0 += SEL_THREADS) {
-    const uint32_t i = i0 + tid;
-    uint32_t key = 0;
-    bool gt = false, eq = false;
-    if (i < n && C > 0) {
-      key = wkey[i];
-      gt = key > tau; eq = key == tau;
+  for (uint32_t i0 = 0; i0 < n; i0 += SEL_TOKENS) {
+    uint32_t kv[TPT];
+    uint32_t packed = 0;
+#pragma unroll
+    for (int u = 0; u < TPT; ++u) {
+      const uint32_t i = i0 + (uint32_t)tid * TPT + u;
+      kv[u] = (i < n && C > 0) ? wkey[i] : 0u;
+      if (i < n && C > 0) packed += (kv[u] > tau ? 1u : 0u) | (kv[u] == tau ? 0x10000u : 0u);
     }
     uint32_t tot;
-    const uint32_t packed = block_scan((gt ? 1u : 0u) | (eq ? 0x10000u : 0u), scan_sh, tot);
-    if (i < n) {
-      const uint32_t gt_before = run_gt + (packed & 0xffffu);
-      const uint32_t eq_before = run_eq + (packed >> 16);
-      const bool keep = gt || (eq && eq_before < need);
-      const int32_t t = wtok[i];
-      int32_t row = -1;
-      if (keep) {
-        row = (int32_t)(off + gt_before + (eq_before < need ? eq_before : need));
-        atomicOr(&keep_mask[(int64_t)t * W + (e >> 6)], 1ull << (e & 63));
+    const uint32_t before = block_scan(packed, scan_sh, tot);   // per round <= 4096 of each: fits 16 bits
+    uint32_t gt_before = run_gt + (before & 0xffffu);
+    uint32_t eq_before = run_eq + (before >> 16);
+#pragma unroll
+    for (int u = 0; u < TPT; ++u) {
+      const uint32_t i = i0 + (uint32_t)tid * TPT + u;
+      if (i < n) {
+        const bool gt = C > 0 && kv[u] > tau, eq = C > 0 && kv[u] == tau;
+        const bool keep = gt || (eq && eq_before < need);
+        const int32_t t = wtok[i];
+        int32_t row = -1;
+        if (keep) {
+          row = (int32_t)(off + gt_before + (eq_before < need ? eq_before : need));
+          atomicOr(&keep_mask[(int64_t)t * W + (e >> 6)], 1ull << (e & 63));
+        }
+        slot_row[(int64_t)t * slots + wslot[i]] = row;
+        gt_before += gt ? 1u : 0u;
+        eq_before += eq ? 1u : 0u;
       }
-      slot_row[(int64_t)t * slots + wslot[i]] = row;
     }
     run_gt += tot & 0xffffu;
     run_eq += tot >> 16;
@@ -258,8 +300,6 @@ template <bool EXPANDED>
 int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C, int D,
              const int32_t* token_group, uint64_t* keep_mask, int32_t* cand_out, int32_t* kept,
              int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr, size_t ws_bytes, cudaStream_t st) {
-  const int W = (E + 63) / 64;
-  const int slots = EXPANDED ? k + E / D : k;
   cudaError_t err;
   if (N == 0) {
     if ((err = cudaMemsetAsync(kept, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
@@ -271,12 +311,8 @@ int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, 
   DropWs ws = carve(ws_ptr, N, E, k, D, EXPANDED ? 1 : 0);
   int32_t* cand = cand_out ? cand_out : ws.cand;
   if ((err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
-  if ((err = cudaMemsetAsync(keep_mask, 0, sizeof(uint64_t) * N * W, st)) != cudaSuccess) return note_cuda(err);
-  if (EXPANDED) {   // local-expert slots that are already top-k slots are never written: preset -1
-    if ((err = cudaMemsetAsync(slot_row, 0xff, sizeof(int32_t) * N * slots, st)) != cudaSuccess) return note_cuda(err);
-  }
-  k_count_candidates<EXPANDED><<<(unsigned)ceil_div(N, CNT_THREADS), CNT_THREADS, sizeof(int) * E, st>>>(
-      topk_idx, N, E, k, D, token_group, cand);
+  k_count_candidates<EXPANDED><<<(unsigned)ceil_div(N, CNT_TOKENS), CNT_THREADS, sizeof(int) * E, st>>>(
+      topk_idx, N, E, k, D, token_group, cand, (unsigned long long*)keep_mask, slot_row);
   int rc = check_launch();
   if (rc != CAPMOE_OK) return rc;
   k_select<EXPANDED><<<E, SEL_THREADS, 0, st>>>(score_src, topk_idx, N, E, k, C, D, token_group, cand, ws,
@@ -336,8 +372,8 @@ namespace capmoe {
 namespace {
 
 constexpr int64_t STATIC_MAX_PAIRS = CAPMOE_STATIC_DROP_MAX_PAIRS;
-// same layout as carve(): 256 counters, then three int32 lists of STATIC_MAX_PAIRS entries
-constexpr size_t STATIC_WS_BYTES = 256 * sizeof(int32_t) + 3 * sizeof(int32_t) * (size_t)STATIC_MAX_PAIRS;
+// same layout as carve(): the candidate counters, then three int32 lists of STATIC_MAX_PAIRS entries
+constexpr size_t STATIC_WS_BYTES = sizeof(int32_t) * E_STRIDE + 3 * sizeof(int32_t) * (size_t)STATIC_MAX_PAIRS;
 static_assert((sizeof(int32_t) * (size_t)STATIC_MAX_PAIRS) % 256 == 0, "lists must stay 256-byte aligned");
 
 static __device__ __align__(256) unsigned char g_static_drop_ws[STATIC_WS_BYTES];
@@ -381,8 +417,9 @@ extern "C" int capmoe_token_drop_static(const float* topk_score, const int32_t* 
   void* ws = nullptr;
   rc = static_ws_for_current_device(&ws);
   if (rc != CAPMOE_OK) return rc;
-  // run_drop zeroes the candidate counters itself; the three lists are fully rewritten before
-  // they are read, so nothing else of the previous call's contents matters.
+  // run_drop zeroes the candidate counters itself (the only part that has to start at zero); the
+  // three lists are fully rewritten before they are read, so nothing else of the previous call's
+  // contents matters.
   return run_drop<false>(topk_score, topk_idx, N, E, k, C, 1, nullptr, keep_mask, nullptr, kept,
                          expert_offsets, slot_row, ws, STATIC_WS_BYTES, as_stream(stream));
 }

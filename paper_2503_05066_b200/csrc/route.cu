@@ -83,6 +83,69 @@ __device__ __forceinline__ float exp_fixed(float x) {
 // every lane divides; top-k is k rounds of a warp arg-max on (score, lower expert id wins).
 constexpr int SW_WARPS = 8;
 
+// The whole warp handles one token: lrow = its E logits (global or shared memory), prow = E floats
+// of scratch owned by this warp, hist = the CTA's shared-memory load histogram.
+template <int EPL>
+__device__ __forceinline__ void softmax_topk_token(const float* lrow, int E, int k, int64_t t, float* prow,
+                                                   float* __restrict__ scores, int32_t* __restrict__ topk_idx,
+                                                   float* __restrict__ topk_score, int* hist) {
+  const int lane = threadIdx.x & 31;
+  float v[EPL];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const int e = lane + 32 * i;
+    v[i] = e < E ? lrow[e] : -INFINITY;
+    mx = v[i] > mx ? v[i] : mx;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float other = __shfl_xor_sync(0xffffffffu, mx, o);
+    mx = other > mx ? other : mx;
+  }
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const int e = lane + 32 * i;
+    if (e < E) { v[i] = exp_fixed(__fsub_rn(v[i], mx)); prow[e] = v[i]; }
+  }
+  __syncwarp();
+  float sum = 0.f;
+  if (lane == 0)
+    for (int e = 0; e < E; ++e) sum = __fadd_rn(sum, prow[e]);
+  sum = __shfl_sync(0xffffffffu, sum, 0);
+  __syncwarp();                                              // prow is rewritten by the next token
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const int e = lane + 32 * i;
+    if (e < E) { v[i] = __fdiv_rn(v[i], sum); scores[t * E + e] = v[i]; }
+    else v[i] = -1.f;                                        // never selected (scores are >= 0)
+  }
+  float my_score = 0.f;
+  int my_idx = 0;
+  for (int j = 0; j < k; ++j) {
+    float best = -1.f;
+    int be = 0x7fffffff;
+#pragma unroll
+    for (int i = 0; i < EPL; ++i)                            // ascending expert id inside the lane
+      if (v[i] > best) { best = v[i]; be = lane + 32 * i; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+      if (ob > best || (ob == best && oe < be)) { best = ob; be = oe; }
+    }
+#pragma unroll
+    for (int i = 0; i < EPL; ++i)
+      if (be == lane + 32 * i) v[i] = -2.f;                  // taken
+    if (lane == j) { my_score = best; my_idx = be; }
+  }
+  if (lane < k) {
+    topk_idx[t * k + lane] = my_idx;
+    topk_score[t * k + lane] = my_score;
+    atomicAdd(&hist[my_idx], 1);
+  }
+}
+
 template <int EPL>
 __global__ void __launch_bounds__(SW_WARPS * 32)
 k_softmax_topk_warp(const float* __restrict__ logits, int64_t N, int E, int k, float* __restrict__ scores,
@@ -90,67 +153,11 @@ k_softmax_topk_warp(const float* __restrict__ logits, int64_t N, int E, int k, f
   extern __shared__ float smem[];
   float* prow = smem + (threadIdx.x >> 5) * (EPL * 32);       // this warp's E exponentials
   int* hist = reinterpret_cast<int*>(smem + SW_WARPS * EPL * 32);
-  const int lane = threadIdx.x & 31;
   for (int i = threadIdx.x; i < E; i += SW_WARPS * 32) hist[i] = 0;
   __syncthreads();
   const int64_t warps_total = (int64_t)gridDim.x * SW_WARPS;
-  for (int64_t t = (int64_t)blockIdx.x * SW_WARPS + (threadIdx.x >> 5); t < N; t += warps_total) {
-    const float* lrow = logits + t * E;
-    float v[EPL];
-    float mx = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < EPL; ++i) {
-      const int e = lane + 32 * i;
-      v[i] = e < E ? lrow[e] : -INFINITY;
-      mx = v[i] > mx ? v[i] : mx;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float other = __shfl_xor_sync(0xffffffffu, mx, o);
-      mx = other > mx ? other : mx;
-    }
-#pragma unroll
-    for (int i = 0; i < EPL; ++i) {
-      const int e = lane + 32 * i;
-      if (e < E) { v[i] = exp_fixed(__fsub_rn(v[i], mx)); prow[e] = v[i]; }
-    }
-    __syncwarp();
-    float sum = 0.f;
-    if (lane == 0)
-      for (int e = 0; e < E; ++e) sum = __fadd_rn(sum, prow[e]);
-    sum = __shfl_sync(0xffffffffu, sum, 0);
-    __syncwarp();                                              // prow is rewritten by the next token
-#pragma unroll
-    for (int i = 0; i < EPL; ++i) {
-      const int e = lane + 32 * i;
-      if (e < E) { v[i] = __fdiv_rn(v[i], sum); scores[t * E + e] = v[i]; }
-      else v[i] = -1.f;                                        // never selected (scores are >= 0)
-    }
-    float my_score = 0.f;
-    int my_idx = 0;
-    for (int j = 0; j < k; ++j) {
-      float best = -1.f;
-      int be = 0x7fffffff;
-#pragma unroll
-      for (int i = 0; i < EPL; ++i)                            // ascending expert id inside the lane
-        if (v[i] > best) { best = v[i]; be = lane + 32 * i; }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-        const int oe = __shfl_xor_sync(0xffffffffu, be, o);
-        if (ob > best || (ob == best && oe < be)) { best = ob; be = oe; }
-      }
-#pragma unroll
-      for (int i = 0; i < EPL; ++i)
-        if (be == lane + 32 * i) v[i] = -2.f;                  // taken
-      if (lane == j) { my_score = best; my_idx = be; }
-    }
-    if (lane < k) {
-      topk_idx[t * k + lane] = my_idx;
-      topk_score[t * k + lane] = my_score;
-      atomicAdd(&hist[my_idx], 1);
-    }
-  }
+  for (int64_t t = (int64_t)blockIdx.x * SW_WARPS + (threadIdx.x >> 5); t < N; t += warps_total)
+    softmax_topk_token<EPL>(logits + t * E, E, k, t, prow, scores, topk_idx, topk_score, hist);
   __syncthreads();
   for (int i = threadIdx.x; i < E; i += SW_WARPS * 32)
     if (hist[i]) atomicAdd(&load[i], hist[i]);
@@ -218,11 +225,15 @@ __device__ __forceinline__ void mma_bf16_16816(float* c, uint32_t a0, uint32_t a
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int MT, int NT>
+// FUSED: the CTA goes on to softmax / top-k / load histogram for its tokens (E <= 32), so the
+// router is a single pass over X.
+template <int MT, int NT, bool FUSED>
 __global__ void __launch_bounds__(RM_WARPS * 32)
 k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
-             const float* __restrict__ bias, int64_t N, int d, int E, float* __restrict__ logits) {
-  extern __shared__ float red[];                       // [RM_WARPS][16*MT][NT*8 + 1]
+             const float* __restrict__ bias, int64_t N, int d, int E, float* __restrict__ logits, int k,
+             float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
+             int32_t* __restrict__ load) {
+  extern __shared__ float red[];                       // [RM_WARPS][16*MT][NT*8 + 1] (+ fused scratch)
   constexpr int ROWS = 16 * MT, EP = NT * 8, LD = EP + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, q = lane & 3;
@@ -293,36 +304,57 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
     float sum = 0.f;
 #pragma unroll
     for (int wv = 0; wv < RM_WARPS; ++wv) sum += red[((size_t)wv * ROWS + r) * LD + e];
-    logits[t * E + e] = sum + (bias ? bias[e] : 0.f);
+    sum += bias ? bias[e] : 0.f;
+    logits[t * E + e] = sum;
+    if (FUSED) red[(size_t)RM_WARPS * ROWS * LD + r * 32 + e] = sum;      // final logits tile [ROWS][32]
+  }
+  if (FUSED) {
+    float* fin = red + (size_t)RM_WARPS * ROWS * LD;                       // [ROWS][32]
+    float* prow = fin + ROWS * 32 + warp * 32;                             // [RM_WARPS][32]
+    int* hist = reinterpret_cast<int*>(fin + ROWS * 32 + RM_WARPS * 32);   // [32]
+    if (threadIdx.x < 32) hist[threadIdx.x] = 0;
+    __syncthreads();
+    for (int r = warp; r < ROWS; r += RM_WARPS) {
+      const int64_t t = t0 + r;
+      if (t < N) softmax_topk_token<1>(fin + r * 32, E, k, t, prow, scores, topk_idx, topk_score, hist);
+    }
+    __syncthreads();
+    if (threadIdx.x < E && hist[threadIdx.x]) atomicAdd(&load[threadIdx.x], hist[threadIdx.x]);
   }
 }
 
 bool router_mma_ok(int d, int E) { return d % (RM_WARPS * 32) == 0 && E <= 128; }
 
-template <int MT, int NT>
+struct RouteOut { int k; float* scores; int32_t* topk_idx; float* topk_score; int32_t* load; };
+
+template <int MT, int NT, bool FUSED>
 int launch_router_mma_inst(const __nv_bfloat16* x, const __nv_bfloat16* w, const float* bias, int64_t N, int d,
-                           int E, float* logits, cudaStream_t st) {
-  const size_t smem = (size_t)RM_WARPS * 16 * MT * (NT * 8 + 1) * sizeof(float);
+                           int E, float* logits, const RouteOut& o, cudaStream_t st) {
+  size_t smem = (size_t)RM_WARPS * 16 * MT * (NT * 8 + 1) * sizeof(float);
+  if (FUSED) smem += (size_t)(16 * MT * 32 + RM_WARPS * 32 + 32) * sizeof(float);
   if (smem > 48 * 1024) {
-    cudaError_t e_ = cudaFuncSetAttribute(k_router_mma<MT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)smem);
+    cudaError_t e_ = cudaFuncSetAttribute(k_router_mma<MT, NT, FUSED>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e_ != cudaSuccess) return note_cuda(e_);
   }
-  k_router_mma<MT, NT><<<(unsigned)ceil_div(N, 16 * MT), RM_WARPS * 32, smem, st>>>(x, w, bias, N, d, E, logits);
+  k_router_mma<MT, NT, FUSED><<<(unsigned)ceil_div(N, 16 * MT), RM_WARPS * 32, smem, st>>>(
+      x, w, bias, N, d, E, logits, o.k, o.scores, o.topk_idx, o.topk_score, o.load);
   return check_launch();
 }
 
+// fused = true: the kernel also produced scores, top-k and the load histogram.
 int launch_router_mma(const __nv_bfloat16* x, const __nv_bfloat16* w, const float* bias, int64_t N, int d, int E,
-                      float* logits, cudaStream_t st) {
+                      float* logits, const RouteOut& o, bool* fused, cudaStream_t st) {
   const int nt = (E + 7) / 8;
-  if (nt <= 1) return launch_router_mma_inst<1, 1>(x, w, bias, N, d, E, logits, st);
-  if (nt <= 2) return launch_router_mma_inst<1, 2>(x, w, bias, N, d, E, logits, st);
+  *fused = nt <= 2;
+  if (nt <= 1) return launch_router_mma_inst<1, 1, true>(x, w, bias, N, d, E, logits, o, st);
+  if (nt <= 2) return launch_router_mma_inst<1, 2, true>(x, w, bias, N, d, E, logits, o, st);
   const bool wide = N >= (int64_t)32 * 2 * sm_count();      // enough tokens for 32-token CTAs to fill the GPU
-  if (nt <= 4) return wide ? launch_router_mma_inst<2, 4>(x, w, bias, N, d, E, logits, st)
-                           : launch_router_mma_inst<1, 4>(x, w, bias, N, d, E, logits, st);
-  if (nt <= 8) return wide ? launch_router_mma_inst<2, 8>(x, w, bias, N, d, E, logits, st)
-                           : launch_router_mma_inst<1, 8>(x, w, bias, N, d, E, logits, st);
-  return launch_router_mma_inst<1, 16>(x, w, bias, N, d, E, logits, st);
+  if (nt <= 4) return wide ? launch_router_mma_inst<2, 4, false>(x, w, bias, N, d, E, logits, o, st)
+                           : launch_router_mma_inst<1, 4, false>(x, w, bias, N, d, E, logits, o, st);
+  if (nt <= 8) return wide ? launch_router_mma_inst<2, 8, false>(x, w, bias, N, d, E, logits, o, st)
+                           : launch_router_mma_inst<1, 8, false>(x, w, bias, N, d, E, logits, o, st);
+  return launch_router_mma_inst<1, 16, false>(x, w, bias, N, d, E, logits, o, st);
 }
 
 }  // namespace
@@ -346,16 +378,20 @@ extern "C" int capmoe_route(const void* x, const void* w_router, const float* bi
   const float* lg = logits_in;
   if (!logits_in) {
     int rc;
+    bool fused = false;
+    const RouteOut ro{k, scores, topk_idx, topk_score, load};
     if (dtype == CAPMOE_F32)
       rc = launch_gemm<float>((const float*)x, (const float*)w_router, bias, N, d, E, logits, st);
     else if (E > 16 && router_tc_supported(N, d, E) && aligned16(x) && aligned16(w_router))
       rc = router_tc(x, w_router, bias, N, d, E, logits, st);
     else if (router_mma_ok(d, E) && aligned16(x) && aligned16(w_router))
-      rc = launch_router_mma((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, N, d, E, logits, st);
+      rc = launch_router_mma((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, N, d, E, logits, ro,
+                             &fused, st);
     else
       rc = launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, N, d, E,
                                       logits, st);
     if (rc != CAPMOE_OK) return rc;
+    if (fused) return CAPMOE_OK;
     lg = logits;
   } else if (logits && logits != logits_in) {
     err = cudaMemcpyAsync(logits, logits_in, sizeof(float) * N * E, cudaMemcpyDeviceToDevice, st);
