@@ -208,19 +208,17 @@ def main():
         return
 
     import torch
-    import torch.distributed as dist
-    from paper_2503_05066_b200 import capmoe, synth
+    from paper_2503_05066_b200 import capmoe, distrib, synth
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    info = distrib.RankInfo(rank, world, local_rank)
+    distrib.init(info, backend="nccl", device=torch.device("cuda", local_rank))
     capmoe.lib()
     peaks = _peaks()
 
-    cfg = synth.CONFIGS[args.config].with_(seed=synth.CONFIGS[args.config].seed + rank)
+    cfg = synth.CONFIGS[args.config].with_(seed=distrib.shard_seed(synth.CONFIGS[args.config].seed, info))
     if not cfg.straggler:
         args.straggler = args.straggler and False
     inp = synth.make_layer_inputs(cfg)
@@ -233,16 +231,12 @@ def main():
                                cfg.D, mode, gamma=gamma, straggler=straggler, shared=shared)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        torch.cuda.synchronize()
+        distrib.barrier(info)
         torch.cuda.synchronize()
 
     def max_over_ranks(v: float) -> float:
-        if world == 1:
-            return v
-        t = torch.tensor([v], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return distrib.max_over_ranks(v, info, device=dev)
 
     # ------------------------------------------------------------------ headline: K timed steps
     layer = make(args.mode, args.gamma, args.straggler)
@@ -269,7 +263,7 @@ def main():
     layer.set_stage_events(None)
     layer.check_device_status()
     ms_step = max_over_ranks(e0.elapsed_time(e1) / K)
-    value = world * cfg.N / (ms_step * 1e-3)
+    value = distrib.job_throughput(cfg.N, ms_step, info)
 
     stage_ms = {}
     for si, name in enumerate(capmoe.STAGE_NAMES):
@@ -323,7 +317,7 @@ def main():
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1) / K)
     nbytes = xh.numel() * xh.element_size()
-    e2e = {"value": world * cfg.N / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+    e2e = {"value": distrib.job_throughput(cfg.N, ms_e2e, info), "unit": UNIT, "ms_per_step": ms_e2e,
            "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes}
     del layer
 
@@ -369,9 +363,7 @@ def main():
             "peaks": peaks,
         }
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    distrib.finish(info)
 
 
 def layer_C(cfg, args, capmoe):

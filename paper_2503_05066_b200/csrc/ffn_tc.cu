@@ -10,7 +10,7 @@
 //   warp 0      TMA producer (one lane): ring of STAGES {A 128x64, B 256x64} bf16 tiles
 //   warp 1      MMA issuer (one lane): 128 x 256 x 16 tcgen05.mma, accumulators ping-pong
 //               between two 256-column halves of the CTA's 512 TMEM columns
-//   warps 2-5   epilogue: tcgen05.ld the finished accumulator, SwiGLU / convert, 16-byte stores,
+//   warps 2-9   epilogue: tcgen05.ld the finished accumulator, SwiGLU / convert, 16-byte stores,
 //               overlapping the next tile's MMAs
 // GEMM1 puts 128 gate rows and 128 up rows of the same output columns into one 256-row B tile,
 // so one MMA yields both halves of the SwiGLU pair.  Tiles are enumerated on the device from
@@ -35,7 +35,8 @@ constexpr int MAX_STAGES = 16;         // router ring depth limit (smaller stage
 constexpr int A_BYTES = BM * BK * 2;         // 16 KB
 constexpr int B_BYTES = BNB * BK * 2;        // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int TC_THREADS = 192;
+constexpr int EPI_WARPS = 8;              // two warps per TMEM lane quarter, each takes half the columns
+constexpr int TC_THREADS = 64 + EPI_WARPS * 32;
 constexpr int MAX_E = 256;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/ +
                            2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/;
@@ -209,7 +210,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
 
   if (tid == 0) {
     for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 128); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), EPI_WARPS * 32); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -260,14 +261,13 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int cursor = 0;
-      uint32_t kc = 0;
+      int s = 0;                                         // ring position and phase, advanced without division
+      uint32_t ph = 0;
       Tile t;
       bool ok = true;
       for (int tile = first; ok && tile < tile_hi; tile += stride) {
         if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
-        for (int kb = 0; kb < num_kb; ++kb, ++kc) {
-          const int s = (int)(kc % (uint32_t)n_stages);
-          const uint32_t ph = (kc / (uint32_t)n_stages) & 1u;
+        for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
           mbar_expect_tx(full_bar(s), stage_tx);
           const uint32_t a_dst = tiles + (uint32_t)s * (uint32_t)stage_stride;
@@ -279,6 +279,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
           } else {
             tma_load_3d(b_dst, &map_b0, kb * BK, MODE == MODE_ROUTER ? 0 : t.n0, t.e, full_bar(s));
           }
+          if (++s == n_stages) { s = 0; ph ^= 1u; }
         }
       }
     }
@@ -286,7 +287,14 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       int cursor = 0;
-      uint32_t kc = 0, it = 0;
+      uint32_t it = 0;
+      int s = 0;                                         // ring position and phase, advanced without division
+      uint32_t ph = 0;
+      // descriptors of stage 0; a stage further on adds its byte offset >> 4 to the address field
+      const uint64_t adesc0 = umma_desc(tiles);
+      const uint64_t bdesc0 = umma_desc(tiles + a_bytes);
+      const uint64_t stage_step = (uint64_t)((uint32_t)stage_stride >> 4);
+      uint64_t stage_off = 0;
       Tile t;
       bool ok = true;
       for (int tile = first; ok && tile < tile_hi; tile += stride, ++it) {
@@ -295,28 +303,28 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
         if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + b * (uint32_t)BNB;
-        for (int kb = 0; kb < num_kb; ++kb, ++kc) {
-          const int s = (int)(kc % (uint32_t)n_stages);
-          const uint32_t ph = (kc / (uint32_t)n_stages) & 1u;
+        for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_src = tiles + (uint32_t)s * (uint32_t)stage_stride;
-          const uint64_t adesc = umma_desc(a_src);
-          const uint64_t bdesc = umma_desc(a_src + a_bytes);
+          const uint64_t adesc = adesc0 + stage_off;
+          const uint64_t bdesc = bdesc0 + stage_off;
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advance 32 bytes (16 bf16) inside the swizzled 128-byte row: +2 in 16-byte units
             umma(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
           }
           umma_commit(empty_bar(s));                    // frees the stage when these MMAs have read it
+          stage_off += stage_step;
+          if (++s == n_stages) { s = 0; ph ^= 1u; stage_off = 0; }
         }
         if (ok) umma_commit(tfull_bar(b));              // accumulator complete
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..9)
     const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
     const int row_in_tile = quarter * 32 + lane;
+    const int half = (warp - 2) >> 2;                    // which half of the columns this warp converts
     int cursor = 0;
     uint32_t it = 0;
     Tile t;
@@ -332,7 +340,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       if (MODE == MODE_ROUTER) {
         float* lrow = reinterpret_cast<float*>(out_ptr) + (int64_t)(t.row0 + row_in_tile) * Nout;
 #pragma unroll 1
-        for (int c = 0; c < n_mma; c += 32) {
+        for (int c = half * 32; c < n_mma; c += 64) {
           uint32_t g[32];
           tmem_ld32(taddr + (uint32_t)c, g);
           tmem_ld_wait();
@@ -357,7 +365,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       }
       __nv_bfloat16* orow = out + (int64_t)(t.row0 + row_in_tile) * Nout + t.n0;
 #pragma unroll 1
-      for (int c = 0; c < N_TILE; c += 32) {
+      for (int c = half * (N_TILE / 2); c < (half + 1) * (N_TILE / 2); c += 32) {
         uint32_t g[32];
         uint32_t packed[16];
         if (SWIGLU) {
