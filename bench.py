@@ -32,6 +32,13 @@ if ROOT not in sys.path:
 METRIC = "MoE-layer tokens/s at Mixtral shape"
 UNIT = "tokens/s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMM launch, from single-pass ncu
+# captures (see profiles/k_ffn_tc_dram_traffic.md); key = (config, N, F, mode, gamma)
+NCU_TRAFFIC_GATE_UP = {
+    ("mixtral", 8192, 14336, "expanded_drop", 1.0): 2270196736 + 462499072,
+    ("olmoe", 4096, 1024, "expanded_drop", 1.0): 673051392 + 56401664,
+}
+
 
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -131,7 +138,7 @@ def run_reference(args, rank):
     from paper_2503_05066_b200 import synth
     if rank != 0:
         return
-    cfg = synth.CONFIGS[args.config]
+    cfg = _pick_config(args)
     inp = synth.make_layer_inputs(cfg)
     sample = args.ref_tokens or 64
     vals = []
@@ -151,6 +158,16 @@ def run_reference(args, rank):
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
+
+
+def _pick_config(args):
+    from paper_2503_05066_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    if args.N is not None:
+        cfg = cfg.with_(N=args.N)
+    if args.F is not None:
+        cfg = cfg.with_(F=args.F)
+    return cfg
 
 
 def _config_dict(cfg, args):
@@ -186,6 +203,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--config", default="mixtral")
+    ap.add_argument("--N", type=int, default=None, help="override the number of tokens (sweeps, small ncu cases)")
+    ap.add_argument("--F", type=int, default=None, help="override the expert FFN width (small ncu cases)")
     ap.add_argument("--mode", default="expanded_drop", choices=["nodrop", "token_drop", "expanded_drop"])
     ap.add_argument("--gamma", type=float, default=1.0)
     ap.add_argument("--no-straggler", dest="straggler", action="store_false")
@@ -218,7 +237,8 @@ def main():
     capmoe.lib()
     peaks = _peaks()
 
-    cfg = synth.CONFIGS[args.config].with_(seed=distrib.shard_seed(synth.CONFIGS[args.config].seed, info))
+    cfg = _pick_config(args)
+    cfg = cfg.with_(seed=distrib.shard_seed(cfg.seed, info))
     if not cfg.straggler:
         args.straggler = args.straggler and False
     inp = synth.make_layer_inputs(cfg)
@@ -288,7 +308,10 @@ def main():
         "peak_source": peaks["source"] + " (sustained cuBLAS bf16: kernel timed inside a long step)",
         "peak_burst": peaks["bf16_tflops"],
         "flops_per_launch": gemm1_flops,
-        "traffic": None,
+        # DRAM bytes of one gate/up launch (ncu, dram__bytes_read.sum + dram__bytes_write.sum; summary in
+        # profiles/k_ffn_tc_dram_traffic.md), known for the workloads that were captured
+        "traffic": NCU_TRAFFIC_GATE_UP.get((cfg.name, cfg.N, cfg.F, args.mode, args.gamma)),
+        "algorithmic_bytes": (2 * cfg.E * cfg.F * cfg.d + A * cfg.d + A * cfg.F) * elt,
         "down_gemm": {"achieved": gemm2_flops / t2 / 1e12 if t2 > 0 else None,
                       "frac": (gemm2_flops / t2 / 1e12 / peak_tf) if (t2 > 0 and peak_tf) else None},
     }

@@ -106,7 +106,7 @@ __device__ __forceinline__ void axpy_row(float (*acc)[Vec16<T>::n], const uint4*
 }
 
 template <typename T>
-__global__ void __launch_bounds__(PC_WARPS * 32)
+__global__ void __launch_bounds__(PC_WARPS * 32, 4)
 k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row,
           const float* __restrict__ perm_weight, int64_t N, int row_vecs, int chunks, int slots,
           const uint4* __restrict__ y_shared, uint4* __restrict__ y) {
