@@ -171,6 +171,13 @@ int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offsets, int E,
                        void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
                        int32_t* dev_status, void* stream);
 
+/* Self-test of the bounded device-side wait used inside the tensor-core kernels (no counterpart
+ * in the paper).  Launches one warp that waits on a barrier nothing will ever signal, with the
+ * same wait routine and a limit of limit_cycles SM clock cycles (1 .. 4e9); the wait must run
+ * out, the kernel must return normally and *dev_status must read CAPMOE_ETIMEOUT afterwards
+ * (the caller zeroes it first).  The context stays usable. */
+int capmoe_debug_wait_probe(int64_t limit_cycles, int32_t* dev_status, void* stream);
+
 /* ---------------------------------------------------------------- stage 6: combine
  * y[t] = sum over slots s with slot_row[t,s] >= 0 of perm_weight[row] * y_perm[row], added in
  * ascending slot order in fp32, plus y_shared[t] (weight 1) when y_shared is not NULL; a token

@@ -26,7 +26,7 @@ MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2}
 EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_drop_workspace_bytes", "capmoe_status_str",
            "capmoe_last_cuda_error", "capmoe_launch_count", "capmoe_ffn_uses_tensor_cores", "capmoe_route",
            "capmoe_token_drop", "capmoe_token_drop_static", "capmoe_expanded_drop", "capmoe_permute", "capmoe_grouped_ffn",
-           "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host"]
+           "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe"]
 
 
 class CapmoeError(RuntimeError):
@@ -268,6 +268,14 @@ def combine(y_perm, slot_row, perm_weight, y_shared=None, y=None, stream=None):
     _check(lib().capmoe_combine(_ptr(y_perm), _ptr(slot_row), _ptr(perm_weight), _i64(N), int(d), int(slots),
                                 _dt(y_perm), _ptr(y_shared), _ptr(y), _stream(stream)), "capmoe_combine")
     return y
+
+
+def debug_wait_probe(limit_cycles: int = 50_000_000, stream=None) -> int:
+    """Runs the bounded-wait self-test; returns the device status it produced (ETIMEOUT expected)."""
+    st = torch.zeros((1,), device="cuda", dtype=torch.int32)
+    _check(lib().capmoe_debug_wait_probe(_i64(limit_cycles), _ptr(st), _stream(stream)), "capmoe_debug_wait_probe")
+    torch.cuda.synchronize()
+    return int(st.item())
 
 
 # ----------------------------------------------------------------------------- whole layer

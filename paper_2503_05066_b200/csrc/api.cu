@@ -44,6 +44,7 @@ bool ffn_tc_supported(int d, int F, int dtype);
 int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
            const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
            int32_t* dev_status, cudaEvent_t mid, cudaStream_t st);
+int wait_probe(long long limit_cycles, int32_t* dev_status, cudaStream_t st);
 
 static int grouped_ffn_impl(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
                             const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
@@ -110,6 +111,11 @@ extern "C" const char* capmoe_status_str(int status) {
 extern "C" const char* capmoe_last_cuda_error(void) { return g_cuda_err; }
 extern "C" uint64_t capmoe_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 extern "C" int capmoe_ffn_uses_tensor_cores(int d, int F, int dtype) { return ffn_tc_supported(d, F, dtype) ? 1 : 0; }
+
+extern "C" int capmoe_debug_wait_probe(int64_t limit_cycles, int32_t* dev_status, void* stream) {
+  if (!dev_status || limit_cycles < 1 || limit_cycles > 4000000000LL) return CAPMOE_EINVAL;
+  return wait_probe((long long)limit_cycles, dev_status, as_stream(stream));
+}
 
 extern "C" int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F,
                                   int dtype, const void* w_gate, const void* w_up, const void* w_down,

@@ -66,14 +66,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false if the wait ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = WAIT_LIMIT_CYCLES) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1; it < 0x40000000u; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 127u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+      if (clock64() - t0 > limit_cycles) break;
     }
   }
   *abort_flag = 1;
@@ -444,7 +445,29 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, ui
   return r == CUDA_SUCCESS;
 }
 
+// Exercises the bounded wait on a barrier that nothing ever signals: the wait must run out, the
+// kernel must return, and the status word must say so.  One warp, no tensor memory.
+__global__ void k_wait_probe(long long limit_cycles, int32_t* __restrict__ dev_status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_cycles);
+    if (!ok && dev_status) atomicExch(dev_status, (int)CAPMOE_ETIMEOUT);
+  }
+}
+
 }  // namespace
+
+int wait_probe(long long limit_cycles, int32_t* dev_status, cudaStream_t st) {
+  k_wait_probe<<<1, 32, 0, st>>>(limit_cycles, dev_status);
+  return check_launch();
+}
 
 bool ffn_tc_supported(int d, int F, int dtype) {
   return dtype == CAPMOE_BF16 && d % 64 == 0 && F % 64 == 0 && d >= 64 && F >= 64;
