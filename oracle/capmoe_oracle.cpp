@@ -127,6 +127,24 @@ int oracle_capacity(int64_t N, int E, int k, double gamma, int round_mode, int64
   return 0;
 }
 
+// Device-level capacity n_l * gamma * N_bar = gamma * N k / D for a device holding n_l = E/D experts
+// ("Advanced Variant" paragraph), evaluated as (gamma * (N*k)) / D in double, rounded like
+// oracle_capacity, clamped to [0, N * E/D] (a device cannot hold more pairs than that).
+int oracle_device_capacity(int64_t N, int E, int k, int D, double gamma, int round_mode, int64_t* C_dev) {
+  if (N < 0 || E < 1 || k < 1 || k > E || D < 1 || E % D != 0 || !(gamma >= 0.0)) return 1;
+  const double most = (double)N * (double)(E / D);
+  double c;
+  if (std::isinf(gamma)) c = most;
+  else {
+    double v = (gamma * (double)(N * (int64_t)k)) / (double)D;
+    c = round_mode == 1 ? std::floor(v) : std::ceil(v);
+  }
+  if (c > most) c = most;
+  if (c < 0.0) c = 0.0;
+  *C_dev = (int64_t)c;
+  return 0;
+}
+
 // Router logits l[t,e] = sum_j x[t,j] w[e,j] + b[e] (the gate of Eq. 1), accumulated in
 // double, rounded once to binary32.
 void oracle_router_logits(const void* x, const void* w, const float* bias, int64_t N, int d, int E,
@@ -215,6 +233,59 @@ void oracle_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t 
   }
   for (int e = 0; e < E; ++e) cand[e] = (int32_t)cands[e].size();
   select_and_place(cands, N, E, k + m, C, keep_mask, kept, offsets, slot_row);
+}
+
+// Device-level capacity ("Advanced Variant: Device-Level Capacity-Aware Inference"): the constraint
+// is on the aggregated load of a device, N_1 + ... + N_{n_l} <= C_dev, not on each expert.  The
+// candidates of device g are all (token, expert) pairs with the expert on g (top-k pairs, plus
+// the home-device pairs when expanded != 0, as in Expanded Drop); the device keeps its
+// min(|Cand_g|, C_dev) best pairs by score, equal scores going to the lower token index and,
+// inside one token, to the lower expert id.  Rows stay expert-major, token-ascending.
+void oracle_device_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C_dev,
+                        int D, int expanded, const int32_t* token_group, uint64_t* keep_mask, int32_t* cand,
+                        int32_t* kept, int32_t* offsets, int32_t* slot_row) {
+  const int m = E / D;
+  const int slots = expanded ? k + m : k;
+  const int W = (E + 63) / 64;
+  struct Pair { float s; int32_t t; int32_t e; int32_t slot; };
+  std::vector<std::vector<Pair>> dev(D);          // per device, ordered by (token, expert)
+  std::vector<int32_t> slot_of(E);
+  for (int e = 0; e < E; ++e) cand[e] = 0;
+  for (int64_t t = 0; t < N; ++t) {
+    std::fill(slot_of.begin(), slot_of.end(), -1);
+    for (int j = 0; j < k; ++j) slot_of[topk_idx[t * k + j]] = j;
+    if (expanded) {
+      const int64_t g = home_group(t, N, D, token_group);
+      for (int i = 0; i < m; ++i)
+        if (slot_of[g * m + i] < 0) slot_of[g * m + i] = k + i;
+    }
+    for (int e = 0; e < E; ++e)                   // ascending expert id inside the token
+      if (slot_of[e] >= 0) {
+        dev[e / m].push_back(Pair{scores[t * E + e], (int32_t)t, e, slot_of[e]});
+        cand[e] += 1;
+      }
+  }
+  for (int64_t i = 0; i < N * W; ++i) keep_mask[i] = 0;
+  for (int64_t i = 0; i < N * slots; ++i) slot_row[i] = -1;
+  std::vector<std::vector<std::pair<int32_t, int32_t>>> rows(E);   // per expert: (token, slot) kept
+  for (int g = 0; g < D; ++g) {
+    std::vector<Pair> order(dev[g]);
+    std::stable_sort(order.begin(), order.end(), [](const Pair& a, const Pair& b) { return a.s > b.s; });
+    const int64_t keep_n = std::min<int64_t>((int64_t)order.size(), C_dev);
+    for (int64_t i = 0; i < keep_n; ++i) {
+      const Pair& p = order[i];
+      keep_mask[(int64_t)p.t * W + (p.e >> 6)] |= (uint64_t)1 << (p.e & 63);
+      rows[p.e].push_back({p.t, p.slot});
+    }
+  }
+  offsets[0] = 0;
+  for (int e = 0; e < E; ++e) {
+    std::sort(rows[e].begin(), rows[e].end());    // ascending token index inside the segment
+    kept[e] = (int32_t)rows[e].size();
+    int32_t row = offsets[e];
+    for (auto& ts : rows[e]) slot_row[(int64_t)ts.first * slots + ts.second] = row++;
+    offsets[e + 1] = row;
+  }
 }
 
 // Expert id served by slot s of token t (slots < k: top-k order; slots >= k: local experts).

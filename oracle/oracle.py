@@ -19,7 +19,8 @@ _SRC = os.path.join(_HERE, "capmoe_oracle.cpp")
 _LIB = os.path.join(_HERE, "libcapmoe_oracle.so")
 _lib = None
 
-__all__ = ["build", "capacity", "router_logits", "softmax", "topk", "token_drop", "expanded_drop",
+__all__ = ["build", "capacity", "device_capacity", "device_drop", "router_logits", "softmax", "topk", "token_drop",
+           "expanded_drop",
            "permute", "expert_ffn", "combine", "layer_tokens", "stats", "layer_forward", "num_threads"]
 
 
@@ -134,6 +135,37 @@ def expanded_drop(scores: np.ndarray, topk_idx: np.ndarray, C: int, D: int,
     tg = None if token_group is None else np.ascontiguousarray(token_group, np.int32)
     _load().oracle_expanded_drop(_p(scores), _p(topk_idx), _i64(N), int(E), int(k), _i64(C), int(D),
                                  _p(tg), _p(keep), _p(cand), _p(kept), _p(off), _p(slot_row))
+    return dict(keep_mask=keep, cand=cand, kept=kept, offsets=off, slot_row=slot_row)
+
+
+def device_capacity(N: int, E: int, k: int, D: int, gamma: float, round_mode: str = "ceil") -> int:
+    out = ctypes.c_int64(0)
+    rc = _load().oracle_device_capacity(_i64(N), int(E), int(k), int(D), ctypes.c_double(gamma),
+                                        0 if round_mode == "ceil" else 1, ctypes.byref(out))
+    if rc != 0:
+        raise ValueError("bad device capacity arguments")
+    return out.value
+
+
+def device_drop(scores: np.ndarray, topk_idx: np.ndarray, C_dev: int, D: int, expanded: bool,
+                token_group: Optional[np.ndarray] = None):
+    """Capacity enforced per device (sum over its E/D experts) instead of per expert."""
+    scores = np.ascontiguousarray(scores, np.float32)
+    topk_idx = np.ascontiguousarray(topk_idx, np.int32)
+    N, E = scores.shape
+    k = topk_idx.shape[1]
+    assert E % D == 0
+    m = E // D
+    W = (E + 63) // 64
+    slots = k + m if expanded else k
+    keep = np.empty((N, W), np.uint64)
+    cand = np.empty((E,), np.int32)
+    kept = np.empty((E,), np.int32)
+    off = np.empty((E + 1,), np.int32)
+    slot_row = np.empty((N, slots), np.int32)
+    tg = None if token_group is None else np.ascontiguousarray(token_group, np.int32)
+    _load().oracle_device_drop(_p(scores), _p(topk_idx), _i64(N), int(E), int(k), _i64(C_dev), int(D),
+                               int(bool(expanded)), _p(tg), _p(keep), _p(cand), _p(kept), _p(off), _p(slot_row))
     return dict(keep_mask=keep, cand=cand, kept=kept, offsets=off, slot_row=slot_row)
 
 
