@@ -139,6 +139,22 @@ int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t N
                          int32_t* cand, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row,
                          void* ws, size_t ws_bytes, void* stream);
 
+/* ---------------------------------------------------------------- device-level capacity
+ * The paper's "Advanced Variant: Device-Level Capacity-Aware Inference": the bound applies to the
+ * aggregated load of a device, N_1 + ... + N_{n_l} <= C_dev = n_l * gamma * N_bar, not to each
+ * expert.  capmoe_device_capacity evaluates (gamma*(N*k))/D like capmoe_capacity (host pointer
+ * out; clamped to [0, N*E/D]).  capmoe_device_drop keeps, per device, the C_dev best of all
+ * (token, expert) pairs whose expert lives on it - the top-k pairs, plus every pair of the token's
+ * home device when expanded != 0 (the candidate set of Expanded Drop) - by scores[t,e]; equal scores
+ * go to the lower token index and, inside a token, to the lower expert id.  Outputs have the
+ * layout of stages 2/3 (slot_row [N,k] or [N,k+E/D]; rows expert-major, token-ascending).
+ * Requires E/D <= 32.  ws: capmoe_drop_workspace_bytes(N,E,k,D,expanded) bytes. */
+int capmoe_device_capacity(int64_t N, int E, int k, int D, double gamma, int round, int64_t* C_dev);
+int capmoe_device_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
+                       int64_t C_dev, int D, int expanded, const int32_t* token_group,
+                       uint64_t* keep_mask, int32_t* cand, int32_t* kept, int32_t* expert_offsets,
+                       int32_t* slot_row, void* ws, size_t ws_bytes, void* stream);
+
 /* ---------------------------------------------------------------- stage 4: permute
  * x_perm[r] = x[t], perm_token[r] = t, perm_weight[r] = scores[t,e] for every kept (t,e) with
  * r = its slot_row entry.  slots = k after Token Drop (pass D = 0) or k+E/D after Expanded Drop.
@@ -193,8 +209,9 @@ int capmoe_combine(const void* y_perm, const int32_t* slot_row, const float* per
 typedef struct {
   /* problem */
   int64_t N; int d, E, k, F, D, dtype;
-  int mode;              /* 0 = no drop (C = N), 1 = Token Drop, 2 = Expanded Drop */
-  int64_t C;             /* capacity (ignored for mode 0) */
+  int mode;              /* 0 = no drop (C = N), 1 = Token Drop, 2 = Expanded Drop,
+                            3 / 4 = Token / Expanded Drop candidates under device-level capacity */
+  int64_t C;             /* capacity per expert (modes 1, 2) or per device (modes 3, 4); ignored for mode 0 */
   int straggler;         /* 0/1: run the FFN in straggler-emulation mode over D devices */
   /* inputs */
   const void* x; const void* w_router; const float* bias;

@@ -21,11 +21,12 @@ _lib = None
 OK, EINVAL, EUNSUPPORTED, EWORKSPACE, ECUDA, ETIMEOUT = range(6)
 F32, BF16 = 0, 1
 MODE_NODROP, MODE_TOKEN_DROP, MODE_EXPANDED_DROP = 0, 1, 2
-MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2}
+MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2, "device_token_drop": 3, "device_expanded_drop": 4}
 
 EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_drop_workspace_bytes", "capmoe_status_str",
            "capmoe_last_cuda_error", "capmoe_launch_count", "capmoe_ffn_uses_tensor_cores", "capmoe_route",
-           "capmoe_token_drop", "capmoe_token_drop_static", "capmoe_expanded_drop", "capmoe_permute", "capmoe_grouped_ffn",
+           "capmoe_token_drop", "capmoe_token_drop_static", "capmoe_expanded_drop", "capmoe_device_capacity",
+           "capmoe_device_drop", "capmoe_permute", "capmoe_grouped_ffn",
            "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe"]
 
 
@@ -225,6 +226,39 @@ def expanded_drop(scores, topk_idx, C: int, D: int, token_group=None, ws=None, s
     return out
 
 
+def device_capacity(N: int, E: int, k: int, D: int, gamma: float, round_mode: str = "ceil") -> int:
+    out = ctypes.c_int64(0)
+    _check(lib().capmoe_device_capacity(_i64(N), int(E), int(k), int(D), ctypes.c_double(gamma),
+                                        0 if round_mode == "ceil" else 1, ctypes.byref(out)),
+           "capmoe_device_capacity")
+    return out.value
+
+
+def device_drop(scores, topk_idx, C_dev: int, D: int, expanded: bool, token_group=None, ws=None, stream=None):
+    """Capacity per device instead of per expert.  -> dict(keep_mask, cand, kept, offsets, slot_row)"""
+    N, E = scores.shape
+    k = topk_idx.shape[1]
+    dev = scores.device
+    if D < 1 or E % D != 0:
+        raise CapmoeError(EINVAL, "capmoe_device_drop: E % D != 0")
+    m = E // D
+    W = (E + 63) // 64
+    slots = k + m if expanded else k
+    if ws is None:
+        ws = torch.empty((drop_workspace_bytes(N, E, k, D, expanded),), device=dev, dtype=torch.uint8)
+    out = dict(keep_mask=torch.empty((N, W), device=dev, dtype=torch.int64),
+               cand=torch.empty((E,), device=dev, dtype=torch.int32),
+               kept=torch.empty((E,), device=dev, dtype=torch.int32),
+               offsets=torch.empty((E + 1,), device=dev, dtype=torch.int32),
+               slot_row=torch.empty((N, slots), device=dev, dtype=torch.int32))
+    _check(lib().capmoe_device_drop(_ptr(scores), _ptr(topk_idx), _i64(N), int(E), int(k), _i64(C_dev), int(D),
+                                    int(bool(expanded)), _ptr(token_group), _ptr(out["keep_mask"]),
+                                    _ptr(out["cand"]), _ptr(out["kept"]), _ptr(out["offsets"]),
+                                    _ptr(out["slot_row"]), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(stream)),
+           "capmoe_device_drop")
+    return out
+
+
 def permute(x, scores, topk_idx, slot_row, A_max: int, D: int = 0, token_group=None, stream=None):
     """-> dict(x_perm [A_max,d], perm_token [A_max], perm_weight [A_max]); rows >= A are left unwritten"""
     N, d = x.shape
@@ -291,12 +325,18 @@ class MoELayer:
         self.N, self.d, self.E, self.k, self.F, self.D = N, d, E, k, F, D
         self.mode = mode
         m = E // D
-        expanded = mode == "expanded_drop"
+        expanded = mode in ("expanded_drop", "device_expanded_drop")
+        device_level = mode.startswith("device_")
         if C is None:
-            C = N if mode == "nodrop" else capacity(N, E, k, gamma, round_mode)
+            if mode == "nodrop":
+                C = N
+            elif device_level:
+                C = device_capacity(N, E, k, D, gamma, round_mode)
+            else:
+                C = capacity(N, E, k, gamma, round_mode)
         self.C = C
         self.slots = k + m if expanded else k
-        A_max = max_rows(N, E, k, D, C, expanded)
+        A_max = min(D * C, N * self.slots) if device_level else max_rows(N, E, k, D, C, expanded)
         self.A_max = A_max
         W = (E + 63) // 64
         f32 = dict(device=dev, dtype=torch.float32)

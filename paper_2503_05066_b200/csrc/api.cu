@@ -87,6 +87,23 @@ extern "C" int capmoe_capacity(int64_t N, int E, int k, double gamma, int round,
   return CAPMOE_OK;
 }
 
+extern "C" int capmoe_device_capacity(int64_t N, int E, int k, int D, double gamma, int round, int64_t* C_dev) {
+  if (!C_dev || N < 0 || E < 1 || k < 1 || k > E || D < 1 || E % D != 0 || !(gamma >= 0.0)) return CAPMOE_EINVAL;
+  if (round != CAPMOE_CAP_CEIL && round != CAPMOE_CAP_FLOOR) return CAPMOE_EINVAL;
+  const double most = (double)N * (double)(E / D);
+  double c;
+  if (std::isinf(gamma)) {
+    c = most;
+  } else {
+    const double v = (gamma * (double)(N * (int64_t)k)) / (double)D;
+    c = round == CAPMOE_CAP_FLOOR ? std::floor(v) : std::ceil(v);
+  }
+  if (c > most) c = most;
+  if (c < 0.0) c = 0.0;
+  *C_dev = (int64_t)c;
+  return CAPMOE_OK;
+}
+
 extern "C" int capmoe_max_rows(int64_t N, int E, int k, int D, int64_t C, int expanded, int64_t* A_max) {
   if (!A_max || N < 0 || E < 1 || k < 1 || k > E || C < 0) return CAPMOE_EINVAL;
   if (expanded && (D < 1 || E % D != 0)) return CAPMOE_EINVAL;
@@ -127,7 +144,7 @@ extern "C" int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offs
 
 extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if (!L) return CAPMOE_EINVAL;
-  if (L->mode < 0 || L->mode > 2) return CAPMOE_EINVAL;
+  if (L->mode < 0 || L->mode > 4) return CAPMOE_EINVAL;
   cudaStream_t st = as_stream(stream);
   auto mark = [&](int i) -> int {
     if (!L->stage_events) return CAPMOE_OK;
@@ -140,7 +157,14 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if (rc != CAPMOE_OK) return rc;
   if ((rc = mark(1)) != CAPMOE_OK) return rc;
   int slots, Dp;
-  if (L->mode == 2) {
+  if (L->mode >= 3) {                     // device-level capacity: L->C is the per-device bound
+    if (L->D < 1 || L->E % L->D != 0) return CAPMOE_EINVAL;
+    const int expanded = L->mode == 4;
+    rc = capmoe_device_drop(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, expanded, nullptr, L->keep_mask,
+                            L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream);
+    slots = expanded ? L->k + L->E / L->D : L->k;
+    Dp = expanded ? L->D : 0;
+  } else if (L->mode == 2) {
     if (L->D < 1 || L->E % L->D != 0) return CAPMOE_EINVAL;
     rc = capmoe_expanded_drop(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, nullptr, L->keep_mask,
                               L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes,
