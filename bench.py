@@ -116,7 +116,11 @@ def cpu_oracle_run(cfg, inp, mode: str, gamma: float, budget_tokens: int):
     scores = oracle.softmax(logits)
     idx, _, load = oracle.topk(scores, cfg.k)
     C = cfg.N if mode == "nodrop" else oracle.capacity(cfg.N, cfg.E, cfg.k, gamma)
-    if mode == "expanded_drop":
+    if mode.startswith("device_"):
+        expanded = mode == "device_expanded_drop"
+        r = oracle.device_drop(scores, idx, oracle.device_capacity(cfg.N, cfg.E, cfg.k, cfg.D, gamma), cfg.D, expanded)
+        Dp = cfg.D if expanded else 0
+    elif mode == "expanded_drop":
         r = oracle.expanded_drop(scores, idx, C, cfg.D)
         Dp = cfg.D
     else:
@@ -205,7 +209,7 @@ def main():
     ap.add_argument("--config", default="mixtral")
     ap.add_argument("--N", type=int, default=None, help="override the number of tokens (sweeps, small ncu cases)")
     ap.add_argument("--F", type=int, default=None, help="override the expert FFN width (small ncu cases)")
-    ap.add_argument("--mode", default="expanded_drop", choices=["nodrop", "token_drop", "expanded_drop"])
+    ap.add_argument("--mode", default="expanded_drop", choices=["nodrop", "token_drop", "expanded_drop", "device_token_drop", "device_expanded_drop"])
     ap.add_argument("--gamma", type=float, default=1.0)
     ap.add_argument("--no-straggler", dest="straggler", action="store_false")
     ap.add_argument("--no-sweep", dest="sweep", action="store_false", help="skip the other modes")
@@ -350,7 +354,9 @@ def main():
         sweep_steps = max(3, min(K, 10))
         nodrop_ms = {}
         for strag in ([False, True] if cfg.straggler else [False]):
-            for mode, gam in [("nodrop", None)] + [(m, gm) for gm in cfg.gammas for m in ("token_drop", "expanded_drop")]:
+            variants = ("token_drop", "expanded_drop") + (
+                ("device_token_drop", "device_expanded_drop") if cfg.E // cfg.D <= 32 and cfg.D < cfg.E else ())
+            for mode, gam in [("nodrop", None)] + [(m, gm) for gm in cfg.gammas for m in variants]:
                 lay = make(mode, 1.0 if gam is None else gam, strag)
                 ms = time_layer(lay, sweep_steps, 3, torch)
                 if mode == "nodrop":
@@ -390,7 +396,11 @@ def main():
 
 
 def layer_C(cfg, args, capmoe):
-    return cfg.N if args.mode == "nodrop" else capmoe.capacity(cfg.N, cfg.E, cfg.k, args.gamma)
+    if args.mode == "nodrop":
+        return cfg.N
+    if args.mode.startswith("device_"):
+        return capmoe.device_capacity(cfg.N, cfg.E, cfg.k, cfg.D, args.gamma)
+    return capmoe.capacity(cfg.N, cfg.E, cfg.k, args.gamma)
 
 
 if __name__ == "__main__":

@@ -148,7 +148,7 @@ int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t N
  * home device when expanded != 0 (the candidate set of Expanded Drop) - by scores[t,e]; equal scores
  * go to the lower token index and, inside a token, to the lower expert id.  Outputs have the
  * layout of stages 2/3 (slot_row [N,k] or [N,k+E/D]; rows expert-major, token-ascending).
- * Requires E/D <= 32.  ws: capmoe_drop_workspace_bytes(N,E,k,D,expanded) bytes. */
+ * ws: capmoe_drop_workspace_bytes(N,E,k,D,expanded) bytes. */
 int capmoe_device_capacity(int64_t N, int E, int k, int D, double gamma, int round, int64_t* C_dev);
 int capmoe_device_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
                        int64_t C_dev, int D, int expanded, const int32_t* token_group,

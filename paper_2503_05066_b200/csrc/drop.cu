@@ -16,7 +16,18 @@
 #include "common.cuh"
 
 namespace capmoe {
+
+// token-parallel select (drop_parallel.cu): large batches and device-level capacity
+size_t drop_parallel_ws_bytes(int64_t N, int E);
+int drop_parallel(const float* scores, const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
+                  int64_t C_seg, int D, int seg_m, int expanded, const int32_t* token_group, uint64_t* keep_mask,
+                  int32_t* cand_out, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr,
+                  size_t ws_bytes, cudaStream_t st);
+
 namespace {
+
+// From this many tokens on, the token-parallel select is faster than one CTA per expert.
+constexpr int64_t PARALLEL_MIN_TOKENS = 16384;
 
 constexpr int CNT_THREADS = 256;
 constexpr int TPT = 4;                               // tokens (candidates) per thread per round in k_select
@@ -320,245 +331,6 @@ int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, 
   return check_launch();
 }
 
-// ---------------------------------------------------------------------------------------------
-// Device-level capacity (the paper's "Advanced Variant"): the bound is on the aggregated load of
-// a device, so the select runs once per device over all its (token, expert) candidate pairs,
-// ordered by (token, expert id); rows stay expert-major.
-//   k_count_candidates  as above (candidate counts per expert, output initialisation)
-//   k_device_select     one CTA per device: ordered compaction of the device's pairs, radix select
-//                       of the C_dev-th key, ordered placement giving each kept pair its rank
-//                       inside its own expert (packed per-expert block scans), kept[e]
-//   k_rank_to_row       per token: rank -> row by adding the expert's offset; writes the offsets
-constexpr int MAX_M = 32;             // experts per device handled by the packed rank scans
-constexpr int RANK_FIELDS = 5;        // 12-bit per-expert counters packed in one 64-bit word
-
-__device__ __forceinline__ unsigned long long block_scan64(unsigned long long v, unsigned long long* sh,
-                                                            unsigned long long& total) {
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  unsigned long long incl = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    unsigned long long n = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += n;
-  }
-  if (lane == 31) sh[wid] = incl;
-  __syncthreads();
-  if (wid == 0) {
-    unsigned long long w = sh[lane], wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      unsigned long long n = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += n;
-    }
-    sh[lane] = wi - w;
-    if (lane == 31) sh[SEL_WARPS] = wi;
-  }
-  __syncthreads();
-  const unsigned long long res = incl - v + sh[wid];
-  total = sh[SEL_WARPS];
-  __syncthreads();
-  return res;
-}
-
-template <bool EXPANDED>
-__global__ void __launch_bounds__(SEL_THREADS)
-k_device_select(const float* __restrict__ scores, const int32_t* __restrict__ topk_idx, int64_t N, int E, int k,
-                int64_t C_dev, int D, const int32_t* __restrict__ token_group, const int32_t* __restrict__ cand,
-                DropWs ws, unsigned long long* __restrict__ keep_mask, int32_t* __restrict__ kept,
-                int32_t* __restrict__ slot_row) {
-  __shared__ int hist[RADIX_BINS];
-  __shared__ uint32_t scan_sh[SEL_WARPS + 1];
-  __shared__ unsigned long long scan64_sh[SEL_WARPS + 1];
-  __shared__ uint32_t found[3];
-  __shared__ uint32_t run_rank[MAX_M];                 // kept pairs so far, per expert of this device
-  const int g = blockIdx.x;
-  const int tid = threadIdx.x;
-  const int m = E / D;
-  const int slots = EXPANDED ? k + m : k;
-  const int W = (E + 63) >> 6;
-
-  // pairs of this device and where its list starts (devices own consecutive experts)
-  uint32_t base, n, total;
-  {
-    const uint32_t c = tid < E ? (uint32_t)cand[tid] : 0u;
-    const uint32_t b = block_scan(c, scan_sh, total);
-    const uint32_t mine = (tid < E && tid / m == g) ? c : 0u;
-    uint32_t ng;
-    block_scan(mine, scan_sh, ng);
-    if (tid == g * m) { found[0] = b; }
-    if (tid == 0) found[1] = ng;
-    __syncthreads();
-    base = found[0]; n = found[1];
-    __syncthreads();
-  }
-  const uint32_t cdev = C_dev > 0x7fffffffLL ? 0x7fffffffu : (uint32_t)C_dev;
-  const bool need_select = n > cdev;
-  for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) hist[i] = 0;
-  if (tid < MAX_M) run_rank[tid] = 0;
-  __syncthreads();
-
-  // pass 1: the device's pairs in (token, expert id) order
-  uint32_t* wkey = ws.key + base;
-  int32_t* wtok = ws.tok + base;
-  int32_t* wslot = ws.slot + base;                     // (expert index inside the device) | slot << 8
-  uint32_t running = 0;
-  for (int64_t t0 = 0; t0 < N; t0 += SEL_THREADS) {
-    const int64_t t = t0 + tid;
-    uint32_t mask = 0;                                 // bit i: expert g*m+i is a candidate of token t
-    int slot_of[MAX_M];
-    if (t < N) {
-      const int32_t* row = topk_idx + t * k;
-      const bool home = EXPANDED && home_group(t, N, D, token_group) == g;
-#pragma unroll 1
-      for (int j = 0; j < k; ++j) {
-        const int i = row[j] - g * m;
-        if (i >= 0 && i < m) { mask |= 1u << i; slot_of[i] = j; }
-      }
-      if (home) {
-        for (int i = 0; i < m; ++i)
-          if (!((mask >> i) & 1u)) { mask |= 1u << i; slot_of[i] = k + i; }
-      }
-    }
-    uint32_t tot;
-    uint32_t p = running + block_scan((uint32_t)__popc(mask), scan_sh, tot);
-    while (mask) {                                     // ascending expert id
-      const int i = __ffs(mask) - 1;
-      mask &= mask - 1;
-      const uint32_t key = __float_as_uint(scores[t * E + g * m + i]);
-      wkey[p] = key; wtok[p] = (int32_t)t; wslot[p] = i | (slot_of[i] << 8);
-      ++p;
-      if (need_select) atomicAdd(&hist[key >> 21], 1);
-    }
-    running += tot;
-  }
-  __syncthreads();
-
-  uint32_t tau = 0, need = 0;
-  if (need_select && cdev > 0) {
-    uint32_t rank = cdev;
-    find_bin(hist, RADIX_BINS, rank, scan_sh, found);
-    const uint32_t b1 = found[0]; rank = found[1];
-    __syncthreads();
-    for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) hist[i] = 0;
-    __syncthreads();
-    for (uint32_t i = tid; i < n; i += SEL_THREADS) {
-      const uint32_t kv = wkey[i];
-      if ((kv >> 21) == b1) atomicAdd(&hist[(kv >> 10) & 2047u], 1);
-    }
-    __syncthreads();
-    find_bin(hist, RADIX_BINS, rank, scan_sh, found);
-    const uint32_t b2 = found[0]; rank = found[1];
-    __syncthreads();
-    for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) hist[i] = 0;
-    __syncthreads();
-    const uint32_t prefix = (b1 << 11) | b2;
-    for (uint32_t i = tid; i < n; i += SEL_THREADS) {
-      const uint32_t kv = wkey[i];
-      if ((kv >> 10) == prefix) atomicAdd(&hist[kv & 1023u], 1);
-    }
-    __syncthreads();
-    find_bin(hist, 1024, rank, scan_sh, found);
-    tau = (prefix << 10) | found[0];
-    need = found[1];
-    __syncthreads();
-  }
-
-  // ordered pass: keep decision in list order, then the rank of each kept pair inside its expert
-  const int words = (m + RANK_FIELDS - 1) / RANK_FIELDS;
-  uint32_t run_gt = 0, run_eq = 0;
-  for (uint32_t i0 = 0; i0 < n; i0 += SEL_THREADS) {
-    const uint32_t i = i0 + tid;
-    uint32_t kv = 0;
-    int ei = 0, slot = 0;
-    bool gt = false, eq = false;
-    if (i < n) {
-      kv = wkey[i];
-      const int32_t ps = wslot[i];
-      ei = ps & 0xff; slot = ps >> 8;
-      if (!need_select) gt = true;                     // everything fits
-      else if (cdev > 0) { gt = kv > tau; eq = kv == tau; }
-    }
-    uint32_t tot;
-    const uint32_t packed = block_scan((gt ? 1u : 0u) | (eq ? 0x10000u : 0u), scan_sh, tot);
-    const bool keep = gt || (eq && run_eq + (packed >> 16) < need);
-    run_gt += tot & 0xffffu;
-    run_eq += tot >> 16;
-    uint32_t my_rank = 0;
-    for (int w = 0; w < words; ++w) {                  // experts w*5 .. w*5+4 share one 64-bit scan
-      const int f = ei - w * RANK_FIELDS;
-      const unsigned long long v = (keep && f >= 0 && f < RANK_FIELDS) ? (1ull << (12 * f)) : 0ull;
-      unsigned long long tot64;
-      const unsigned long long before = block_scan64(v, scan64_sh, tot64);
-      if (v) my_rank = run_rank[ei] + (uint32_t)((before >> (12 * f)) & 0xfffull);
-      __syncthreads();                                 // every reader of run_rank is done
-      if (tid < RANK_FIELDS && w * RANK_FIELDS + tid < m)
-        run_rank[w * RANK_FIELDS + tid] += (uint32_t)((tot64 >> (12 * tid)) & 0xfffull);
-      __syncthreads();
-    }
-    if (i < n) {
-      const int32_t t = wtok[i];
-      const int e = g * m + ei;
-      if (keep) atomicOr(&keep_mask[(int64_t)t * W + (e >> 6)], 1ull << (e & 63));
-      slot_row[(int64_t)t * slots + slot] = keep ? (int32_t)my_rank : -1;   // rank now, row later
-    }
-  }
-  __syncthreads();
-  if (tid < m) kept[g * m + tid] = (int32_t)run_rank[tid];
-}
-
-// rank inside the expert -> row of the permuted matrix; expert_offsets = exclusive prefix of kept
-__global__ void __launch_bounds__(CNT_THREADS)
-k_rank_to_row(const int32_t* __restrict__ topk_idx, int64_t N, int E, int k, int slots, int D,
-              const int32_t* __restrict__ token_group, const int32_t* __restrict__ kept,
-              int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
-  __shared__ int off[E_STRIDE + 1];
-  if (threadIdx.x == 0) {
-    int acc = 0;
-    for (int e = 0; e < E; ++e) { off[e] = acc; acc += kept[e]; }
-    off[E] = acc;
-  }
-  __syncthreads();
-  if (blockIdx.x == 0)
-    for (int i = threadIdx.x; i <= E; i += CNT_THREADS) expert_offsets[i] = off[i];
-  const int64_t t = (int64_t)blockIdx.x * CNT_THREADS + threadIdx.x;
-  if (t >= N) return;
-  const int m = E / D;
-  const int g = slots > k ? home_group(t, N, D, token_group) : 0;
-  for (int s = 0; s < slots; ++s) {
-    const int32_t r = slot_row[t * slots + s];
-    if (r < 0) continue;
-    const int e = s < k ? topk_idx[t * k + s] : g * m + (s - k);
-    slot_row[t * slots + s] = r + off[e];
-  }
-}
-
-template <bool EXPANDED>
-int run_device_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C_dev, int D,
-                    const int32_t* token_group, uint64_t* keep_mask, int32_t* cand, int32_t* kept,
-                    int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr, size_t ws_bytes, cudaStream_t st) {
-  cudaError_t err;
-  if (N == 0) {
-    if ((err = cudaMemsetAsync(kept, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
-    if ((err = cudaMemsetAsync(expert_offsets, 0, sizeof(int32_t) * (E + 1), st)) != cudaSuccess) return note_cuda(err);
-    if ((err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
-    return CAPMOE_OK;
-  }
-  if (ws_bytes < ws_bytes_needed(N, E, k, D, EXPANDED ? 1 : 0)) return CAPMOE_EWORKSPACE;
-  DropWs ws = carve(ws_ptr, N, E, k, D, EXPANDED ? 1 : 0);
-  const int slots = EXPANDED ? k + E / D : k;
-  if ((err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
-  k_count_candidates<EXPANDED><<<(unsigned)ceil_div(N, CNT_TOKENS), CNT_THREADS, sizeof(int) * E, st>>>(
-      topk_idx, N, E, k, D, token_group, cand, (unsigned long long*)keep_mask, slot_row);
-  int rc = check_launch();
-  if (rc != CAPMOE_OK) return rc;
-  k_device_select<EXPANDED><<<D, SEL_THREADS, 0, st>>>(scores, topk_idx, N, E, k, C_dev, D, token_group, cand, ws,
-                                                        (unsigned long long*)keep_mask, kept, slot_row);
-  if ((rc = check_launch()) != CAPMOE_OK) return rc;
-  k_rank_to_row<<<(unsigned)ceil_div(N, CNT_THREADS), CNT_THREADS, 0, st>>>(topk_idx, N, E, k, slots, D, token_group,
-                                                                            kept, expert_offsets, slot_row);
-  return check_launch();
-}
-
 int validate(int64_t N, int E, int k, int64_t C) {
   if (N < 0 || E < 1 || k < 1 || k > E || C < 0 || C > N) return CAPMOE_EINVAL;
   if (E > 256 || k > 32) return CAPMOE_EUNSUPPORTED;
@@ -574,7 +346,9 @@ extern "C" int capmoe_drop_workspace_bytes(int64_t N, int E, int k, int D, int e
   if (!bytes || N < 0 || E < 1 || k < 1 || k > E) return CAPMOE_EINVAL;
   if (expanded && (D < 1 || E % D != 0)) return CAPMOE_EINVAL;
   if (N * (int64_t)(expanded ? k + E / D : k) >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
-  *bytes = ws_bytes_needed(N, E, k, expanded ? D : 1, expanded);
+  const size_t a = ws_bytes_needed(N, E, k, expanded ? D : 1, expanded);
+  const size_t b = drop_parallel_ws_bytes(N, E);
+  *bytes = a > b ? a : b;
   return CAPMOE_OK;
 }
 
@@ -586,6 +360,9 @@ extern "C" int capmoe_token_drop(const float* topk_score, const int32_t* topk_id
   if (!kept || !expert_offsets) return CAPMOE_EINVAL;
   if (N > 0 && (!topk_score || !topk_idx || !keep_mask || !slot_row || !ws)) return CAPMOE_EINVAL;
   if (N * (int64_t)k >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  if (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32))
+    return drop_parallel(nullptr, topk_score, topk_idx, N, E, k, C, 1, 1, 0, nullptr, keep_mask, nullptr, kept,
+                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream));
   return run_drop<false>(topk_score, topk_idx, N, E, k, C, 1, nullptr, keep_mask, nullptr, kept,
                          expert_offsets, slot_row, ws, ws_bytes, as_stream(stream));
 }
@@ -600,6 +377,9 @@ extern "C" int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx
   if (!kept || !expert_offsets || !cand) return CAPMOE_EINVAL;
   if (N > 0 && (!scores || !topk_idx || !keep_mask || !slot_row || !ws)) return CAPMOE_EINVAL;
   if (N * (int64_t)(k + E / D) >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  if (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32))
+    return drop_parallel(scores, nullptr, topk_idx, N, E, k, C, D, 1, 1, token_group, keep_mask, cand, kept,
+                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream));
   return run_drop<true>(scores, topk_idx, N, E, k, C, D, token_group, keep_mask, cand, kept, expert_offsets,
                         slot_row, ws, ws_bytes, as_stream(stream));
 }
@@ -610,14 +390,20 @@ extern "C" int capmoe_device_drop(const float* scores, const int32_t* topk_idx, 
                                   int32_t* slot_row, void* ws, size_t ws_bytes, void* stream) {
   if (N < 0 || E < 1 || k < 1 || k > E || D < 1 || E % D != 0 || C_dev < 0) return CAPMOE_EINVAL;
   if (C_dev > N * (int64_t)(E / D)) return CAPMOE_EINVAL;
-  if (E > 256 || k > 32 || E / D > MAX_M) return CAPMOE_EUNSUPPORTED;
+  if (E > 256 || k > 32) return CAPMOE_EUNSUPPORTED;
   if (!kept || !expert_offsets || !cand) return CAPMOE_EINVAL;
   if (N > 0 && (!scores || !topk_idx || !keep_mask || !slot_row || !ws)) return CAPMOE_EINVAL;
   if (N * (int64_t)(k + E / D) >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
-  return expanded ? run_device_drop<true>(scores, topk_idx, N, E, k, C_dev, D, token_group, keep_mask, cand, kept,
-                                          expert_offsets, slot_row, ws, ws_bytes, as_stream(stream))
-                  : run_device_drop<false>(scores, topk_idx, N, E, k, C_dev, D, token_group, keep_mask, cand, kept,
-                                           expert_offsets, slot_row, ws, ws_bytes, as_stream(stream));
+  cudaStream_t st = as_stream(stream);
+  if (N == 0) {
+    cudaError_t err;
+    if ((err = cudaMemsetAsync(kept, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
+    if ((err = cudaMemsetAsync(expert_offsets, 0, sizeof(int32_t) * (E + 1), st)) != cudaSuccess) return note_cuda(err);
+    if ((err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
+    return CAPMOE_OK;
+  }
+  return drop_parallel(scores, nullptr, topk_idx, N, E, k, C_dev, D, E / D, expanded ? 1 : 0, token_group, keep_mask,
+                       cand, kept, expert_offsets, slot_row, ws, ws_bytes, st);
 }
 
 // ---------------------------------------------------------------------------------------------

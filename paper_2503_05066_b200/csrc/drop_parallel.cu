@@ -1,0 +1,365 @@
+// Token-parallel capacity select, used for large batches and for device-level capacity.
+//
+// The single-CTA-per-expert kernels in drop.cu walk the token list with block scans, which is
+// fine up to a few thousand candidates per expert but serialises at N = 65536 or when one
+// "segment" is a whole device.  Here every step is spread over all SMs (one CTA per 256 tokens):
+//
+//   segment        the set that shares one capacity: an expert (Token / Expanded Drop) or a
+//                  device (device-level capacity); S = E / seg_m segments.
+//   key            64 bits per candidate pair (t, e): score bits in the high word, the inverted
+//                  position  (2^P - 1) - (t*E + e)  in the low word.  Descending key order is
+//                  (score descending, token ascending, expert ascending): exactly the keep order,
+//                  and all keys are distinct, so "keep the C best" is just  key >= tau[segment].
+//   pk_hist        one radix level: histogram of one digit of the keys that match the prefix
+//                  found so far (integer atomics into [S][2048] counters); the last CTA to finish
+//                  picks, per segment, the bin that holds the C-th largest key, extends the prefix,
+//                  and clears the counters for the next level.  Score digits 11/11/10 bits, then
+//                  position digits; a segment stops as soon as its whole selected bin is kept
+//                  (no ties at the threshold: after the three score levels).
+//   pk_count       kept pairs per (chunk, expert)
+//   pk_scan        per expert: exclusive scan over chunks -> rank base per chunk, kept[e]
+//   pk_place       per chunk: bitmap of kept tokens per expert -> rank inside the chunk by popcount;
+//                  row = offset[e] + base[chunk][e] + rank; writes slot_row, keep_mask, offsets.
+// Every output word is written exactly once, without atomics, so nothing needs initialising
+// except the histogram area (one memset).
+#include "common.cuh"
+
+namespace capmoe {
+namespace {
+
+constexpr int CHUNK = 256;           // tokens per CTA
+constexpr int BINS = 2048;
+constexpr int MAX_LEVELS = 6;
+constexpr int MAX_SEG = 256;
+
+struct Level { int shift, bits; };
+
+struct SegState {                    // one per segment, in global memory
+  unsigned long long prefix;         // key bits fixed so far (tau once done)
+  uint32_t rank;                     // how many keys of the current bin are still to be kept
+  uint32_t done;                     // 1: tau final
+  uint32_t n;                        // candidate pairs of the segment
+  uint32_t pad;
+};
+
+struct PWs {
+  uint32_t* hist;        // [S][BINS]
+  uint32_t* ticket;      // [8]
+  int32_t* cand;         // [256]
+  SegState* seg;         // [S]
+  int32_t* cnt;          // [chunks][E] kept pairs per chunk and expert
+  int32_t* base;         // [chunks][E] exclusive scan of cnt over chunks
+};
+
+inline size_t al256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct PArgs {
+  const float* scores;       // [N,E] or null (then only top-k slots exist and topk_score is used)
+  const float* topk_score;   // [N,k] or null
+  const int32_t* topk_idx;   // [N,k]
+  const int32_t* token_group;
+  int64_t N;
+  int E, k, D, m, seg_m, slots, expanded, pos_bits;
+  unsigned long long C_seg;
+};
+
+// Expert and key of slot s of token t; returns false if the slot is not a candidate.
+__device__ __forceinline__ bool pair_of(const PArgs& a, int64_t t, int s, const int32_t* row, int home, int& e,
+                                        unsigned long long& key) {
+  float sc;
+  if (s < a.k) {
+    e = row[s];
+    sc = a.topk_score ? a.topk_score[t * a.k + s] : a.scores[t * a.E + e];
+  } else {
+    e = home * a.m + (s - a.k);
+    for (int j = 0; j < a.k; ++j)
+      if (row[j] == e) return false;                 // already a top-k slot
+    sc = a.scores[t * a.E + e];
+  }
+  const unsigned long long pos = (unsigned long long)t * (unsigned)a.E + (unsigned)e;
+  const unsigned long long inv = ((1ull << a.pos_bits) - 1ull) - pos;
+  key = ((unsigned long long)__float_as_uint(sc) << 32) | inv;
+  return true;
+}
+
+__global__ void __launch_bounds__(CHUNK)
+pk_hist(PArgs a, PWs w, int level, Level lv, int n_levels, int first_level_counts_cand) {
+  __shared__ int cand_s[MAX_SEG];
+  __shared__ int is_last;
+  const int S = a.E / a.seg_m;
+  const int tid = threadIdx.x;
+  if (first_level_counts_cand)
+    for (int i = tid; i < a.E; i += CHUNK) cand_s[i] = 0;
+  __syncthreads();
+  const int64_t t = (int64_t)blockIdx.x * CHUNK + tid;
+  if (t < a.N) {
+    const int32_t* row = a.topk_idx + t * a.k;
+    const int home = a.expanded ? home_group(t, a.N, a.D, a.token_group) : 0;
+    for (int s = 0; s < a.slots; ++s) {
+      int e;
+      unsigned long long key;
+      if (!pair_of(a, t, s, row, home, e, key)) continue;
+      if (first_level_counts_cand) atomicAdd(&cand_s[e], 1);
+      const int sg = e / a.seg_m;
+      if (level > 0) {
+        const SegState st = w.seg[sg];
+        if (st.done) continue;
+        const int hi = lv.shift + lv.bits;                       // < 64 for every level after the first
+        if ((key >> hi) != (st.prefix >> hi)) continue;
+      }
+      const uint32_t digit = (uint32_t)(key >> lv.shift) & ((1u << lv.bits) - 1u);
+      atomicAdd(&w.hist[(size_t)sg * BINS + digit], 1u);
+    }
+  }
+  __syncthreads();
+  if (first_level_counts_cand)
+    for (int i = tid; i < a.E; i += CHUNK)
+      if (cand_s[i]) atomicAdd(&w.cand[i], cand_s[i]);
+  // the last CTA to arrive resolves this level for every segment
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = (atomicAdd(&w.ticket[level], 1u) == gridDim.x - 1) ? 1 : 0;
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const int warp = tid >> 5, lane = tid & 31;
+  const int nb = 1 << lv.bits;
+  for (int sg = warp; sg < S; sg += CHUNK / 32) {
+    uint32_t* h = w.hist + (size_t)sg * BINS;
+    SegState st;
+    if (level == 0) { st.prefix = 0; st.rank = 0; st.done = 0; st.n = 0; st.pad = 0; }
+    else st = w.seg[sg];
+    // lane owns bins [nb-1 - 64*lane - 63, nb-1 - 64*lane] scanned from the top down (nb <= 2048)
+    uint32_t local = 0;
+    const int per = (nb + 31) / 32;
+    for (int i = 0; i < per; ++i) {
+      const int b = nb - 1 - (lane * per + i);
+      if (b >= 0) local += __ldcg(&h[b]);
+    }
+    uint32_t incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+    if (level == 0) {
+      st.n = total;
+      const unsigned long long C = a.C_seg;
+      if (C == 0) { st.prefix = ~0ull; st.done = 1; }                       // keep nothing
+      else if ((unsigned long long)total <= C) { st.prefix = 0; st.done = 1; }   // keep everything
+      else st.rank = (uint32_t)C;
+    }
+    if (!st.done) {
+      const uint32_t before = incl - local;                    // keys in bins above this lane's range
+      int found_bin = -1;
+      uint32_t found_rank = 0, found_cnt = 0;
+      if (before < st.rank && st.rank <= incl) {               // the rank-th largest is in my range
+        uint32_t acc = before;
+        for (int i = 0; i < per; ++i) {
+          const int b = nb - 1 - (lane * per + i);
+          const uint32_t c = b >= 0 ? __ldcg(&h[b]) : 0u;
+          if (acc < st.rank && st.rank <= acc + c) { found_bin = b; found_rank = st.rank - acc; found_cnt = c; break; }
+          acc += c;
+        }
+      }
+      const unsigned who = __ballot_sync(0xffffffffu, found_bin >= 0);
+      const int src = __ffs(who) - 1;                          // exactly one lane finds it
+      found_bin = __shfl_sync(0xffffffffu, found_bin, src);
+      found_rank = __shfl_sync(0xffffffffu, found_rank, src);
+      found_cnt = __shfl_sync(0xffffffffu, found_cnt, src);
+      st.prefix |= (unsigned long long)(unsigned)found_bin << lv.shift;
+      st.rank = found_rank;
+      if (found_rank == found_cnt || level == n_levels - 1) st.done = 1;    // the whole bin is kept
+    }
+    for (int i = lane; i < nb; i += 32) h[i] = 0u;              // ready for the next level
+    if (lane == 0) w.seg[sg] = st;
+  }
+}
+
+__global__ void __launch_bounds__(CHUNK)
+pk_count(PArgs a, PWs w) {
+  __shared__ int cnt_s[MAX_SEG];
+  const int tid = threadIdx.x;
+  for (int i = tid; i < a.E; i += CHUNK) cnt_s[i] = 0;
+  __syncthreads();
+  const int64_t t = (int64_t)blockIdx.x * CHUNK + tid;
+  if (t < a.N) {
+    const int32_t* row = a.topk_idx + t * a.k;
+    const int home = a.expanded ? home_group(t, a.N, a.D, a.token_group) : 0;
+    for (int s = 0; s < a.slots; ++s) {
+      int e;
+      unsigned long long key;
+      if (!pair_of(a, t, s, row, home, e, key)) continue;
+      if (key >= w.seg[e / a.seg_m].prefix) atomicAdd(&cnt_s[e], 1);
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < a.E; i += CHUNK) w.cnt[(int64_t)blockIdx.x * a.E + i] = cnt_s[i];
+}
+
+// one CTA per expert: exclusive scan of its per-chunk counts
+__global__ void __launch_bounds__(CHUNK)
+pk_scan(PWs w, int E, int chunks, int32_t* __restrict__ kept, int32_t* __restrict__ cand_out) {
+  __shared__ int warp_tot[CHUNK / 32 + 1];
+  const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  int running = 0;
+  for (int c0 = 0; c0 < chunks; c0 += CHUNK) {
+    const int c = c0 + tid;
+    const int v = c < chunks ? w.cnt[(int64_t)c * E + e] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    if (tid == 0) {
+      int acc = 0;
+      for (int i = 0; i < CHUNK / 32; ++i) { const int x = warp_tot[i]; warp_tot[i] = acc; acc += x; }
+      warp_tot[CHUNK / 32] = acc;
+    }
+    __syncthreads();
+    if (c < chunks) w.base[(int64_t)c * E + e] = running + warp_tot[wid] + incl - v;
+    running += warp_tot[CHUNK / 32];
+    __syncthreads();
+  }
+  if (tid == 0) {
+    kept[e] = running;
+    if (cand_out) cand_out[e] = w.cand[e];
+  }
+}
+
+__global__ void __launch_bounds__(CHUNK)
+pk_place(PArgs a, PWs w, const int32_t* __restrict__ kept, unsigned long long* __restrict__ keep_mask,
+         int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
+  __shared__ int off[MAX_SEG + 1];
+  __shared__ uint32_t bitmap[MAX_SEG][CHUNK / 32];
+  __shared__ int wtot[CHUNK / 32 + 1];
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  // offsets = exclusive prefix of kept (E <= 256 = CHUNK)
+  {
+    const int v = tid < a.E ? kept[tid] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) wtot[wid] = incl;
+    __syncthreads();
+    if (tid == 0) {
+      int acc = 0;
+      for (int i = 0; i < CHUNK / 32; ++i) { const int x = wtot[i]; wtot[i] = acc; acc += x; }
+      wtot[CHUNK / 32] = acc;
+    }
+    __syncthreads();
+    if (tid < a.E) off[tid] = wtot[wid] + incl - v;
+    if (tid == 0) off[a.E] = wtot[CHUNK / 32];
+  }
+  for (int i = tid; i < a.E * (CHUNK / 32); i += CHUNK) (&bitmap[0][0])[i] = 0u;
+  __syncthreads();
+  if (blockIdx.x == 0)
+    for (int i = tid; i <= a.E; i += CHUNK) expert_offsets[i] = off[i];
+
+  const int64_t t = (int64_t)blockIdx.x * CHUNK + tid;
+  const bool live = t < a.N;
+  const int32_t* row = a.topk_idx + (live ? t : 0) * a.k;
+  const int home = (live && a.expanded) ? home_group(t, a.N, a.D, a.token_group) : 0;
+  const int W = (a.E + 63) >> 6;
+  if (live) {
+    for (int s = 0; s < a.slots; ++s) {
+      int e;
+      unsigned long long key;
+      if (!pair_of(a, t, s, row, home, e, key)) continue;
+      if (key >= w.seg[e / a.seg_m].prefix) atomicOr(&bitmap[e][wid], 1u << lane);
+    }
+  }
+  __syncthreads();
+  if (!live) return;
+  unsigned long long mask[4] = {0ull, 0ull, 0ull, 0ull};        // E <= 256
+  for (int s = 0; s < a.slots; ++s) {
+    int e;
+    unsigned long long key;
+    int32_t out = -1;
+    if (pair_of(a, t, s, row, home, e, key) && ((bitmap[e][wid] >> lane) & 1u)) {
+      int r = __popc(bitmap[e][wid] & ((1u << lane) - 1u));
+      for (int i = 0; i < wid; ++i) r += __popc(bitmap[e][i]);
+      out = off[e] + w.base[(int64_t)blockIdx.x * a.E + e] + r;
+      mask[e >> 6] |= 1ull << (e & 63);
+    }
+    slot_row[t * a.slots + s] = out;
+  }
+  for (int i = 0; i < W; ++i) keep_mask[t * W + i] = mask[i];
+}
+
+PWs carve_p(void* ws, int64_t N, int E, int S) {
+  const int64_t chunks = ceil_div(N, CHUNK);
+  char* p = (char*)ws;
+  PWs w;
+  w.hist = (uint32_t*)p;  p += al256(sizeof(uint32_t) * (size_t)S * BINS);
+  w.ticket = (uint32_t*)p; p += 256;
+  w.cand = (int32_t*)p;   p += al256(sizeof(int32_t) * 256);
+  w.seg = (SegState*)p;   p += al256(sizeof(SegState) * (size_t)S);
+  w.cnt = (int32_t*)p;    p += al256(sizeof(int32_t) * (size_t)chunks * E);
+  w.base = (int32_t*)p;
+  return w;
+}
+
+}  // namespace
+
+size_t drop_parallel_ws_bytes(int64_t N, int E) {
+  const int64_t chunks = ceil_div(N, CHUNK);
+  // sized for the largest segment count (S = E)
+  return al256(sizeof(uint32_t) * (size_t)E * BINS) + 256 + al256(sizeof(int32_t) * 256) +
+         al256(sizeof(SegState) * (size_t)E) + 2 * al256(sizeof(int32_t) * (size_t)chunks * E);
+}
+
+// C_seg: capacity of one segment (expert: C; device: C_dev).  seg_m: experts per segment.
+int drop_parallel(const float* scores, const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
+                  int64_t C_seg, int D, int seg_m, int expanded, const int32_t* token_group, uint64_t* keep_mask,
+                  int32_t* cand_out, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr,
+                  size_t ws_bytes, cudaStream_t st) {
+  if (E > MAX_SEG) return CAPMOE_EUNSUPPORTED;
+  if ((unsigned long long)N * (unsigned)E >= (1ull << 32)) return CAPMOE_EUNSUPPORTED;   // position word
+  if (ws_bytes < drop_parallel_ws_bytes(N, E)) return CAPMOE_EWORKSPACE;
+  const int S = E / seg_m;
+  PWs w = carve_p(ws_ptr, N, E, S);
+  PArgs a;
+  a.scores = scores; a.topk_score = topk_score; a.topk_idx = topk_idx; a.token_group = token_group;
+  a.N = N; a.E = E; a.k = k; a.D = D; a.m = expanded ? E / D : 1; a.seg_m = seg_m;
+  a.slots = expanded ? k + E / D : k; a.expanded = expanded;
+  int pos_bits = 1;
+  while ((1ull << pos_bits) < (unsigned long long)N * (unsigned)E) ++pos_bits;
+  a.pos_bits = pos_bits;
+  a.C_seg = (unsigned long long)C_seg;
+  // radix levels: the score word top down (11, 11, 10 bits), then the position word
+  Level lv[MAX_LEVELS];
+  int nl = 0;
+  lv[nl++] = {53, 11}; lv[nl++] = {42, 11}; lv[nl++] = {32, 10};
+  int left = pos_bits;
+  while (left > 0) {
+    const int b = left > 11 ? (left % 11 ? left % 11 : 11) : left;
+    lv[nl++] = {left - b, b};
+    left -= b;
+  }
+  // hist, tickets and candidate counters start at zero
+  const size_t zero_bytes = (size_t)((char*)w.seg - (char*)w.hist);
+  cudaError_t err = cudaMemsetAsync(w.hist, 0, zero_bytes, st);
+  if (err != cudaSuccess) return note_cuda(err);
+  const unsigned chunks = (unsigned)ceil_div(N, CHUNK);
+  int rc;
+  for (int l = 0; l < nl; ++l) {
+    pk_hist<<<chunks, CHUNK, 0, st>>>(a, w, l, lv[l], nl, l == 0 ? 1 : 0);
+    if ((rc = check_launch()) != CAPMOE_OK) return rc;
+  }
+  pk_count<<<chunks, CHUNK, 0, st>>>(a, w);
+  if ((rc = check_launch()) != CAPMOE_OK) return rc;
+  pk_scan<<<E, CHUNK, 0, st>>>(w, E, (int)chunks, kept, cand_out);
+  if ((rc = check_launch()) != CAPMOE_OK) return rc;
+  pk_place<<<chunks, CHUNK, 0, st>>>(a, w, kept, (unsigned long long*)keep_mask, expert_offsets, slot_row);
+  return check_launch();
+}
+
+}  // namespace capmoe

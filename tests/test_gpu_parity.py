@@ -111,6 +111,13 @@ DROP_CASES = [
     (100, 8, 2, 2, float("inf"), 0.0),
     (1, 8, 2, 2, 1.0, 0.0),
     (7, 4, 1, 2, 1.0, 0.0),
+    # large batches take the token-parallel select
+    (20000, 8, 2, 2, 1.0, 0.5),      # ties at the threshold resolved by position
+    (16384, 64, 8, 8, 1.0, 0.0),
+    (17001, 60, 4, 4, 0.5, 1.0),
+    (16400, 130, 6, 10, 1.0, 0.0),
+    (16384, 8, 2, 2, 0.0, 0.0),
+    (16384, 8, 2, 2, float("inf"), 0.0),
 ]
 
 
