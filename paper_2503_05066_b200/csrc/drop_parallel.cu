@@ -11,11 +11,12 @@
 //                  (score descending, token ascending, expert ascending): exactly the keep order,
 //                  and all keys are distinct, so "keep the C best" is just  key >= tau[segment].
 //   pk_hist        one radix level: histogram of one digit of the keys that match the prefix
-//                  found so far (integer atomics into [S][2048] counters); the last CTA to finish
-//                  picks, per segment, the bin that holds the C-th largest key, extends the prefix,
-//                  and clears the counters for the next level.  Score digits 11/11/10 bits, then
+//                  found so far (integer atomics into [S][2048] counters).
+//   pk_find        one CTA per segment: the bin that holds the C-th largest key extends the prefix;
+//                  clears the counters for the next level.  Score digits 11/11/10 bits, then
 //                  position digits; a segment stops as soon as its whole selected bin is kept
-//                  (no ties at the threshold: after the three score levels).
+//                  (no ties at the threshold: after the three score levels), and once no segment
+//                  is left the remaining levels return at once.
 //   pk_count       kept pairs per (chunk, expert)
 //   pk_scan        per expert: exclusive scan over chunks -> rank base per chunk, kept[e]
 //   pk_place       per chunk: bitmap of kept tokens per expert -> rank inside the chunk by popcount;
@@ -44,7 +45,7 @@ struct SegState {                    // one per segment, in global memory
 
 struct PWs {
   uint32_t* hist;        // [S][BINS]
-  uint32_t* ticket;      // [8]
+  uint32_t* active;      // [8] per level: segments that still need another level
   int32_t* cand;         // [256]
   SegState* seg;         // [S]
   int32_t* cnt;          // [chunks][E] kept pairs per chunk and expert
@@ -83,11 +84,10 @@ __device__ __forceinline__ bool pair_of(const PArgs& a, int64_t t, int s, const 
 }
 
 __global__ void __launch_bounds__(CHUNK)
-pk_hist(PArgs a, PWs w, int level, Level lv, int n_levels, int first_level_counts_cand) {
+pk_hist(PArgs a, PWs w, int level, Level lv, int first_level_counts_cand) {
   __shared__ int cand_s[MAX_SEG];
-  __shared__ int is_last;
-  const int S = a.E / a.seg_m;
   const int tid = threadIdx.x;
+  if (level > 0 && __ldcg(&w.active[level - 1]) == 0u) return;       // every segment already has its tau
   if (first_level_counts_cand)
     for (int i = tid; i < a.E; i += CHUNK) cand_s[i] = 0;
   __syncthreads();
@@ -115,65 +115,80 @@ pk_hist(PArgs a, PWs w, int level, Level lv, int n_levels, int first_level_count
   if (first_level_counts_cand)
     for (int i = tid; i < a.E; i += CHUNK)
       if (cand_s[i]) atomicAdd(&w.cand[i], cand_s[i]);
-  // the last CTA to arrive resolves this level for every segment
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(&w.ticket[level], 1u) == gridDim.x - 1) ? 1 : 0;
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  const int warp = tid >> 5, lane = tid & 31;
+}
+
+// One CTA per segment: pick the bin that holds the rank-th largest key of this level, extend the
+// prefix, clear the counters.  Thread i owns 8 consecutive bins, highest bins first.
+__global__ void __launch_bounds__(CHUNK)
+pk_find(PWs w, unsigned long long C_seg, int level, Level lv, int n_levels) {
+  __shared__ uint32_t wtot[CHUNK / 32 + 1];
+  __shared__ uint32_t res[3];
+  const int sg = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (level > 0 && __ldcg(&w.active[level - 1]) == 0u) return;
+  uint32_t* h = w.hist + (size_t)sg * BINS;
+  SegState st;
+  if (level == 0) { st.prefix = 0; st.rank = 0; st.done = 0; st.n = 0; st.pad = 0; }
+  else st = w.seg[sg];
+  if (st.done) return;                                            // nothing was counted for it
   const int nb = 1 << lv.bits;
-  for (int sg = warp; sg < S; sg += CHUNK / 32) {
-    uint32_t* h = w.hist + (size_t)sg * BINS;
-    SegState st;
-    if (level == 0) { st.prefix = 0; st.rank = 0; st.done = 0; st.n = 0; st.pad = 0; }
-    else st = w.seg[sg];
-    // lane owns bins [nb-1 - 64*lane - 63, nb-1 - 64*lane] scanned from the top down (nb <= 2048)
-    uint32_t local = 0;
-    const int per = (nb + 31) / 32;
-    for (int i = 0; i < per; ++i) {
-      const int b = nb - 1 - (lane * per + i);
-      if (b >= 0) local += __ldcg(&h[b]);
-    }
-    uint32_t incl = local;
+  constexpr int PER = BINS / CHUNK;                               // 8
+  uint32_t c[PER];
+  uint32_t local = 0;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += v;
-    }
-    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-    if (level == 0) {
-      st.n = total;
-      const unsigned long long C = a.C_seg;
-      if (C == 0) { st.prefix = ~0ull; st.done = 1; }                       // keep nothing
-      else if ((unsigned long long)total <= C) { st.prefix = 0; st.done = 1; }   // keep everything
-      else st.rank = (uint32_t)C;
-    }
-    if (!st.done) {
-      const uint32_t before = incl - local;                    // keys in bins above this lane's range
-      int found_bin = -1;
-      uint32_t found_rank = 0, found_cnt = 0;
-      if (before < st.rank && st.rank <= incl) {               // the rank-th largest is in my range
-        uint32_t acc = before;
-        for (int i = 0; i < per; ++i) {
-          const int b = nb - 1 - (lane * per + i);
-          const uint32_t c = b >= 0 ? __ldcg(&h[b]) : 0u;
-          if (acc < st.rank && st.rank <= acc + c) { found_bin = b; found_rank = st.rank - acc; found_cnt = c; break; }
-          acc += c;
+  for (int i = 0; i < PER; ++i) {
+    const int b = nb - 1 - (tid * PER + i);
+    c[i] = b >= 0 ? __ldcg(&h[b]) : 0u;
+    local += c[i];
+  }
+  uint32_t incl = local;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) wtot[wid] = incl;
+  if (tid < 3) res[tid] = 0xffffffffu;
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t acc = 0;
+    for (int i = 0; i < CHUNK / 32; ++i) { const uint32_t x = wtot[i]; wtot[i] = acc; acc += x; }
+    wtot[CHUNK / 32] = acc;
+  }
+  __syncthreads();
+  const uint32_t total = wtot[CHUNK / 32];
+  const uint32_t before = wtot[wid] + incl - local;               // keys in bins above this thread's
+  if (level == 0) {
+    st.n = total;
+    if (C_seg == 0) { st.prefix = ~0ull; st.done = 1; }                          // keep nothing
+    else if ((unsigned long long)total <= C_seg) { st.prefix = 0; st.done = 1; } // keep everything
+    else st.rank = (uint32_t)C_seg;
+  }
+  if (!st.done) {
+    if (before < st.rank && st.rank <= before + local) {          // exactly one thread
+      uint32_t acc = before;
+#pragma unroll
+      for (int i = 0; i < PER; ++i) {
+        if (acc < st.rank && st.rank <= acc + c[i]) {
+          res[0] = (uint32_t)(nb - 1 - (tid * PER + i)); res[1] = st.rank - acc; res[2] = c[i];
         }
+        acc += c[i];
       }
-      const unsigned who = __ballot_sync(0xffffffffu, found_bin >= 0);
-      const int src = __ffs(who) - 1;                          // exactly one lane finds it
-      found_bin = __shfl_sync(0xffffffffu, found_bin, src);
-      found_rank = __shfl_sync(0xffffffffu, found_rank, src);
-      found_cnt = __shfl_sync(0xffffffffu, found_cnt, src);
-      st.prefix |= (unsigned long long)(unsigned)found_bin << lv.shift;
-      st.rank = found_rank;
-      if (found_rank == found_cnt || level == n_levels - 1) st.done = 1;    // the whole bin is kept
     }
-    for (int i = lane; i < nb; i += 32) h[i] = 0u;              // ready for the next level
-    if (lane == 0) w.seg[sg] = st;
+  }
+  __syncthreads();
+  if (!st.done) {
+    st.prefix |= (unsigned long long)res[0] << lv.shift;
+    st.rank = res[1];
+    if (res[1] == res[2] || level == n_levels - 1) st.done = 1;   // the whole selected bin is kept
+  }
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const int b = nb - 1 - (tid * PER + i);
+    if (b >= 0) h[b] = 0u;                                         // ready for the next level
+  }
+  if (tid == 0) {
+    w.seg[sg] = st;
+    if (!st.done) atomicAdd(&w.active[level], 1u);
   }
 }
 
@@ -299,7 +314,7 @@ PWs carve_p(void* ws, int64_t N, int E, int S) {
   char* p = (char*)ws;
   PWs w;
   w.hist = (uint32_t*)p;  p += al256(sizeof(uint32_t) * (size_t)S * BINS);
-  w.ticket = (uint32_t*)p; p += 256;
+  w.active = (uint32_t*)p; p += 256;
   w.cand = (int32_t*)p;   p += al256(sizeof(int32_t) * 256);
   w.seg = (SegState*)p;   p += al256(sizeof(SegState) * (size_t)S);
   w.cnt = (int32_t*)p;    p += al256(sizeof(int32_t) * (size_t)chunks * E);
@@ -351,7 +366,9 @@ int drop_parallel(const float* scores, const float* topk_score, const int32_t* t
   const unsigned chunks = (unsigned)ceil_div(N, CHUNK);
   int rc;
   for (int l = 0; l < nl; ++l) {
-    pk_hist<<<chunks, CHUNK, 0, st>>>(a, w, l, lv[l], nl, l == 0 ? 1 : 0);
+    pk_hist<<<chunks, CHUNK, 0, st>>>(a, w, l, lv[l], l == 0 ? 1 : 0);
+    if ((rc = check_launch()) != CAPMOE_OK) return rc;
+    pk_find<<<S, CHUNK, 0, st>>>(w, a.C_seg, l, lv[l], nl);
     if ((rc = check_launch()) != CAPMOE_OK) return rc;
   }
   pk_count<<<chunks, CHUNK, 0, st>>>(a, w);
