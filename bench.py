@@ -355,7 +355,7 @@ def main():
         nodrop_ms = {}
         for strag in ([False, True] if cfg.straggler else [False]):
             variants = ("token_drop", "expanded_drop") + (
-                ("device_token_drop", "device_expanded_drop") if cfg.E // cfg.D <= 32 and cfg.D < cfg.E else ())
+                ("device_token_drop", "device_expanded_drop") if cfg.D < cfg.E else ())
             for mode, gam in [("nodrop", None)] + [(m, gm) for gm in cfg.gammas for m in variants]:
                 lay = make(mode, 1.0 if gam is None else gam, strag)
                 ms = time_layer(lay, sweep_steps, 3, torch)

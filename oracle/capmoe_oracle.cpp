@@ -235,6 +235,83 @@ void oracle_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t 
   select_and_place(cands, N, E, k + m, C, keep_mask, kept, offsets, slot_row);
 }
 
+// Drop metrics ("Order", "Reverse Order", "Random", "Score" in the Token Drop paragraph).  Each
+// (token, expert) entry gets a 32-bit key; the drop keeps the entries with the largest keys, equal
+// keys going to the lower token index.
+//   metric 0  Score          key = bit pattern of the score (non-negative floats order like their bits)
+//   metric 1  Order          one constant key: everything ties, so earlier tokens fill the capacity
+//   metric 2  Reverse Order  key = token index: later tokens win, earlier ones are removed
+//   metric 3  Random         key = high word of a 64-bit mix of (seed, t*E + e): every candidate
+//                            has the same chance
+// scores [N,cols]; idx [N,cols] expert ids, or null when cols == E and column c is expert c.
+static inline uint64_t mix64(uint64_t z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+void oracle_drop_keys(int metric, uint64_t seed, const float* scores, const int32_t* idx, int64_t N, int cols,
+                      int E, uint32_t* keys) {
+  for (int64_t t = 0; t < N; ++t)
+    for (int c = 0; c < cols; ++c) {
+      const int64_t i = t * cols + c;
+      const int e = idx ? idx[i] : c;
+      uint32_t key;
+      if (metric == 0) key = bits_from_f32(scores[i]);
+      else if (metric == 1) key = 0x3f800000u;
+      else if (metric == 2) key = (uint32_t)t;
+      else key = (uint32_t)(mix64(seed + 0x9E3779B97F4A7C15ull * ((uint64_t)t * (uint64_t)E + (uint64_t)e + 1ull)) >> 32);
+      keys[i] = key;
+    }
+}
+
+// Token Drop / Expanded Drop on arbitrary 32-bit keys [N,E] (same candidate sets, capacity rule and
+// output layout as oracle_token_drop / oracle_expanded_drop; expanded = 0 ignores D).
+void oracle_drop_keyed(const uint32_t* keys, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C, int D,
+                       int expanded, const int32_t* token_group, uint64_t* keep_mask, int32_t* cand, int32_t* kept,
+                       int32_t* offsets, int32_t* slot_row) {
+  const int m = expanded ? E / D : 0;
+  const int slots = k + m;
+  const int W = (E + 63) / 64;
+  struct KC { uint32_t key; int32_t t; int32_t slot; };
+  std::vector<std::vector<KC>> cands(E);
+  std::vector<char> in_topk(E);
+  for (int64_t t = 0; t < N; ++t) {
+    std::fill(in_topk.begin(), in_topk.end(), 0);
+    for (int j = 0; j < k; ++j) {
+      const int e = topk_idx[t * k + j];
+      in_topk[e] = 1;
+      cands[e].push_back(KC{keys[t * E + e], (int32_t)t, j});
+    }
+    if (expanded) {
+      const int64_t g = home_group(t, N, D, token_group);
+      for (int i = 0; i < m; ++i) {
+        const int e = (int)g * m + i;
+        if (!in_topk[e]) cands[e].push_back(KC{keys[t * E + e], (int32_t)t, k + i});
+      }
+    }
+  }
+  for (int64_t i = 0; i < N * W; ++i) keep_mask[i] = 0;
+  for (int64_t i = 0; i < N * slots; ++i) slot_row[i] = -1;
+  offsets[0] = 0;
+  for (int e = 0; e < E; ++e) {
+    cand[e] = (int32_t)cands[e].size();
+    std::vector<KC> order(cands[e]);
+    std::stable_sort(order.begin(), order.end(), [](const KC& a, const KC& b) { return a.key > b.key; });
+    const int64_t keep_n = std::min<int64_t>((int64_t)order.size(), C);
+    std::vector<char> is_kept(N > 0 ? N : 1, 0);
+    for (int64_t i = 0; i < keep_n; ++i) is_kept[order[i].t] = 1;
+    kept[e] = (int32_t)keep_n;
+    int32_t row = offsets[e];
+    for (const KC& x : cands[e])
+      if (is_kept[x.t]) {
+        keep_mask[(int64_t)x.t * W + (e >> 6)] |= (uint64_t)1 << (e & 63);
+        slot_row[(int64_t)x.t * slots + x.slot] = row++;
+      }
+    offsets[e + 1] = row;
+  }
+}
+
 // Device-level capacity ("Advanced Variant: Device-Level Capacity-Aware Inference"): the constraint
 // is on the aggregated load of a device, N_1 + ... + N_{n_l} <= C_dev, not on each expert.  The
 // candidates of device g are all (token, expert) pairs with the expert on g (top-k pairs, plus

@@ -19,7 +19,7 @@ _SRC = os.path.join(_HERE, "capmoe_oracle.cpp")
 _LIB = os.path.join(_HERE, "libcapmoe_oracle.so")
 _lib = None
 
-__all__ = ["build", "capacity", "device_capacity", "device_drop", "router_logits", "softmax", "topk", "token_drop",
+__all__ = ["build", "capacity", "device_capacity", "device_drop", "drop_keys", "drop_keyed", "METRICS", "router_logits", "softmax", "topk", "token_drop",
            "expanded_drop",
            "permute", "expert_ffn", "combine", "layer_tokens", "stats", "layer_forward", "num_threads"]
 
@@ -135,6 +135,41 @@ def expanded_drop(scores: np.ndarray, topk_idx: np.ndarray, C: int, D: int,
     tg = None if token_group is None else np.ascontiguousarray(token_group, np.int32)
     _load().oracle_expanded_drop(_p(scores), _p(topk_idx), _i64(N), int(E), int(k), _i64(C), int(D),
                                  _p(tg), _p(keep), _p(cand), _p(kept), _p(off), _p(slot_row))
+    return dict(keep_mask=keep, cand=cand, kept=kept, offsets=off, slot_row=slot_row)
+
+
+METRICS = {"score": 0, "order": 1, "reverse_order": 2, "random": 3}
+
+
+def drop_keys(metric: str, seed: int, scores: np.ndarray, idx: Optional[np.ndarray], E: int) -> np.ndarray:
+    """32-bit drop keys for every entry of scores [N,cols] (idx [N,cols] expert ids, or None for a
+    dense [N,E] matrix)."""
+    scores = np.ascontiguousarray(scores, np.float32)
+    N, cols = scores.shape
+    ix = None if idx is None else np.ascontiguousarray(idx, np.int32)
+    out = np.empty((N, cols), np.uint32)
+    _load().oracle_drop_keys(METRICS[metric], ctypes.c_uint64(seed), _p(scores), _p(ix), _i64(N), int(cols), int(E),
+                             _p(out))
+    return out
+
+
+def drop_keyed(keys: np.ndarray, topk_idx: np.ndarray, C: int, D: int = 1, expanded: bool = False,
+               token_group: Optional[np.ndarray] = None):
+    """Token Drop (expanded=False) or Expanded Drop on a dense [N,E] matrix of 32-bit keys."""
+    keys = np.ascontiguousarray(keys, np.uint32)
+    topk_idx = np.ascontiguousarray(topk_idx, np.int32)
+    N, E = keys.shape
+    k = topk_idx.shape[1]
+    m = E // D if expanded else 0
+    W = (E + 63) // 64
+    keep = np.empty((N, W), np.uint64)
+    cand = np.empty((E,), np.int32)
+    kept = np.empty((E,), np.int32)
+    off = np.empty((E + 1,), np.int32)
+    slot_row = np.empty((N, k + m), np.int32)
+    tg = None if token_group is None else np.ascontiguousarray(token_group, np.int32)
+    _load().oracle_drop_keyed(_p(keys), _p(topk_idx), _i64(N), int(E), int(k), _i64(C), int(D), int(bool(expanded)),
+                              _p(tg), _p(keep), _p(cand), _p(kept), _p(off), _p(slot_row))
     return dict(keep_mask=keep, cand=cand, kept=kept, offsets=off, slot_row=slot_row)
 
 
