@@ -139,6 +139,25 @@ int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t N
                          int32_t* cand, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row,
                          void* ws, size_t ws_bytes, void* stream);
 
+/* ---------------------------------------------------------------- drop metrics
+ * The Token Drop paragraph names four ways to rank the tokens an overloaded expert received:
+ * Score (the gating score, the default), Order (later tokens are discarded once earlier ones
+ * filled the capacity), Reverse Order (earlier tokens are removed) and Random (every token has
+ * the same chance).  capmoe_drop_keys turns a metric into one 32-bit key per entry; the drop
+ * stages compare their score input by bit pattern (larger = kept first, equal = lower token
+ * index first), so the key array, passed where capmoe_token_drop expects topk_score [N,k] or
+ * capmoe_expanded_drop / capmoe_device_drop expect scores [N,E], selects by that metric.  The
+ * gate weights of the kept rows still come from the real scores (stage 4).
+ *   scores [N,cols] fp32 (read for CAPMOE_METRIC_SCORE only), idx [N,cols] expert ids or NULL when
+ *   cols == E and column c is expert c; keys [N,cols] uint32 out.
+ *   Random keys are the high word of a 64-bit mix of (seed, t*E + e): a pure function of the
+ *   seed and the (token, expert) position. */
+typedef enum {
+  CAPMOE_METRIC_SCORE = 0, CAPMOE_METRIC_ORDER = 1, CAPMOE_METRIC_REVERSE_ORDER = 2, CAPMOE_METRIC_RANDOM = 3
+} capmoe_metric;
+int capmoe_drop_keys(int metric, uint64_t seed, const float* scores, const int32_t* idx, int64_t N, int cols,
+                     int E, uint32_t* keys, void* stream);
+
 /* ---------------------------------------------------------------- device-level capacity
  * The paper's "Advanced Variant: Device-Level Capacity-Aware Inference": the bound applies to the
  * aggregated load of a device, N_1 + ... + N_{n_l} <= C_dev = n_l * gamma * N_bar, not to each

@@ -26,7 +26,7 @@ MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2, "device_token_drop": 
 EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_drop_workspace_bytes", "capmoe_status_str",
            "capmoe_last_cuda_error", "capmoe_launch_count", "capmoe_ffn_uses_tensor_cores", "capmoe_route",
            "capmoe_token_drop", "capmoe_token_drop_static", "capmoe_expanded_drop", "capmoe_device_capacity",
-           "capmoe_device_drop", "capmoe_permute", "capmoe_grouped_ffn",
+           "capmoe_device_drop", "capmoe_drop_keys", "capmoe_permute", "capmoe_grouped_ffn",
            "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe"]
 
 
@@ -224,6 +224,20 @@ def expanded_drop(scores, topk_idx, C: int, D: int, token_group=None, ws=None, s
                                       _ptr(out["kept"]), _ptr(out["offsets"]), _ptr(out["slot_row"]), _ptr(ws),
                                       ctypes.c_size_t(ws.numel()), _stream(stream)), "capmoe_expanded_drop")
     return out
+
+
+METRICS = {"score": 0, "order": 1, "reverse_order": 2, "random": 3}
+
+
+def drop_keys(metric: str, seed: int, scores, idx, E: int, stream=None):
+    """32-bit drop keys for every entry of scores [N,cols] (idx [N,cols] expert ids, or None for a
+    dense [N,E] matrix).  Returned as a float32-typed tensor holding the key bit patterns, so it
+    can be passed straight to token_drop / expanded_drop / device_drop in place of the scores."""
+    N, cols = scores.shape
+    keys = torch.empty((N, cols), device=scores.device, dtype=torch.float32)
+    _check(lib().capmoe_drop_keys(METRICS[metric], ctypes.c_uint64(seed), _ptr(scores), _ptr(idx), _i64(N),
+                                  int(cols), int(E), _ptr(keys), _stream(stream)), "capmoe_drop_keys")
+    return keys
 
 
 def device_capacity(N: int, E: int, k: int, D: int, gamma: float, round_mode: str = "ceil") -> int:

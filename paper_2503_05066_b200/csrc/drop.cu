@@ -464,3 +464,50 @@ extern "C" int capmoe_token_drop_static(const float* topk_score, const int32_t* 
   return run_drop<false>(topk_score, topk_idx, N, E, k, C, 1, nullptr, keep_mask, nullptr, kept,
                          expert_offsets, slot_row, ws, STATIC_WS_BYTES, as_stream(stream));
 }
+
+// ---------------------------------------------------------------------------------------------
+// Drop metrics: 32-bit keys for the select (the paper's "Score", "Order", "Reverse Order",
+// "Random").  The drop entry points compare their score input by bit pattern, so a key array
+// passed in place of the scores selects by that metric.
+namespace capmoe {
+namespace {
+
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__global__ void __launch_bounds__(256)
+k_drop_keys(int metric, unsigned long long seed, const float* __restrict__ scores, const int32_t* __restrict__ idx,
+            int64_t total, int cols, int E, uint32_t* __restrict__ keys) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= total) return;
+  const int64_t t = i / cols;
+  const int c = (int)(i - t * cols);
+  const int e = idx ? idx[i] : c;
+  uint32_t key;
+  if (metric == CAPMOE_METRIC_SCORE) key = __float_as_uint(scores[i]);
+  else if (metric == CAPMOE_METRIC_ORDER) key = 0x3f800000u;              // all equal: earlier tokens first
+  else if (metric == CAPMOE_METRIC_REVERSE_ORDER) key = (uint32_t)t;      // later tokens first
+  else
+    key = (uint32_t)(mix64(seed + 0x9E3779B97F4A7C15ull *
+                                      ((unsigned long long)t * (unsigned)E + (unsigned)e + 1ull)) >> 32);
+  keys[i] = key;
+}
+
+}  // namespace
+}  // namespace capmoe
+
+extern "C" int capmoe_drop_keys(int metric, uint64_t seed, const float* scores, const int32_t* idx, int64_t N,
+                                int cols, int E, uint32_t* keys, void* stream) {
+  if (metric < CAPMOE_METRIC_SCORE || metric > CAPMOE_METRIC_RANDOM) return CAPMOE_EINVAL;
+  if (N < 0 || cols < 1 || E < 1 || (!idx && cols != E)) return CAPMOE_EINVAL;
+  if (N == 0) return CAPMOE_OK;
+  if (!keys || (metric == CAPMOE_METRIC_SCORE && !scores)) return CAPMOE_EINVAL;
+  const int64_t total = N * cols;
+  if (total >= ((int64_t)1 << 38)) return CAPMOE_EUNSUPPORTED;
+  k_drop_keys<<<(unsigned)ceil_div(total, 256), 256, 0, as_stream(stream)>>>(
+      metric, (unsigned long long)seed, scores, idx, total, cols, E, keys);
+  return check_launch();
+}
