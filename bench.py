@@ -331,6 +331,47 @@ def main():
                       "frac_of_measured_copy": v / (stage_ms[k] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
                   for k, v in hbm.items() if stage_ms[k] > 0}
 
+    # Kernel-only bandwidth of the three HBM-bound stages: the same launches back to back, rotating
+    # over input copies that together exceed L2 (126 MB), so that no launch finds its input cached
+    # and no event record sits between launches.
+    hbm_kernels = {}
+    if rank == 0:
+        reps = 24
+
+        def timed(fn):
+            for i in range(4):
+                fn(i)
+            torch.cuda.synchronize()
+            e0.record()
+            for i in range(reps):
+                fn(i)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        t = layer.t
+        ncopy = max(2, int(200e6 // (cfg.N * cfg.d * elt)) + 1)
+        xs = [g["x"]] + [g["x"].clone() for _ in range(ncopy - 1)]
+        r_out = capmoe.route(g["x"], g["w_router"], g["bias"], cfg.k)
+        ms = timed(lambda i: capmoe.route(xs[i % ncopy], g["w_router"], g["bias"], cfg.k, out=r_out))
+        hbm_kernels["route"] = ms
+        A_rows = t["x_perm"].shape[0]
+        pcopy = max(2, int(200e6 // (A_rows * cfg.d * elt)) + 1)
+        p_outs = [dict(x_perm=torch.empty_like(t["x_perm"]), perm_token=torch.empty_like(t["perm_token"]),
+                       perm_weight=torch.empty_like(t["perm_weight"])) for _ in range(pcopy)]
+        Dp = cfg.D if layer.slots > cfg.k else 0
+        ms = timed(lambda i: capmoe.permute(xs[i % ncopy], t["scores"], t["topk_idx"], t["slot_row"], A_rows, Dp,
+                                            out=p_outs[i % pcopy]))
+        hbm_kernels["permute"] = ms
+        ys = [t["y_perm"]] + [t["y_perm"].clone() for _ in range(pcopy - 1)]
+        y_outs = [torch.empty_like(t["y"]) for _ in range(2)]
+        ms = timed(lambda i: capmoe.combine(ys[i % pcopy], t["slot_row"], t["perm_weight"], y=y_outs[i % 2]))
+        hbm_kernels["combine"] = ms
+        hbm_kernels = {k: {"ms": v, "bytes": hbm[k], "GB/s": hbm[k] / (v * 1e-3) / 1e9,
+                           "frac_of_measured_copy": hbm[k] / (v * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                       for k, v in hbm_kernels.items()}
+        del xs, p_outs, ys, y_outs
+
     # ------------------------------------------------------------------ e2e through the host-buffer entry point
     # Every step copies its activations in from pinned host memory and its output back out, inside
     # the timed region.  Two layer instances (own activation buffers, shared weights) alternate on
@@ -419,7 +460,7 @@ def main():
             "dtype": cfg.dtype, "data": "synthetic", "config": _config_dict(cfg, args),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu,
-            "stages_ms": stage_ms, "hbm_stages": hbm_stages,
+            "stages_ms": stage_ms, "hbm_stages": hbm_stages, "hbm_kernels": hbm_kernels,
             "workload_stats": {"A": A, "C": int(layer_C(cfg, args, capmoe)), "max_load_over_mean": max(load) / nbar,
                                "kept_fraction_of_Nk": A / (cfg.N * cfg.k), "kept_per_expert": kept,
                                "load_per_expert": load},

@@ -141,8 +141,8 @@ def ffn_uses_tensor_cores(d: int, F: int, dtype) -> bool:
 
 
 # ----------------------------------------------------------------------------- stages
-def route(x, w_router, bias, k: int, logits_in=None, stream=None):
-    """-> dict(logits, scores, topk_idx, topk_score, load)"""
+def route(x, w_router, bias, k: int, logits_in=None, out=None, stream=None):
+    """-> dict(logits, scores, topk_idx, topk_score, load); `out` may hand in those buffers to be reused."""
     if logits_in is not None:
         N, E = logits_in.shape
         d, dev, dt = 0, logits_in.device, F32
@@ -152,9 +152,10 @@ def route(x, w_router, bias, k: int, logits_in=None, stream=None):
         dev, dt = x.device, _dt(x)
     f32 = dict(device=dev, dtype=torch.float32)
     i32 = dict(device=dev, dtype=torch.int32)
-    out = dict(logits=torch.empty((N, E), **f32), scores=torch.empty((N, E), **f32),
-               topk_idx=torch.empty((N, k), **i32), topk_score=torch.empty((N, k), **f32),
-               load=torch.empty((E,), **i32))
+    if out is None:
+        out = dict(logits=torch.empty((N, E), **f32), scores=torch.empty((N, E), **f32),
+                   topk_idx=torch.empty((N, k), **i32), topk_score=torch.empty((N, k), **f32),
+                   load=torch.empty((E,), **i32))
     _check(lib().capmoe_route(_ptr(x), _ptr(w_router), _ptr(bias), _ptr(logits_in), _i64(N), int(d), int(E),
                               int(k), dt, _ptr(out["logits"]), _ptr(out["scores"]), _ptr(out["topk_idx"]),
                               _ptr(out["topk_score"]), _ptr(out["load"]), _stream(stream)), "capmoe_route")
@@ -273,16 +274,18 @@ def device_drop(scores, topk_idx, C_dev: int, D: int, expanded: bool, token_grou
     return out
 
 
-def permute(x, scores, topk_idx, slot_row, A_max: int, D: int = 0, token_group=None, stream=None):
-    """-> dict(x_perm [A_max,d], perm_token [A_max], perm_weight [A_max]); rows >= A are left unwritten"""
+def permute(x, scores, topk_idx, slot_row, A_max: int, D: int = 0, token_group=None, out=None, stream=None):
+    """-> dict(x_perm [A_max,d], perm_token [A_max], perm_weight [A_max]); rows >= A are left unwritten.
+    `out` may hand in those three buffers to be reused."""
     N, d = x.shape
     E = scores.shape[1]
     k = topk_idx.shape[1]
     slots = slot_row.shape[1]
     dev = x.device
-    out = dict(x_perm=torch.zeros((A_max, d), device=dev, dtype=x.dtype),
-               perm_token=torch.full((A_max,), -1, device=dev, dtype=torch.int32),
-               perm_weight=torch.zeros((A_max,), device=dev, dtype=torch.float32))
+    if out is None:
+        out = dict(x_perm=torch.zeros((A_max, d), device=dev, dtype=x.dtype),
+                   perm_token=torch.full((A_max,), -1, device=dev, dtype=torch.int32),
+                   perm_weight=torch.zeros((A_max,), device=dev, dtype=torch.float32))
     _check(lib().capmoe_permute(_ptr(x), _i64(N), int(d), int(E), int(k), int(slots), int(D), _dt(x),
                                 _ptr(scores), _ptr(topk_idx), _ptr(token_group), _ptr(slot_row),
                                 _ptr(out["x_perm"]), _ptr(out["perm_token"]), _ptr(out["perm_weight"]),

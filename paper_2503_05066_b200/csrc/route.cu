@@ -238,7 +238,7 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, q = lane & 3;
   const int64_t t0 = (int64_t)blockIdx.x * ROWS;
-  const int kw = d / RM_WARPS;                         // columns per warp (multiple of 32)
+  const int kw = d / RM_WARPS;                         // columns per warp (multiple of 64)
   const int kbeg = warp * kw;
 
   float acc[MT][NT][4];
@@ -254,32 +254,39 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
 #pragma unroll
   for (int i = 0; i < MT; ++i) {
     const int64_t ta = t0 + i * 16 + g, tb = ta + 8;
-    xrow[i][0] = ta < N ? reinterpret_cast<const uint4*>(x + ta * d + kbeg) + q : nullptr;
-    xrow[i][1] = tb < N ? reinterpret_cast<const uint4*>(x + tb * d + kbeg) + q : nullptr;
+    xrow[i][0] = ta < N ? reinterpret_cast<const uint4*>(x + ta * d + kbeg) + 2 * q : nullptr;
+    xrow[i][1] = tb < N ? reinterpret_cast<const uint4*>(x + tb * d + kbeg) + 2 * q : nullptr;
   }
   const uint4* wrow[NT];
 #pragma unroll
   for (int j = 0; j < NT; ++j) {
     const int e = j * 8 + g;
-    wrow[j] = e < E ? reinterpret_cast<const uint4*>(w + (int64_t)e * d + kbeg) + q : nullptr;
+    wrow[j] = e < E ? reinterpret_cast<const uint4*>(w + (int64_t)e * d + kbeg) + 2 * q : nullptr;
   }
 
-  const int steps = kw / 32;                           // 32 columns (4 lanes x 8) per step
+  // 64 columns per step: each lane takes 32 contiguous bytes (two 16-byte loads) of its two rows, so
+  // the four lanes of a row cover one full 128-byte line per step
+  const int steps = kw / 64;
 #pragma unroll 4
   for (int s = 0; s < steps; ++s) {
-    uint4 xa[MT], xb[MT];
+    uint4 xa[MT][2], xb[MT][2];
 #pragma unroll
-    for (int i = 0; i < MT; ++i) {
-      xa[i] = xrow[i][0] ? __ldcs(xrow[i][0] + s * 4) : zero;       // streamed once: evict first
-      xb[i] = xrow[i][1] ? __ldcs(xrow[i][1] + s * 4) : zero;
-    }
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        xa[i][h] = xrow[i][0] ? __ldcs(xrow[i][0] + s * 8 + h) : zero;   // streamed once: evict first
+        xb[i][h] = xrow[i][1] ? __ldcs(xrow[i][1] + s * 8 + h) : zero;
+      }
 #pragma unroll
     for (int j = 0; j < NT; ++j) {
-      const uint4 wv = wrow[j] ? __ldg(wrow[j] + s * 4) : zero;
 #pragma unroll
-      for (int i = 0; i < MT; ++i) {
-        mma_bf16_16816(acc[i][j], xa[i].x, xb[i].x, xa[i].y, xb[i].y, wv.x, wv.y);
-        mma_bf16_16816(acc[i][j], xa[i].z, xb[i].z, xa[i].w, xb[i].w, wv.z, wv.w);
+      for (int h = 0; h < 2; ++h) {
+        const uint4 wv = wrow[j] ? __ldg(wrow[j] + s * 8 + h) : zero;
+#pragma unroll
+        for (int i = 0; i < MT; ++i) {
+          mma_bf16_16816(acc[i][j], xa[i][h].x, xb[i][h].x, xa[i][h].y, xb[i][h].y, wv.x, wv.y);
+          mma_bf16_16816(acc[i][j], xa[i][h].z, xb[i][h].z, xa[i][h].w, xb[i][h].w, wv.z, wv.w);
+        }
       }
     }
   }
@@ -323,7 +330,7 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
   }
 }
 
-bool router_mma_ok(int d, int E) { return d % (RM_WARPS * 32) == 0 && E <= 128; }
+bool router_mma_ok(int d, int E) { return d % (RM_WARPS * 64) == 0 && E <= 128; }
 
 struct RouteOut { int k; float* scores; int32_t* topk_idx; float* topk_score; int32_t* load; };
 
