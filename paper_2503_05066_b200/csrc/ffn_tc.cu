@@ -413,6 +413,260 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   if (tid == 0 && *abort_flag && dev_status) atomicExch(dev_status, (int)CAPMOE_ETIMEOUT);
 }
 
+// ---------------------------------------------------------------- CTA-pair variant (cta_group::2)
+// Two CTAs of a cluster work on one 256 x 256 tile: each loads its own 128 rows of A and half of
+// the B rows (for gate/up: CTA 0 the W_g tile, CTA 1 the W_u tile), the even CTA issues
+// tcgen05.mma.cta_group::2 (M = 256) for both, and each CTA's tensor memory receives the 128
+// accumulator rows it loaded A for.  Per k-block a CTA now fills 32 KB of shared memory instead of
+// 48 KB for the same MMA work, which cuts L2->SM traffic by a third, and the ring is six deep.
+// No multicast loads are used; tcgen05.commit multicasts the "stage free" and "accumulator
+// ready" signals to both CTAs.
+constexpr int STAGES2 = 6;
+constexpr int HALF_B_BYTES = 128 * BK * 2;                 // 16 KB
+constexpr int STAGE2_BYTES = A_BYTES + HALF_B_BYTES;       // 32 KB per CTA
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;                // shared::cluster address of the even CTA's copy
+static_assert(STAGES2 * STAGE2_BYTES == STAGES * STAGE_BYTES, "both variants share one smem layout");
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                             uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void umma2(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                      uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives on the barrier at this offset in both CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+          const __grid_constant__ CUtensorMap map_b1, const int32_t* __restrict__ expert_offsets, int E,
+          int K, int Nout, __nv_bfloat16* __restrict__ out, int D_straggler, int32_t* __restrict__ dev_status) {
+  constexpr bool SWIGLU = MODE == MODE_GATE_UP;
+  constexpr int N_TILE = SWIGLU ? 128 : 256;
+  constexpr int BM2 = 2 * BM;                                   // rows of a pair's tile
+  const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BNB >> 3) << 17) |
+                         ((uint32_t)(BM2 >> 4) << 24);          // M = 256, N = 256
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + STAGES * STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* offs = reinterpret_cast<int*>(gen + STAGES * STAGE_BYTES + 512);
+  int* tile_start = offs + (MAX_E + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();                      // 0 = leader (issues the MMAs)
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(MAX_STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 + b); };
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 2 * EPI_WARPS * 32); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = tid; i <= E; i += TC_THREADS) offs[i] = expert_offsets[i];
+  __syncthreads();
+  if (tid == 0) {
+    const int n_blocks = (Nout + N_TILE - 1) / N_TILE;
+    int acc = 0;
+    for (int e = 0; e < E; ++e) {
+      tile_start[e] = acc;
+      acc += ((offs[e + 1] - offs[e] + BM2 - 1) / BM2) * n_blocks;
+    }
+    tile_start[E] = acc;
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();             // the peer's barriers are initialised and its tensor memory allocated
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  int tile_hi, stride, first;
+  if (D_straggler > 0) {
+    const int per = npairs / D_straggler;
+    const int g = pair / per;
+    if (g >= D_straggler) { tile_hi = 0; first = 0; stride = 1; }
+    else {
+      const int m = E / D_straggler;
+      tile_hi = tile_start[(g + 1) * m];
+      first = tile_start[g * m] + (pair - g * per); stride = per;
+    }
+  } else {
+    tile_hi = tile_start[E]; first = pair; stride = npairs;
+  }
+  const int num_kb = (K + BK - 1) / BK;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int cursor = 0, s = 0;
+      uint32_t ph = 0;
+      Tile t;
+      bool ok = true;
+      for (int tile = first; ok && tile < tile_hi; tile += stride) {
+        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
+        const int my_row0 = t.row0 + (int)rank * BM;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t lead_full = full_bar(s) & PEER_MASK;   // the leader's barrier counts both CTAs' bytes
+          if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
+          const uint32_t a_dst = tiles + (uint32_t)s * STAGE2_BYTES;
+          const uint32_t b_dst = a_dst + A_BYTES;
+          tma2_load_2d(a_dst, &map_a, kb * BK, my_row0, lead_full);
+          if (SWIGLU) tma2_load_3d(b_dst, rank == 0 ? &map_b0 : &map_b1, kb * BK, t.n0, t.e, lead_full);
+          else tma2_load_3d(b_dst, &map_b0, kb * BK, t.n0 + (int)rank * 128, t.e, lead_full);
+          if (++s == STAGES2) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      int cursor = 0, s = 0;
+      uint32_t it = 0, ph = 0;
+      const uint64_t adesc0 = umma_desc(tiles);
+      const uint64_t bdesc0 = umma_desc(tiles + A_BYTES);
+      const uint64_t stage_step = (uint64_t)(STAGE2_BYTES >> 4);
+      uint64_t stage_off = 0;
+      Tile t;
+      bool ok = true;
+      for (int tile = first; ok && tile < tile_hi; tile += stride, ++it) {
+        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
+        const uint32_t b = it & 1u, use = it >> 1;
+        if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + b * (uint32_t)BNB;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t adesc = adesc0 + stage_off, bdesc = bdesc0 + stage_off;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma2(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+          umma2_commit_both(empty_bar(s));              // both CTAs may refill this stage
+          stage_off += stage_step;
+          if (++s == STAGES2) { s = 0; ph ^= 1u; stage_off = 0; }
+        }
+        if (ok) umma2_commit_both(tfull_bar(b));        // both halves of the accumulator are complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
+    const int quarter = warp & 3;
+    const int row_in_half = quarter * 32 + lane;
+    const int half = (warp - 2) >> 2;
+    int cursor = 0;
+    uint32_t it = 0;
+    Tile t;
+    for (int tile = first; tile < tile_hi; tile += stride, ++it) {
+      if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
+      const uint32_t b = it & 1u, use = it >> 1;
+      bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
+      ready = __all_sync(0xffffffffu, ready);
+      if (!ready) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)BNB;
+      const int row_in_tile = (int)rank * BM + row_in_half;
+      const bool row_ok = row_in_tile < t.rows;
+      __nv_bfloat16* orow = out + (int64_t)(t.row0 + row_in_tile) * Nout + t.n0;
+#pragma unroll 1
+      for (int c = half * (N_TILE / 2); c < (half + 1) * (N_TILE / 2); c += 32) {
+        uint32_t g[32];
+        uint32_t packed[16];
+        if (SWIGLU) {
+          uint32_t u[32];
+          tmem_ld32(taddr + (uint32_t)c, g);
+          tmem_ld32(taddr + (uint32_t)(128 + c), u);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float g0 = __uint_as_float(g[2 * j]), g1 = __uint_as_float(g[2 * j + 1]);
+            const float u0 = __uint_as_float(u[2 * j]), u1 = __uint_as_float(u[2 * j + 1]);
+            const float h0 = __fdividef(g0, 1.0f + __expf(-g0)) * u0;
+            const float h1 = __fdividef(g1, 1.0f + __expf(-g1)) * u1;
+            packed[j] = pack_bf16(h0, h1);
+          }
+        } else {
+          tmem_ld32(taddr + (uint32_t)c, g);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            packed[j] = pack_bf16(__uint_as_float(g[2 * j]), __uint_as_float(g[2 * j + 1]));
+        }
+        if (row_ok) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (t.n0 + c + v * 8 + 8 <= Nout)
+              *reinterpret_cast<uint4*>(orow + c + v * 8) =
+                  make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive_cluster(tempty_bar(b) & PEER_MASK);   // the leader waits for both CTAs' epilogues
+    }
+  }
+
+  // ------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();             // no signal of the peer can still be on its way to this CTA
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+  if (tid == 0 && *abort_flag && dev_status) atomicExch(dev_status, (int)CAPMOE_ETIMEOUT);
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -490,6 +744,40 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
   err = cudaFuncSetAttribute(k_ffn_tc<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (err != cudaSuccess) return note_cuda(err);
   int grid = sm_count();
+  // CTA pairs (256-row tiles) when the expert segments are long enough that the extra tail
+  // padding does not matter, or are known multiples of 256 rows
+  const int64_t avg_rows = A_max / E;
+  if (grid >= 2 && (avg_rows >= 1024 || (avg_rows >= 256 && avg_rows % 256 == 0)) &&
+      (D_straggler == 0 || grid / 2 >= D_straggler)) {
+    alignas(64) CUtensorMap bd128;
+    if (!make_map(&bd128, w_down, (uint64_t)F, (uint64_t)d, (uint64_t)E, 128)) return note_cuda(cudaErrorInvalidValue);
+    int pairs = grid / 2;
+    if (D_straggler > 0) pairs = (pairs / D_straggler) * D_straggler;
+    err = cudaFuncSetAttribute(k_ffn_tc2<MODE_GATE_UP>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (err != cudaSuccess) return note_cuda(err);
+    err = cudaFuncSetAttribute(k_ffn_tc2<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (err != cudaSuccess) return note_cuda(err);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_GATE_UP>, a1, bg, bu, expert_offsets, E, d, F,
+                             (__nv_bfloat16*)h_ws, D_straggler, dev_status);
+    count_launch(1);
+    if (err != cudaSuccess) return note_cuda(err);
+    int rc2;
+    if (mid && (rc2 = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc2;
+    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_DOWN>, a2, bd128, bd128, expert_offsets, E, F, d,
+                             (__nv_bfloat16*)y_perm, D_straggler, dev_status);
+    count_launch(1);
+    return note_cuda(err);
+  }
   if (D_straggler > 0) {
     if (grid < D_straggler) return CAPMOE_EUNSUPPORTED;
     grid = (grid / D_straggler) * D_straggler;          // equal share of SMs per virtual device
