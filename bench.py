@@ -33,10 +33,11 @@ METRIC = "MoE-layer tokens/s at Mixtral shape"
 UNIT = "tokens/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMM launch, from single-pass ncu
-# captures (see profiles/k_ffn_tc_dram_traffic.md); key = (config, N, F, mode, gamma)
+# captures of the current kernel (profiles/launch_list_mixtral_expanded_drop.md,
+# profiles/k_ffn_tc2_olmoe_ncu_full.md); key = (config, N, F, mode, gamma)
 NCU_TRAFFIC_GATE_UP = {
-    ("mixtral", 8192, 14336, "expanded_drop", 1.0): 2270196736 + 462499072,
-    ("olmoe", 4096, 1024, "expanded_drop", 1.0): 673051392 + 56401664,
+    ("mixtral", 8192, 14336, "expanded_drop", 1.0): 5541300000 + 462400000,
+    ("olmoe", 4096, 1024, "expanded_drop", 1.0): 671821056 + 60885248,
 }
 
 
@@ -305,15 +306,15 @@ def main():
     use_tc = capmoe.ffn_uses_tensor_cores(cfg.d, cfg.F, g["x"].dtype)
     peak_tf = peaks["bf16_tflops_sustained"] if use_tc else None
     roofline = {
-        "kernel": "k_ffn_tc<SWIGLU> (gate/up grouped GEMM + SwiGLU, tcgen05)" if use_tc else "k_grouped_gemm (fp32 FMA)",
+        "kernel": "k_ffn_tc / k_ffn_tc2 <gate/up> (grouped GEMM + SwiGLU, tcgen05)" if use_tc else "k_grouped_gemm (fp32 FMA)",
         "bound": "tensor" if use_tc else "alu",
         "achieved": gemm1_flops / t1 / 1e12 if t1 > 0 else None, "peak": peak_tf, "unit": "TFLOP/s",
         "frac": (gemm1_flops / t1 / 1e12 / peak_tf) if (t1 > 0 and peak_tf) else None,
         "peak_source": peaks["source"] + " (sustained cuBLAS bf16: kernel timed inside a long step)",
         "peak_burst": peaks["bf16_tflops"],
         "flops_per_launch": gemm1_flops,
-        # DRAM bytes of one gate/up launch (ncu, dram__bytes_read.sum + dram__bytes_write.sum; summary in
-        # profiles/k_ffn_tc_dram_traffic.md), known for the workloads that were captured
+        # DRAM bytes of one gate/up launch (ncu, dram__bytes_read.sum + dram__bytes_write.sum), known for
+        # the workloads that were captured
         "traffic": NCU_TRAFFIC_GATE_UP.get((cfg.name, cfg.N, cfg.F, args.mode, args.gamma)),
         "algorithmic_bytes": (2 * cfg.E * cfg.F * cfg.d + A * cfg.d + A * cfg.F) * elt,
         "down_gemm": {"achieved": gemm2_flops / t2 / 1e12 if t2 > 0 else None,
