@@ -474,7 +474,8 @@ template <int MODE>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
           const __grid_constant__ CUtensorMap map_b1, const int32_t* __restrict__ expert_offsets, int E,
-          int K, int Nout, __nv_bfloat16* __restrict__ out, int D_straggler, int32_t* __restrict__ dev_status) {
+          int K, int Nout, __nv_bfloat16* __restrict__ out, int D_straggler, int32_t* __restrict__ dev_status,
+          int group /* consecutive tiles one pair takes before it strides on */) {
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
   constexpr int N_TILE = SWIGLU ? 128 : 256;
   constexpr int BM2 = 2 * BM;                                   // rows of a pair's tile
@@ -537,10 +538,10 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     else {
       const int m = E / D_straggler;
       tile_hi = tile_start[(g + 1) * m];
-      first = tile_start[g * m] + (pair - g * per); stride = per;
+      first = tile_start[g * m] + (pair - g * per) * group; stride = per * group;
     }
   } else {
-    tile_hi = tile_start[E]; first = pair; stride = npairs;
+    tile_hi = tile_start[E]; first = pair * group; stride = npairs * group;
   }
   const int num_kb = (K + BK - 1) / BK;
 
@@ -551,7 +552,9 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       uint32_t ph = 0;
       Tile t;
       bool ok = true;
-      for (int tile = first; ok && tile < tile_hi; tile += stride) {
+      for (int j = 0; ok; ++j) {
+        const int tile = first + (j / group) * stride + (j % group);
+        if (tile >= tile_hi) break;
         if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
         const int my_row0 = t.row0 + (int)rank * BM;
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -578,7 +581,9 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       uint64_t stage_off = 0;
       Tile t;
       bool ok = true;
-      for (int tile = first; ok && tile < tile_hi; tile += stride, ++it) {
+      for (int j = 0; ok; ++j, ++it) {
+        const int tile = first + (j / group) * stride + (j % group);
+        if (tile >= tile_hi) break;
         if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
         const uint32_t b = it & 1u, use = it >> 1;
         if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -606,7 +611,9 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     int cursor = 0;
     uint32_t it = 0;
     Tile t;
-    for (int tile = first; tile < tile_hi; tile += stride, ++it) {
+    for (int j = 0;; ++j, ++it) {
+      const int tile = first + (j / group) * stride + (j % group);
+      if (tile >= tile_hi) break;
       if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
       const uint32_t b = it & 1u, use = it >> 1;
       bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
@@ -757,6 +764,9 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     if (err != cudaSuccess) return note_cuda(err);
     err = cudaFuncSetAttribute(k_ffn_tc2<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (err != cudaSuccess) return note_cuda(err);
+    // Consecutive tiles one pair takes before striding on.  1 is best: the reuse of weight tiles
+    // comes from pairs that work on them at the same time (measured: 2, 4, 8 raise DRAM reads).
+    const int group1 = 1, group2 = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.blockDim = dim3(TC_THREADS);
@@ -768,13 +778,13 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_GATE_UP>, a1, bg, bu, expert_offsets, E, d, F,
-                             (__nv_bfloat16*)h_ws, D_straggler, dev_status);
+                             (__nv_bfloat16*)h_ws, D_straggler, dev_status, group1);
     count_launch(1);
     if (err != cudaSuccess) return note_cuda(err);
     int rc2;
     if (mid && (rc2 = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc2;
     err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_DOWN>, a2, bd128, bd128, expert_offsets, E, F, d,
-                             (__nv_bfloat16*)y_perm, D_straggler, dev_status);
+                             (__nv_bfloat16*)y_perm, D_straggler, dev_status, group2);
     count_launch(1);
     return note_cuda(err);
   }
