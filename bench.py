@@ -165,6 +165,49 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_table(args):
+    """Latency, load statistics and drop rate per (N, gamma, mode) point: device time per layer over
+    `steps` forwards after `warmup`, one JSON line per point."""
+    import torch
+    from paper_2503_05066_b200 import capmoe, synth
+    base = _pick_config(args)
+    Ns = synth.QWEN_SWEEP_N if (base.name == "qwen" and args.N is None) else (base.N,)
+    steps, warmup = max(3, min(args.steps, 30)), max(3, min(args.warmup, 5))
+    for N in Ns:
+        cfg = base.with_(N=N)
+        inp = synth.make_layer_inputs(cfg)
+        g = {k: getattr(inp, k).cuda() for k in ("x", "w_router", "bias", "w_gate", "w_up", "w_down")}
+        shared = None if inp.shared is None else tuple(s.cuda() for s in inp.shared)
+        nodrop_ms = {}
+        points = [("nodrop", None)] + [(m, gm) for gm in cfg.gammas
+                                       for m in ("token_drop", "expanded_drop", "device_token_drop",
+                                                 "device_expanded_drop")]
+        for mode, gamma in points:
+            for strag in ([False, True] if cfg.straggler else [False]):
+                lay = capmoe.MoELayer(g["x"], g["w_router"], g["bias"], g["w_gate"], g["w_up"], g["w_down"], cfg.k,
+                                      cfg.D, mode, gamma=1.0 if gamma is None else gamma, straggler=strag,
+                                      shared=shared)
+                ms = time_layer(lay, steps, warmup, torch)
+                if mode == "nodrop":
+                    nodrop_ms[strag] = ms
+                load = lay.t["load"].cpu().numpy()
+                kept = lay.t["kept"].cpu().numpy()
+                A = int(lay.t["expert_offsets"][-1].item())
+                nbar = N * cfg.k / cfg.E
+                m = cfg.E // cfg.D
+                print(json.dumps({
+                    "config": cfg.name, "N": N, "mode": mode, "gamma": gamma, "straggler_emulation": strag,
+                    "C": int(lay.C), "ms_per_layer": ms, "tokens_per_s": N / (ms * 1e-3),
+                    "speedup_vs_nodrop": nodrop_ms[strag] / ms,
+                    "max_load_over_mean": float(load.max() / nbar), "max_kept_over_mean": float(kept.max() / nbar),
+                    "max_device_kept_over_mean": float(kept.reshape(cfg.D, m).sum(1).max() / (nbar * m)),
+                    "A": A, "kept_over_Nk": A / (N * cfg.k),
+                    "dropped_fraction_of_topk": float(1.0 - min(A, N * cfg.k) / (N * cfg.k)) if "expanded" not in mode
+                    else None}), flush=True)
+                del lay
+        del g, inp
+
+
 def _pick_config(args):
     from paper_2503_05066_b200 import synth
     cfg = synth.CONFIGS[args.config]
@@ -214,6 +257,9 @@ def main():
     ap.add_argument("--gamma", type=float, default=1.0)
     ap.add_argument("--no-straggler", dest="straggler", action="store_false")
     ap.add_argument("--no-sweep", dest="sweep", action="store_false", help="skip the other modes")
+    ap.add_argument("--table", action="store_true",
+                    help="instead of the benchmark line, print one JSON line per (N, gamma, mode) point of the "
+                         "chosen config (for the Qwen-shape sweep: N in 128..65536, gamma in 0.5..2.0)")
     ap.add_argument("--no-cpu", dest="cpu", action="store_false", help="skip the CPU baseline")
     ap.add_argument("--impl", default="capmoe", choices=["capmoe", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=None,
@@ -229,6 +275,9 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.table:
+        run_table(args)
         return
 
     import torch
