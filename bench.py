@@ -188,6 +188,7 @@ def run_table(args):
                                       cfg.D, mode, gamma=1.0 if gamma is None else gamma, straggler=strag,
                                       shared=shared)
                 ms = time_layer(lay, steps, warmup, torch)
+                graph_ms = time_graph(lay, steps, torch)
                 if mode == "nodrop":
                     nodrop_ms[strag] = ms
                 load = lay.t["load"].cpu().numpy()
@@ -197,7 +198,7 @@ def run_table(args):
                 m = cfg.E // cfg.D
                 print(json.dumps({
                     "config": cfg.name, "N": N, "mode": mode, "gamma": gamma, "straggler_emulation": strag,
-                    "C": int(lay.C), "ms_per_layer": ms, "tokens_per_s": N / (ms * 1e-3),
+                    "C": int(lay.C), "ms_per_layer": ms, "ms_per_layer_graph": graph_ms, "tokens_per_s": N / (ms * 1e-3),
                     "speedup_vs_nodrop": nodrop_ms[strag] / ms,
                     "max_load_over_mean": float(load.max() / nbar), "max_kept_over_mean": float(kept.max() / nbar),
                     "max_device_kept_over_mean": float(kept.reshape(cfg.D, m).sum(1).max() / (nbar * m)),
@@ -241,6 +242,22 @@ def time_layer(layer, steps, warmup, torch, events=None):
     e1.record()
     torch.cuda.synchronize()
     layer.set_stage_events(None)
+    layer.check_device_status()
+    return e0.elapsed_time(e1) / steps
+
+
+def time_graph(layer, steps, torch):
+    """ms per step when the whole layer is replayed as one CUDA graph (no per-kernel launch cost on the host)."""
+    layer.capture_graph()
+    for _ in range(3):
+        layer.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        layer.replay()
+    e1.record()
+    torch.cuda.synchronize()
     layer.check_device_status()
     return e0.elapsed_time(e1) / steps
 

@@ -412,6 +412,23 @@ class MoELayer:
         _check(lib().capmoe_layer_forward(ctypes.byref(self.c), _stream(stream)), "capmoe_layer_forward")
         return self.t["y"]
 
+    def capture_graph(self):
+        """Records one forward into a CUDA graph (stage events off), so that `replay()` re-issues the
+        whole layer with one launch call.  Run `forward()` at least once before: kernels are loaded on
+        their first launch, which a capture does not allow.  Buffers and shapes are frozen."""
+        self.set_stage_events(None)
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream(device=self.t["x"].device)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.graph(graph, stream=side):
+            self.forward()
+        self._graph = graph
+        return graph
+
+    def replay(self):
+        self._graph.replay()
+        return self.t["y"]
+
     def forward_host(self, x_host: torch.Tensor, y_host: torch.Tensor, stream=None):
         assert x_host.is_pinned() and y_host.is_pinned() and x_host.is_contiguous() and y_host.is_contiguous()
         _check(lib().capmoe_layer_forward_host(ctypes.byref(self.c), ctypes.c_void_p(x_host.data_ptr()),

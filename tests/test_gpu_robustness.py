@@ -142,3 +142,23 @@ def test_status_codes_from_gpu_calls(cm):
     torch.cuda.synchronize()
     y = cm.grouped_ffn(pm["x_perm"], td["offsets"], g["w_gate"], g["w_up"], g["w_down"])
     assert torch.isfinite(y).all()
+
+
+@pytest.mark.parametrize("name,mode", [("tiny_f32", "token_drop"), ("olmoe", "expanded_drop"),
+                                       ("olmoe", "device_expanded_drop")])
+def test_cuda_graph_replay_matches_direct_launches(cm, name, mode):
+    cfg = synth.CONFIGS[name] if name == "tiny_f32" else synth.CONFIGS[name].with_(N=2048, d=512, F=256, E=16, k=4, D=4)
+    g = _inputs(cfg)
+    layer = cm.MoELayer(g["x"], g["w_router"], g["bias"], g["w_gate"], g["w_up"], g["w_down"], cfg.k, cfg.D, mode,
+                        gamma=1.0)
+    y0 = layer.forward().clone()
+    torch.cuda.synchronize()
+    keep0, rows0 = layer.t["keep_mask"].clone(), layer.t["slot_row"].clone()
+    layer.capture_graph()
+    for _ in range(3):
+        layer.t["y"].zero_()
+        layer.t["slot_row"].fill_(12345)
+        y = layer.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(y, y0) and torch.equal(layer.t["keep_mask"], keep0) and torch.equal(layer.t["slot_row"], rows0)
+    layer.check_device_status()
