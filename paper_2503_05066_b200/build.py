@@ -26,7 +26,8 @@ def _stale(obj: str, src: str) -> bool:
     if not os.path.exists(obj):
         return True
     newest = max(os.path.getmtime(p) for p in
-                 [src, os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "capmoe.h"), __file__])
+                 [src, os.path.join(ROOT, "include", "capmoe.h"), __file__] +
+                 [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh")])
     return os.path.getmtime(obj) < newest
 
 

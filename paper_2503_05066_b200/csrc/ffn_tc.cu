@@ -22,6 +22,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "softmax.cuh"
 
 namespace capmoe {
 namespace {
@@ -37,9 +38,13 @@ constexpr int B_BYTES = BNB * BK * 2;        // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_WARPS = 8;              // two warps per TMEM lane quarter, each takes half the columns
 constexpr int TC_THREADS = 64 + EPI_WARPS * 32;
+// Fused router: four warps per lane quarter, each thread takes a quarter of its token's columns.
+constexpr int RF_SUBS = 4;
+constexpr int RF_THREADS = 64 + 4 * RF_SUBS * 32;
+constexpr int RF_XCH_FLOATS = RF_SUBS * 128 + 128 + 4 * RF_SUBS * 128;   // max, sum relay, top-k candidates
 constexpr int MAX_E = 256;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/ +
-                           2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/;
+                           2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/ + RF_XCH_FLOATS * 4;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -95,6 +100,18 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// One lane of a converged warp, chosen by the hardware.  The compiler knows that the region this
+// guards is single-threaded and issues the asynchronous instructions from uniform registers; with
+// a plain `lane == 0` test each tcgen05.mma took ~90 cycles to issue, this way ~30.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -141,6 +158,38 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+      : "r"(taddr)
+      : "memory");
+}
+// Named barrier over `count` threads (whole warps), and the same with an AND over a predicate.
+__device__ __forceinline__ void group_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ bool group_all(int id, int count, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %3, 0;\n\t"
+      "bar.red.and.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(count), "r"((uint32_t)pred)
+      : "memory");
+  return r != 0;
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
@@ -171,17 +220,25 @@ __device__ __forceinline__ bool locate_tile(int tile, int& cursor, const int* ti
 // MODE_DOWN   : B tile = 256 rows of W_d, output columns n0..n0+255 of y_perm (bf16)
 // MODE_ROUTER : one row segment [0, single_rows), B tile = all n_mma (>= Nout) rows of W_r,
 //               output = fp32 logits [rows, Nout] + bias  (Eq. 1's gate)
-enum { MODE_GATE_UP = 0, MODE_DOWN = 1, MODE_ROUTER = 2 };
+// MODE_ROUTER_FUSED : MODE_ROUTER whose epilogue goes on, one thread per token with the token's
+//               Nout <= EPAD logits in registers, to softmax, top-k and the load histogram
+//               (Eq. 1, Eq. 3): the whole router stage in one launch
+enum { MODE_GATE_UP = 0, MODE_DOWN = 1, MODE_ROUTER = 2, MODE_ROUTER_FUSED = 3 };
 
-template <int MODE>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+// Outputs of the fused router epilogue (unused by the other modes).
+struct RouterFused { float* scores; int32_t* topk_idx; float* topk_score; int32_t* load; int k; };
+
+template <int MODE, int EPAD = 32>
+__global__ void __launch_bounds__(MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, 1)
 k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
          const __grid_constant__ CUtensorMap map_b1, const int32_t* __restrict__ expert_offsets, int E,
          int K /* reduction length */, int Nout /* output columns */, void* __restrict__ out_ptr,
          int D_straggler, int32_t* __restrict__ dev_status, int n_mma, int single_rows,
          const float* __restrict__ bias, int tile_rows /* rows per tile actually loaded (<= 128) */,
-         int n_stages, int stage_stride) {
+         int n_stages, int stage_stride, const RouterFused rf) {
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
+  constexpr bool ROUTER = MODE == MODE_ROUTER || MODE == MODE_ROUTER_FUSED;
+  constexpr bool FUSED = MODE == MODE_ROUTER_FUSED;
   constexpr int N_TILE = SWIGLU ? 128 : 256;
   __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(out_ptr);
   const uint32_t idesc = make_idesc(n_mma);
@@ -201,6 +258,9 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   int* offs = reinterpret_cast<int*>(gen + STAGES * STAGE_BYTES + 512);
   int* tile_start = offs + (MAX_E + 1);
   float* bias_s = reinterpret_cast<float*>(tile_start + (MAX_E + 1) + 2);   // [256], router mode only
+  int* hist = tile_start + 8;                          // [<= 128] load histogram, fused router only
+  float* xch = bias_s + 256;                           // [RF_XCH_FLOATS] exchange between a token's threads
+  const int nthreads = (int)blockDim.x;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -211,15 +271,17 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
 
   if (tid == 0) {
     for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), EPI_WARPS * 32); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), nthreads - 64); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (MODE == MODE_ROUTER) {
+  if (ROUTER) {
     if (tid == 0) { offs[0] = 0; offs[1] = single_rows; }
-    for (int i = tid; i < 256; i += TC_THREADS) bias_s[i] = (bias && i < Nout) ? bias[i] : 0.f;
+    for (int i = tid; i < 256; i += nthreads) bias_s[i] = (bias && i < Nout) ? bias[i] : 0.f;
+    if (FUSED)
+      for (int i = tid; i < EPAD; i += nthreads) hist[i] = 0;
   } else {
-    for (int i = tid; i <= E; i += TC_THREADS) offs[i] = expert_offsets[i];
+    for (int i = tid; i <= E; i += nthreads) offs[i] = expert_offsets[i];
   }
   __syncthreads();
   if (tid == 0) {
@@ -260,7 +322,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (elect_one()) {
       int cursor = 0;
       int s = 0;                                         // ring position and phase, advanced without division
       uint32_t ph = 0;
@@ -278,7 +340,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
             tma_load_3d(b_dst, &map_b0, kb * BK, t.n0, t.e, full_bar(s));
             tma_load_3d(b_dst + B_BYTES / 2, &map_b1, kb * BK, t.n0, t.e, full_bar(s));
           } else {
-            tma_load_3d(b_dst, &map_b0, kb * BK, MODE == MODE_ROUTER ? 0 : t.n0, t.e, full_bar(s));
+            tma_load_3d(b_dst, &map_b0, kb * BK, ROUTER ? 0 : t.n0, t.e, full_bar(s));
           }
           if (++s == n_stages) { s = 0; ph ^= 1u; }
         }
@@ -286,7 +348,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (elect_one()) {
       int cursor = 0;
       uint32_t it = 0;
       int s = 0;                                         // ring position and phase, advanced without division
@@ -334,10 +396,127 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       const uint32_t b = it & 1u, use = it >> 1;
       bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
       ready = __all_sync(0xffffffffu, ready);            // warp-uniform: tcgen05.ld below is .sync.aligned
+      if (FUSED) ready = group_all(1 + quarter, RF_SUBS * 32, ready);   // a token's threads stop together
       if (!ready) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)BNB;
       const bool row_ok = row_in_tile < t.rows;
+      if constexpr (FUSED) {
+        // RF_SUBS threads per token (same lane of the quarter's four warps), each with COLS of the
+        // token's columns in registers.  The accumulator goes back to the MMA issuer as soon as it
+        // has been read; what is not local to a thread passes through shared memory between the
+        // quarter's named-barrier phases.
+        constexpr int COLS = EPAD / RF_SUBS;
+        static_assert(COLS == 8 || COLS == 16, "fused router: 32 or 64 padded experts");
+        const int sub = (warp - 2) >> 2;
+        const int cbase = sub * COLS;
+        const int bar_id = 1 + quarter;
+        float* xmax = xch;                                                 // [RF_SUBS][128]
+        float* xsum = xch + RF_SUBS * 128;                                 // [128]
+        float* xb = xsum + 128;                                            // [2][RF_SUBS][128]
+        int* xi = reinterpret_cast<int*>(xb + 2 * RF_SUBS * 128);          // [2][RF_SUBS][128]
+        uint32_t g[COLS];
+        if constexpr (COLS == 16) tmem_ld16(taddr + (uint32_t)cbase, g);
+        else tmem_ld8(taddr + (uint32_t)cbase, g);
+        tmem_ld_wait();
+        tc_fence_before();
+        mbar_arrive(tempty_bar(b));
+        if (quarter * 32 >= t.rows) continue;            // no token of this tile in this quarter (all four warps agree)
+        float v[COLS];
+#pragma unroll
+        for (int i = 0; i < COLS; ++i)
+          v[i] = cbase + i < Nout ? __fadd_rn(__uint_as_float(g[i]), bias_s[cbase + i]) : -INFINITY;
+        const int64_t tok = (int64_t)t.row0 + row_in_tile;
+        float* lrow = reinterpret_cast<float*>(out_ptr) + tok * Nout + cbase;
+        float* srow = rf.scores + tok * Nout + cbase;
+        const bool vec = (Nout & 3) == 0;                // rows are 16-byte aligned: vector stores
+        if (row_ok) {
+          if (vec) {
+#pragma unroll
+            for (int i = 0; i < COLS; i += 4)
+              if (cbase + i < Nout) *reinterpret_cast<float4*>(lrow + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < COLS; ++i)
+              if (cbase + i < Nout) lrow[i] = v[i];
+          }
+        }
+        float mx = v[0];
+#pragma unroll
+        for (int i = 1; i < COLS; ++i) mx = v[i] > mx ? v[i] : mx;
+        xmax[sub * 128 + row_in_tile] = mx;
+        group_sync(bar_id, RF_SUBS * 32);
+#pragma unroll
+        for (int s2 = 0; s2 < RF_SUBS; ++s2) { const float o = xmax[s2 * 128 + row_in_tile]; mx = o > mx ? o : mx; }
+#pragma unroll
+        for (int i = 0; i < COLS; ++i) v[i] = exp_fixed(__fsub_rn(v[i], mx));     // padding: exp(-inf) = 0
+        // the E terms are added left to right: the partial sum is handed from thread to thread
+#pragma unroll
+        for (int s2 = 0; s2 < RF_SUBS; ++s2) {
+          if (sub == s2) {
+            float acc = s2 ? xsum[row_in_tile] : 0.f;
+#pragma unroll
+            for (int i = 0; i < COLS; ++i) acc = __fadd_rn(acc, v[i]);            // + 0 (padding) is exact
+            xsum[row_in_tile] = acc;
+          }
+          group_sync(bar_id, RF_SUBS * 32);
+        }
+        const float sum = xsum[row_in_tile];                                      // in [1, E]
+        const float rsum = __frcp_rn(sum);
+#pragma unroll
+        for (int i = 0; i < COLS; ++i) v[i] = cbase + i < Nout ? div_by(v[i], sum, rsum) : -1.f;   // padding never selected
+        if (row_ok) {
+          if (vec) {
+#pragma unroll
+            for (int i = 0; i < COLS; i += 4)
+              if (cbase + i < Nout) *reinterpret_cast<float4*>(srow + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < COLS; ++i)
+              if (cbase + i < Nout) srow[i] = v[i];
+          }
+        }
+        // top-k: k rounds; each thread offers the best of its columns (lower id on ties), the
+        // four offers are compared in id order with strict '>', the owner marks its column taken.
+#pragma unroll 1
+        for (int j = 0; j < rf.k; ++j) {
+          float cb0 = -1.f, cb1 = -1.f;
+          int ci0 = 0, ci1 = 0;
+#pragma unroll
+          for (int i = 0; i < COLS / 2; ++i) {
+            const bool g0 = v[i] > cb0, g1 = v[COLS / 2 + i] > cb1;
+            cb0 = g0 ? v[i] : cb0; ci0 = g0 ? i : ci0;
+            cb1 = g1 ? v[COLS / 2 + i] : cb1; ci1 = g1 ? COLS / 2 + i : ci1;
+          }
+          const bool g1 = cb1 > cb0;
+          const float mine = g1 ? cb1 : cb0;
+          const int mine_i = g1 ? ci1 : ci0;
+          const int slot = (j & 1) * RF_SUBS * 128 + row_in_tile;
+          xb[slot + sub * 128] = mine;
+          xi[slot + sub * 128] = cbase + mine_i;
+          group_sync(bar_id, RF_SUBS * 32);
+          float best = xb[slot];
+          int be = xi[slot];
+#pragma unroll
+          for (int s2 = 1; s2 < RF_SUBS; ++s2) {
+            const float ob = xb[slot + s2 * 128];
+            const int oe = xi[slot + s2 * 128];
+            const bool gt = ob > best;
+            best = gt ? ob : best;
+            be = gt ? oe : be;
+          }
+          if (be == cbase + mine_i) {                                              // this thread's offer won
+#pragma unroll
+            for (int i = 0; i < COLS; ++i) v[i] = i == mine_i ? -2.f : v[i];      // taken
+            if (row_ok) {
+              rf.topk_idx[tok * rf.k + j] = be;
+              rf.topk_score[tok * rf.k + j] = best;
+              atomicAdd(&hist[be], 1);
+            }
+          }
+        }
+        continue;
+      }
       if (MODE == MODE_ROUTER) {
         float* lrow = reinterpret_cast<float*>(out_ptr) + (int64_t)(t.row0 + row_in_tile) * Nout;
 #pragma unroll 1
@@ -411,6 +590,9 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
   if (tid == 0 && *abort_flag && dev_status) atomicExch(dev_status, (int)CAPMOE_ETIMEOUT);
+  if (FUSED)
+    for (int i = tid; i < Nout; i += nthreads)
+      if (hist[i]) atomicAdd(&rf.load[i], hist[i]);
 }
 
 // ---------------------------------------------------------------- CTA-pair variant (cta_group::2)
@@ -547,7 +729,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
+    if (elect_one()) {
       int cursor = 0, s = 0;
       uint32_t ph = 0;
       Tile t;
@@ -572,7 +754,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (lane == 0 && rank == 0) {
+    if (rank == 0 && elect_one()) {
       int cursor = 0, s = 0;
       uint32_t it = 0, ph = 0;
       const uint64_t adesc0 = umma_desc(tiles);
@@ -793,26 +975,47 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     grid = (grid / D_straggler) * D_straggler;          // equal share of SMs per virtual device
   }
   k_ffn_tc<MODE_GATE_UP><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a1, bg, bu, expert_offsets, E, d, F, h_ws,
-                                                              D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES);
+                                                              D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES,
+                                                              RouterFused{});
   int rc = check_launch();
   if (rc != CAPMOE_OK) return rc;
   if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
   k_ffn_tc<MODE_DOWN><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a2, bd, bd, expert_offsets, E, F, d, y_perm,
-                                                           D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES);
+                                                           D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES,
+                                                              RouterFused{});
   return check_launch();
 }
 
-// Router logits on the same pipeline: logits[N,E] = x[N,d] . w_router[E,d]^T + bias, fp32 out.
+// Router on the same pipeline: logits[N,E] = x[N,d] . w_router[E,d]^T + bias in fp32 and, when
+// `fused` points at the other outputs and E <= 64, softmax / top-k / load histogram in the epilogue.
 bool router_tc_supported(int64_t N, int d, int E) { return d % 64 == 0 && d >= 64 && E <= 256 && N < (1ll << 31); }
+bool router_tc_fusable(int E, int k) { return E <= 64 && k <= E; }
+
+template <int MODE, int EPAD>
+static int launch_router_tc(const CUtensorMap& ax, const CUtensorMap& bw, int grid, int d, int E, float* logits,
+                            int n_mma, int64_t N, const float* bias, int tile_rows, int n_stages, int stage_stride,
+                            const RouterFused& rf, cudaStream_t st) {
+  cudaError_t err = cudaFuncSetAttribute(k_ffn_tc<MODE, EPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         SMEM_BYTES);
+  if (err != cudaSuccess) return note_cuda(err);
+  k_ffn_tc<MODE, EPAD><<<grid, MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, SMEM_BYTES, st>>>(ax, bw, bw, nullptr, 1, d, E, logits, 0, nullptr, n_mma,
+                                                            (int)N, bias, tile_rows, n_stages, stage_stride, rf);
+  return check_launch();
+}
 
 int router_tc(const void* x, const void* w_router, const float* bias, int64_t N, int d, int E, float* logits,
+              float* scores, int32_t* topk_idx, float* topk_score, int32_t* load, int k, bool fused,
               cudaStream_t st) {
   const int n_mma = (E + 15) / 16 * 16;
-  // The stage reads X once and is bound by HBM, so what matters is bytes in flight: use row tiles
-  // small enough that every SM gets one (the MMA still spans 128 rows; the unused rows cost
-  // nothing that is on the critical path) and as deep a ring as shared memory allows.
+  // The stage reads X once and is bound by HBM, so what matters is bytes in flight and an even
+  // share of rows per SM: the tokens are cut into `rounds` tiles per SM of equal height (a
+  // multiple of 8 rows, the swizzle atom; at most 128, the MMA's M).  The MMA always spans 128
+  // rows; the rows past tile_rows cost nothing that is on the critical path.
   const int sms = sm_count();
-  const int tile_rows = N >= (int64_t)128 * sms ? 128 : (N >= (int64_t)64 * sms ? 64 : 32);
+  const int64_t rounds = ceil_div(N, (int64_t)128 * sms);
+  int tile_rows = (int)((ceil_div(N, (int64_t)sms * rounds) + 7) / 8 * 8);
+  if (tile_rows < 32) tile_rows = 32;
+  if (tile_rows > 128) tile_rows = 128;
   // A stage holds tile_rows rows of A followed by n_mma rows of B (both multiples of 1 KB).  The
   // MMA reads 128 A rows whatever tile_rows is, so the last stage must leave room for that.
   const int b_bytes = n_mma * BK * 2;
@@ -824,14 +1027,18 @@ int router_tc(const void* x, const void* w_router, const float* bias, int64_t N,
   if (!make_map(&ax, x, (uint64_t)d, (uint64_t)N, 0, (uint32_t)tile_rows) ||
       !make_map(&bw, w_router, (uint64_t)d, (uint64_t)E, 1, (uint32_t)n_mma))
     return note_cuda(cudaErrorInvalidValue);
-  cudaError_t err = cudaFuncSetAttribute(k_ffn_tc<MODE_ROUTER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         SMEM_BYTES);
-  if (err != cudaSuccess) return note_cuda(err);
   int grid = (int)ceil_div(N, tile_rows);
-  if (grid > sm_count()) grid = sm_count();
-  k_ffn_tc<MODE_ROUTER><<<grid, TC_THREADS, SMEM_BYTES, st>>>(ax, bw, bw, nullptr, 1, d, E, logits, 0, nullptr,
-                                                             n_mma, (int)N, bias, tile_rows, n_stages, stage_stride);
-  return check_launch();
+  if (grid > sms) grid = sms;
+  const RouterFused rf{scores, topk_idx, topk_score, load, k};
+  if (fused && router_tc_fusable(E, k)) {
+    if (E <= 32)
+      return launch_router_tc<MODE_ROUTER_FUSED, 32>(ax, bw, grid, d, E, logits, n_mma, N, bias, tile_rows, n_stages,
+                                                     stage_stride, rf, st);
+    return launch_router_tc<MODE_ROUTER_FUSED, 64>(ax, bw, grid, d, E, logits, n_mma, N, bias, tile_rows, n_stages,
+                                                   stage_stride, rf, st);
+  }
+  return launch_router_tc<MODE_ROUTER, 32>(ax, bw, grid, d, E, logits, n_mma, N, bias, tile_rows, n_stages,
+                                           stage_stride, rf, st);
 }
 
 }  // namespace capmoe

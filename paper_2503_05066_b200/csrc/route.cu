@@ -1,5 +1,6 @@
 // Stage 1: router GEMM, softmax, per-token top-k, expert load histogram (Eq. 1, Eq. 3).
 #include "common.cuh"
+#include "softmax.cuh"
 
 namespace capmoe {
 namespace {
@@ -56,26 +57,6 @@ k_router_gemm(const T* __restrict__ x, const T* __restrict__ w, const float* __r
       if (e < E) logits[t * E + e] = acc[i] + (bias ? bias[e] : 0.f);
     }
   }
-}
-
-// exp(x), x <= 0, as a fixed sequence of correctly rounded binary32 operations: range
-// reduction x = n ln2 + r with a two-word ln2, a degree-7 Taylor polynomial in Horner/fma
-// form, scaling by 2^n through the exponent field.  x < -80 gives exactly 0.
-__device__ __forceinline__ float exp_fixed(float x) {
-  if (x < -80.0f) return 0.0f;
-  const float n = rintf(__fmul_rn(x, __uint_as_float(0x3fb8aa3bu)));          // x * log2(e)
-  float r = __fmaf_rn(n, -__uint_as_float(0x3f317200u), x);                   // - n * ln2_hi
-  r = __fmaf_rn(n, -__uint_as_float(0x35bfbe8eu), r);                         // - n * ln2_lo
-  float q = __uint_as_float(0x39500d01u);                                     // 1/7!
-  q = __fmaf_rn(q, r, __uint_as_float(0x3ab60b61u));                          // 1/6!
-  q = __fmaf_rn(q, r, __uint_as_float(0x3c088889u));                          // 1/5!
-  q = __fmaf_rn(q, r, __uint_as_float(0x3d2aaaabu));                          // 1/4!
-  q = __fmaf_rn(q, r, __uint_as_float(0x3e2aaaabu));                          // 1/3!
-  q = __fmaf_rn(q, r, 0.5f);
-  q = __fmaf_rn(q, r, 1.0f);
-  q = __fmaf_rn(q, r, 1.0f);
-  const int ni = (int)n;
-  return __uint_as_float(__float_as_uint(q) + ((unsigned)ni << 23));
 }
 
 // Softmax, top-k and load histogram.  One warp per token, EPL = ceil(E/32) experts per lane: the max is a shuffle reduction (exact), every lane evaluates exp for its
@@ -213,7 +194,9 @@ constexpr int RM_WARPS = 8;
 }  // namespace
 // tcgen05 router GEMM (ffn_tc.cu): used when there are enough experts for the MMA work to matter
 bool router_tc_supported(int64_t N, int d, int E);
+bool router_tc_fusable(int E, int k);
 int router_tc(const void* x, const void* w_router, const float* bias, int64_t N, int d, int E, float* logits,
+              float* scores, int32_t* topk_idx, float* topk_score, int32_t* load, int k, bool fused,
               cudaStream_t st);
 namespace {
 
@@ -389,8 +372,10 @@ extern "C" int capmoe_route(const void* x, const void* w_router, const float* bi
     const RouteOut ro{k, scores, topk_idx, topk_score, load};
     if (dtype == CAPMOE_F32)
       rc = launch_gemm<float>((const float*)x, (const float*)w_router, bias, N, d, E, logits, st);
-    else if (E > 16 && router_tc_supported(N, d, E) && aligned16(x) && aligned16(w_router))
-      rc = router_tc(x, w_router, bias, N, d, E, logits, st);
+    else if (E > 16 && router_tc_supported(N, d, E) && aligned16(x) && aligned16(w_router)) {
+      fused = router_tc_fusable(E, k);
+      rc = router_tc(x, w_router, bias, N, d, E, logits, scores, topk_idx, topk_score, load, k, fused, st);
+    }
     else if (router_mma_ok(d, E) && aligned16(x) && aligned16(w_router))
       rc = launch_router_mma((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, N, d, E, logits, ro,
                              &fused, st);

@@ -92,6 +92,41 @@ def test_softmax_extreme_logits(cm):
     assert np.array_equal(out["scores"].cpu().numpy().view(np.uint32), oracle.softmax(lg).view(np.uint32))
 
 
+@pytest.mark.parametrize("N,d,E,k,scale", [
+    (333, 128, 17, 3, 1.0),        # 32 padded experts, scalar stores (E % 4 != 0)
+    (1000, 256, 32, 32, 1.0),      # k = E: every expert selected, in score order
+    (2500, 192, 33, 5, 1.0),       # 64 padded experts, E % 4 != 0
+    (20000, 64, 60, 4, 1.0),       # several row tiles per SM, ragged last tile
+    (19001, 128, 64, 8, 1.0),
+    (700, 128, 63, 6, 40.0),       # logit gaps far beyond 80: exp -> 0 and quotients down to 1e-35
+    (4100, 64, 24, 2, 12.0),
+])
+def test_route_one_launch_router(cm, N, d, E, k, scale):
+    """bf16 inputs with 16 < E <= 64: GEMM, softmax, top-k and histogram in one tensor-core launch.
+    Pairs of identical router rows give exact score ties, which must go to the lower expert id."""
+    g = torch.Generator().manual_seed(1000 + N + E)
+    x = torch.randn((N, d), generator=g).to(torch.bfloat16)
+    w = (torch.randn((E, d), generator=g) * (scale / d ** 0.5)).to(torch.bfloat16)
+    w[E // 2] = w[1]
+    w[E - 1] = w[0]
+    b = torch.zeros(E)
+    b[3] = 0.25
+    out = cm.route(dev(x), dev(w), dev(b), k)
+    torch.cuda.synchronize()
+    got_logits = out["logits"].cpu().numpy()
+    ref_logits = oracle.router_logits(to_np(x), to_np(w), b.numpy(), "bf16")
+    assert rel_err(got_logits.astype(np.float64), ref_logits.astype(np.float64)) <= ROUTER_TOL["bf16"]
+    assert np.array_equal(got_logits[:, E // 2], got_logits[:, 1])
+    s_ref = oracle.softmax(got_logits)
+    assert np.array_equal(out["scores"].cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    idx, val, load = oracle.topk(s_ref, k)
+    assert np.array_equal(out["topk_idx"].cpu().numpy(), idx)
+    assert np.array_equal(out["topk_score"].cpu().numpy().view(np.uint32), val.view(np.uint32))
+    assert np.array_equal(out["load"].cpu().numpy(), load)
+    if scale > 1.0:
+        assert (s_ref == 0).any() or s_ref[s_ref > 0].min() < 1e-20
+
+
 # ----------------------------------------------------------------------------- stages 2, 3
 DROP_CASES = [
     # N, E, k, D, gamma, quantum
