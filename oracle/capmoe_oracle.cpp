@@ -312,6 +312,99 @@ void oracle_drop_keyed(const uint32_t* keys, const int32_t* topk_idx, int64_t N,
   }
 }
 
+// Priority classes on top of a drop metric.  Two of the paper's variants rank candidates first by
+// a class and only then by the metric:
+//   * dropping by modality (multimodal section, "Image First" / "Text First"): every token of the
+//     protected modality outranks every token of the other one, whatever their scores;
+//   * Expanded Drop read as substitution only ("makes no change in the token assignments in experts
+//     that are overflowed by the top-k"): a token's top-k pairs outrank the pairs it only has
+//     through its home device, so the expansion can fill spare capacity but never displace.
+// Class P = 2 * [pair (t,e) is one of t's top-k, when topk_idx is given] + [token_class[t] & 1, when
+// token_class is given] goes into the two high bits of the key; the metric's key goes below it,
+// unchanged when exact != 0 (it must then be below 2^30, as the bit pattern of every score in [0,1]
+// is), else shifted right by two bits.  base/out [N,cols]; idx as in oracle_drop_keys.
+// Returns 1 if an exact key does not fit.
+int oracle_priority_keys(const uint32_t* base, const int32_t* idx, int64_t N, int cols, int E, int exact,
+                         const uint8_t* token_class, const int32_t* topk_idx, int k, uint32_t* out) {
+  (void)E;
+  for (int64_t t = 0; t < N; ++t)
+    for (int c = 0; c < cols; ++c) {
+      const int64_t i = t * cols + c;
+      const int e = idx ? idx[i] : c;
+      uint32_t P = 0;
+      if (topk_idx)
+        for (int j = 0; j < k; ++j)
+          if (topk_idx[t * k + j] == e) P = 2;
+      if (token_class) P += token_class[t] & 1u;
+      uint32_t body = base[i];
+      if (exact) {
+        if (body >= (1u << 30)) return 1;
+      } else {
+        body >>= 2;
+      }
+      out[i] = (P << 30) | body;
+    }
+  return 0;
+}
+
+// "w/ max" ablation of Expanded Drop (appendix "Maximum Number of Selected Experts"): after the
+// drop a token may sit on more than k experts; with the constraint it retains only its k_max
+// best by gating score (ties to the lower expert id).  One pass: capacity freed this way is not
+// handed to anyone else.  keep_mask [N, ceil(E/64)] is edited in place.
+void oracle_limit_experts(const float* scores, int64_t N, int E, int k_max, uint64_t* keep_mask) {
+  const int W = (E + 63) / 64;
+  std::vector<int> es;
+  for (int64_t t = 0; t < N; ++t) {
+    es.clear();
+    for (int e = 0; e < E; ++e)
+      if ((keep_mask[t * W + (e >> 6)] >> (e & 63)) & 1u) es.push_back(e);
+    if ((int)es.size() <= k_max) continue;
+    std::stable_sort(es.begin(), es.end(), [&](int a, int b) { return scores[t * E + a] > scores[t * E + b]; });
+    for (size_t i = (size_t)k_max; i < es.size(); ++i)
+      keep_mask[t * W + (es[i] >> 6)] &= ~((uint64_t)1 << (es[i] & 63));
+  }
+}
+
+// Counts, offsets and rows of a given keep mask, in the layout the drop stages produce: segment e
+// holds the tokens with bit e set in ascending token order; slot_row [N,slots] maps a token's
+// slots (top-k order, then the m = E/D home-device experts when slots = k + m) to rows, -1 where
+// the bit is clear.  A set bit whose expert is none of the token's slots is an error (returns 1).
+int oracle_rows_from_mask(const uint64_t* keep_mask, const int32_t* topk_idx, int64_t N, int E, int k, int slots,
+                          int D, const int32_t* token_group, int32_t* kept, int32_t* offsets, int32_t* slot_row) {
+  const int W = (E + 63) / 64;
+  const int m = slots > k ? E / D : 0;
+  std::vector<int32_t> next(E);
+  for (int e = 0; e < E; ++e) kept[e] = 0;
+  for (int64_t t = 0; t < N; ++t)
+    for (int e = 0; e < E; ++e)
+      if ((keep_mask[t * W + (e >> 6)] >> (e & 63)) & 1u) ++kept[e];
+  offsets[0] = 0;
+  for (int e = 0; e < E; ++e) { offsets[e + 1] = offsets[e] + kept[e]; next[e] = offsets[e]; }
+  for (int64_t t = 0; t < N; ++t) {
+    const int64_t g = m > 0 ? home_group(t, N, D, token_group) : 0;
+    uint64_t seen[4] = {0, 0, 0, 0};
+    for (int s = 0; s < slots; ++s) {
+      const int e = s < k ? topk_idx[t * k + s] : (int)g * m + (s - k);
+      const bool dup = (seen[e >> 6] >> (e & 63)) & 1u;       // a home-device expert that is also a top-k slot
+      seen[e >> 6] |= (uint64_t)1 << (e & 63);
+      const bool set = (keep_mask[t * W + (e >> 6)] >> (e & 63)) & 1u;
+      slot_row[t * slots + s] = (set && !dup) ? -2 : -1;      // -2: row assigned below, in expert order
+    }
+    for (int e = 0; e < E; ++e)
+      if (((keep_mask[t * W + (e >> 6)] >> (e & 63)) & 1u) && !((seen[e >> 6] >> (e & 63)) & 1u)) return 1;
+  }
+  // rows are handed out expert by expert in ascending token order
+  for (int64_t t = 0; t < N; ++t) {
+    const int64_t g = m > 0 ? home_group(t, N, D, token_group) : 0;
+    for (int s = 0; s < slots; ++s)
+      if (slot_row[t * slots + s] == -2) {
+        const int e = s < k ? topk_idx[t * k + s] : (int)g * m + (s - k);
+        slot_row[t * slots + s] = next[e]++;
+      }
+  }
+  return 0;
+}
+
 // Device-level capacity ("Advanced Variant: Device-Level Capacity-Aware Inference"): the constraint
 // is on the aggregated load of a device, N_1 + ... + N_{n_l} <= C_dev, not on each expert.  The
 // candidates of device g are all (token, expert) pairs with the expert on g (top-k pairs, plus

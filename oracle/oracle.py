@@ -19,7 +19,8 @@ _SRC = os.path.join(_HERE, "capmoe_oracle.cpp")
 _LIB = os.path.join(_HERE, "libcapmoe_oracle.so")
 _lib = None
 
-__all__ = ["build", "capacity", "device_capacity", "device_drop", "drop_keys", "drop_keyed", "METRICS", "router_logits", "softmax", "topk", "token_drop",
+__all__ = ["build", "capacity", "device_capacity", "device_drop", "drop_keys", "drop_keyed", "METRICS",
+           "priority_keys", "limit_experts", "rows_from_mask", "router_logits", "softmax", "topk", "token_drop",
            "expanded_drop",
            "permute", "expert_ffn", "combine", "layer_tokens", "stats", "layer_forward", "num_threads"]
 
@@ -171,6 +172,50 @@ def drop_keyed(keys: np.ndarray, topk_idx: np.ndarray, C: int, D: int = 1, expan
     _load().oracle_drop_keyed(_p(keys), _p(topk_idx), _i64(N), int(E), int(k), _i64(C), int(D), int(bool(expanded)),
                               _p(tg), _p(keep), _p(cand), _p(kept), _p(off), _p(slot_row))
     return dict(keep_mask=keep, cand=cand, kept=kept, offsets=off, slot_row=slot_row)
+
+
+def priority_keys(base: np.ndarray, idx: Optional[np.ndarray], E: int, exact: bool,
+                  token_class: Optional[np.ndarray] = None, topk_idx: Optional[np.ndarray] = None) -> np.ndarray:
+    """Keys with a priority class in the two high bits: 2 * [pair is a top-k pair] + token_class[t]
+    (modality-first dropping; Expanded Drop as substitution only)."""
+    base = np.ascontiguousarray(base, np.uint32)
+    N, cols = base.shape
+    ix = None if idx is None else np.ascontiguousarray(idx, np.int32)
+    tc = None if token_class is None else np.ascontiguousarray(token_class, np.uint8)
+    tk = None if topk_idx is None else np.ascontiguousarray(topk_idx, np.int32)
+    k = 0 if tk is None else tk.shape[1]
+    out = np.empty((N, cols), np.uint32)
+    rc = _load().oracle_priority_keys(_p(base), _p(ix), _i64(N), int(cols), int(E), int(bool(exact)), _p(tc), _p(tk),
+                                      int(k), _p(out))
+    if rc != 0:
+        raise ValueError("exact keys must be below 2^30")
+    return out
+
+
+def limit_experts(scores: np.ndarray, keep_mask: np.ndarray, k_max: int) -> np.ndarray:
+    """'w/ max': every token retains at most k_max of the experts that kept it, the best by score."""
+    scores = np.ascontiguousarray(scores, np.float32)
+    N, E = scores.shape
+    out = np.ascontiguousarray(keep_mask, np.uint64).copy()
+    _load().oracle_limit_experts(_p(scores), _i64(N), int(E), int(k_max), _p(out))
+    return out
+
+
+def rows_from_mask(keep_mask: np.ndarray, topk_idx: np.ndarray, E: int, slots: int, D: int = 1,
+                   token_group: Optional[np.ndarray] = None):
+    """Counts, offsets and slot rows of a keep mask (segments in ascending token order)."""
+    keep_mask = np.ascontiguousarray(keep_mask, np.uint64)
+    topk_idx = np.ascontiguousarray(topk_idx, np.int32)
+    N, k = topk_idx.shape
+    kept = np.empty((E,), np.int32)
+    off = np.empty((E + 1,), np.int32)
+    slot_row = np.empty((N, slots), np.int32)
+    tg = None if token_group is None else np.ascontiguousarray(token_group, np.int32)
+    rc = _load().oracle_rows_from_mask(_p(keep_mask), _p(topk_idx), _i64(N), int(E), int(k), int(slots), int(D),
+                                       _p(tg), _p(kept), _p(off), _p(slot_row))
+    if rc != 0:
+        raise ValueError("mask has a bit outside the token's slots")
+    return dict(kept=kept, offsets=off, slot_row=slot_row)
 
 
 def device_capacity(N: int, E: int, k: int, D: int, gamma: float, round_mode: str = "ceil") -> int:
