@@ -174,6 +174,39 @@ int capmoe_device_drop(const float* scores, const int32_t* topk_idx, int64_t N, 
                        uint64_t* keep_mask, int32_t* cand, int32_t* kept, int32_t* expert_offsets,
                        int32_t* slot_row, void* ws, size_t ws_bytes, void* stream);
 
+/* ---------------------------------------------------------------- priority classes, "w/ max"
+ * capmoe_priority_keys puts a priority class above a metric's key, for the two variants that
+ * rank candidates by a class before the metric:
+ *   - dropping by modality (multimodal section: "Image First" drops image tokens before any text
+ *     token, "Text First" the other way round): token_class[t] = 1 for the protected modality;
+ *   - Expanded Drop as substitution only (Expanded Drop paragraph: the expansion "makes no change
+ *     in the token assignments in experts that are overflowed by the top-k"): pass topk_idx and a
+ *     token's top-k pairs outrank the pairs it only has through its home device.  Without this
+ *     class all candidates compete equally, as in Algorithm 2.
+ * keys[i] = ((2*[pair is a top-k pair] + token_class[t]) << 30) | body, body = base[i] when exact != 0
+ * (the caller guarantees base < 2^30, true of every score in [0,1]; higher bits are masked off)
+ * else base[i] >> 2.  base/keys [N,cols] uint32 (may alias); idx as in capmoe_drop_keys;
+ * token_class [N] uint8 or NULL; topk_idx [N,k] or NULL.
+ *
+ * capmoe_limit_experts is the "w/ max" ablation (appendix "Maximum Number of Selected Experts"):
+ * every token retains at most k_max of the experts that kept it, the best by scores[t,e], ties to
+ * the lower expert id; keep_mask [N, ceil(E/64)] is edited in place, freed capacity is not handed
+ * on.  capmoe_rows_from_mask then rebuilds kept [E], expert_offsets [E+1] and slot_row [N,slots]
+ * (slots = k, or k + E/D with the home-device slots of stage 3) for that mask - or for any mask
+ * whose bits lie on the token's slots; *bad (device int32) is set to 1 if one does not, else 0.
+ * ws: ceil(N/256)*E*4 bytes (capmoe_drop_workspace_bytes(...) is enough).
+ * Global expansion (candidates = the token's k+m best experts anywhere) needs no call of its own:
+ * capmoe_route with k+m choices followed by capmoe_token_drop. */
+int capmoe_priority_keys(const uint32_t* base, const int32_t* idx, int64_t N, int cols, int E, int exact,
+                         const uint8_t* token_class, const int32_t* topk_idx, int k, uint32_t* keys,
+                         void* stream);
+int capmoe_limit_experts(const float* scores, int64_t N, int E, int k_max, uint64_t* keep_mask,
+                         void* stream);
+int capmoe_rows_from_mask(const uint64_t* keep_mask, const int32_t* topk_idx, int64_t N, int E, int k,
+                          int slots, int D, const int32_t* token_group, int32_t* kept,
+                          int32_t* expert_offsets, int32_t* slot_row, int32_t* bad, void* ws,
+                          size_t ws_bytes, void* stream);
+
 /* ---------------------------------------------------------------- stage 4: permute
  * x_perm[r] = x[t], perm_token[r] = t, perm_weight[r] = scores[t,e] for every kept (t,e) with
  * r = its slot_row entry.  slots = k after Token Drop (pass D = 0) or k+E/D after Expanded Drop.

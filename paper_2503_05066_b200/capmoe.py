@@ -26,7 +26,8 @@ MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2, "device_token_drop": 
 EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_drop_workspace_bytes", "capmoe_status_str",
            "capmoe_last_cuda_error", "capmoe_launch_count", "capmoe_ffn_uses_tensor_cores", "capmoe_route",
            "capmoe_token_drop", "capmoe_token_drop_static", "capmoe_expanded_drop", "capmoe_device_capacity",
-           "capmoe_device_drop", "capmoe_drop_keys", "capmoe_permute", "capmoe_grouped_ffn",
+           "capmoe_device_drop", "capmoe_drop_keys", "capmoe_priority_keys", "capmoe_limit_experts",
+           "capmoe_rows_from_mask", "capmoe_permute", "capmoe_grouped_ffn",
            "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe"]
 
 
@@ -239,6 +240,45 @@ def drop_keys(metric: str, seed: int, scores, idx, E: int, stream=None):
     _check(lib().capmoe_drop_keys(METRICS[metric], ctypes.c_uint64(seed), _ptr(scores), _ptr(idx), _i64(N),
                                   int(cols), int(E), _ptr(keys), _stream(stream)), "capmoe_drop_keys")
     return keys
+
+
+def priority_keys(base, idx, E: int, exact: bool, token_class=None, topk_idx=None, stream=None):
+    """Keys with a priority class above the metric's key: 2 * [pair is one of the token's top-k]
+    (when topk_idx is given: Expanded Drop as substitution only) + token_class[t] (uint8, 1 = the
+    protected modality).  base: the float32-typed key tensor drop_keys returns; same type back."""
+    N, cols = base.shape
+    keys = torch.empty_like(base)
+    k = 0 if topk_idx is None else topk_idx.shape[1]
+    _check(lib().capmoe_priority_keys(_ptr(base), _ptr(idx), _i64(N), int(cols), int(E), int(bool(exact)),
+                                      _ptr(token_class), _ptr(topk_idx), int(k), _ptr(keys), _stream(stream)),
+           "capmoe_priority_keys")
+    return keys
+
+
+def limit_experts(scores, keep_mask, k_max: int, stream=None):
+    """'w/ max': edits keep_mask in place so that no token sits on more than k_max experts."""
+    N, E = scores.shape
+    _check(lib().capmoe_limit_experts(_ptr(scores), _i64(N), int(E), int(k_max), _ptr(keep_mask), _stream(stream)),
+           "capmoe_limit_experts")
+    return keep_mask
+
+
+def rows_from_mask(keep_mask, topk_idx, E: int, slots: int, D: int = 1, token_group=None, ws=None, stream=None):
+    """-> dict(kept, offsets, slot_row, bad) for a keep mask whose bits lie on the tokens' slots."""
+    N, k = topk_idx.shape
+    dev = topk_idx.device
+    need = ((N + 255) // 256) * E * 4
+    if ws is None:
+        ws = torch.empty((max(need, 16),), device=dev, dtype=torch.uint8)
+    out = dict(kept=torch.empty((E,), device=dev, dtype=torch.int32),
+               offsets=torch.empty((E + 1,), device=dev, dtype=torch.int32),
+               slot_row=torch.empty((N, slots), device=dev, dtype=torch.int32),
+               bad=torch.zeros((1,), device=dev, dtype=torch.int32))
+    _check(lib().capmoe_rows_from_mask(_ptr(keep_mask), _ptr(topk_idx), _i64(N), int(E), int(k), int(slots), int(D),
+                                       _ptr(token_group), _ptr(out["kept"]), _ptr(out["offsets"]),
+                                       _ptr(out["slot_row"]), _ptr(out["bad"]), _ptr(ws),
+                                       ctypes.c_size_t(ws.numel()), _stream(stream)), "capmoe_rows_from_mask")
+    return out
 
 
 def device_capacity(N: int, E: int, k: int, D: int, gamma: float, round_mode: str = "ceil") -> int:
