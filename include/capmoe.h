@@ -230,10 +230,17 @@ int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int slots, int
  * D_straggler > 0 (E % D_straggler == 0) turns on straggler emulation: the experts of virtual
  * device g run only on a fixed share floor(#SM/D) of the SMs, so the most loaded device sets
  * the latency as under expert parallelism (Eq. 4, L proportional to max_i N_i).
- * dev_status [1] int32 (device, may be NULL): set to CAPMOE_ETIMEOUT if a bounded wait inside
- * the tensor-core kernel ran out; the caller zeroes it and reads it after synchronising.
+ * dev_status: NULL, or a device block of CAPMOE_FFN_STATUS_WORDS int32.  Word 0 is set to
+ * CAPMOE_ETIMEOUT if a bounded wait inside the tensor-core kernel ran out; the caller zeroes it
+ * and reads it after synchronising.  The other words are scratch that the call itself clears: the
+ * tile counters from which the kernels take their work in list order (so that tiles sharing an
+ * operand run at the same time whatever the speed of their SMs); with NULL, or more than
+ * CAPMOE_FFN_SCHED_GROUPS straggler groups, every CTA walks a fixed list of tiles instead.  Calls
+ * that overlap on the GPU need a block each.
  * bf16 with d % 64 == 0 and F % 128 == 0 runs on tcgen05 tensor cores with TMA-fed tiles;
  * everything else (fp32, odd shapes) runs a plain fp32-FMA kernel. */
+#define CAPMOE_FFN_SCHED_GROUPS 63
+#define CAPMOE_FFN_STATUS_WORDS (1 + 2 * CAPMOE_FFN_SCHED_GROUPS + 1)   /* 128 */
 int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F,
                        int dtype, const void* w_gate, const void* w_up, const void* w_down,
                        void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
@@ -278,7 +285,7 @@ typedef struct {
   const int32_t* one_segment;   /* [2] int32 holding {0, N}: the shared expert's single row segment */
   void* y;
   void* drop_ws; size_t drop_ws_bytes;
-  int32_t* dev_status;
+  int32_t* dev_status;   /* CAPMOE_FFN_STATUS_WORDS int32, see capmoe_grouped_ffn */
   /* Optional stage timing.  NULL, or CAPMOE_N_STAGE_EVENTS cudaEvent_t handles (as void*) that the
    * layer records on `stream`: [0] start, [1] after route, [2] after drop, [3] after permute,
    * [4] after the gate/up GEMM + SwiGLU, [5] after the down GEMM, [6] after the shared expert,

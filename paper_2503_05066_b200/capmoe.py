@@ -63,6 +63,7 @@ class _Layer(ctypes.Structure):
     ]
 
 N_STAGE_EVENTS = 8
+FFN_STATUS_WORDS = 128     # CAPMOE_FFN_STATUS_WORDS: status word + scratch of the FFN's tile schedulers
 STAGE_NAMES = ["route", "drop", "permute", "ffn_gate_up", "ffn_down", "shared_ffn", "combine"]
 
 
@@ -335,10 +336,12 @@ def permute(x, scores, topk_idx, slot_row, A_max: int, D: int = 0, token_group=N
 
 def grouped_ffn(x_perm, offsets, w_gate, w_up, w_down, D_straggler: int = 0, h_ws=None, y_perm=None,
                 dev_status=None, stream=None):
-    """-> y_perm [A_max, d]"""
+    """-> y_perm [A_max, d].  dev_status: int32 [FFN_STATUS_WORDS] (word 0 = device status), made here if None."""
     A_max, d = x_perm.shape
     E, F, _ = w_gate.shape
     dev = x_perm.device
+    if dev_status is None:
+        dev_status = torch.zeros((FFN_STATUS_WORDS,), device=dev, dtype=torch.int32)
     if h_ws is None:
         h_ws = torch.empty((A_max, F), device=dev, dtype=x_perm.dtype)
     if y_perm is None:
@@ -419,7 +422,7 @@ class MoELayer:
         t["y_perm"] = torch.zeros((max(A_max, 1), d), **act)
         t["y"] = torch.empty((N, d), **act)
         t["drop_ws"] = torch.empty((drop_workspace_bytes(N, E, k, D, expanded),), device=dev, dtype=torch.uint8)
-        t["dev_status"] = torch.zeros((1,), **i32)
+        t["dev_status"] = torch.zeros((FFN_STATUS_WORDS,), **i32)
         F_shared = 0
         if shared is not None:
             t["ws_gate"], t["ws_up"], t["ws_down"] = shared
@@ -477,6 +480,6 @@ class MoELayer:
         return y_host
 
     def check_device_status(self):
-        s = int(self.t["dev_status"].item())
+        s = int(self.t["dev_status"][0].item())
         if s != OK:
             raise CapmoeError(s, "device status")

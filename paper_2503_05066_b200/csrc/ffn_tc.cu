@@ -197,6 +197,94 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;                // shared::cluster address of the even CTA's copy
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Release at cluster scope: what this thread wrote into the other CTA's shared memory before the
+// arrive is visible to whoever acquires the barrier there.
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded like mbar_wait, acquiring at cluster scope (the signal may come from the other CTA).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1; it < 0x40000000u; ++it) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((it & 127u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// Tile queue of a CTA pair.  With a scheduler counter the pair does not walk a fixed list of
+// tiles: the leader's producer thread takes the next tile index from a global counter when it is
+// ready to load it and hands it to every role of both CTAs through a small ring in shared memory
+// (value + "full" barrier in each CTA, one "empty" barrier in the leader that all readers arrive
+// on).  Tiles that are neighbours in the list (same weight tile, next row block) are then
+// started within microseconds of each other whatever the speed of the SMs they run on, so their
+// shared operand tiles meet in L2, and no pair is left with a longer list than the others.
+__device__ __forceinline__ uint32_t peer_addr(uint32_t own) {   // same offset in CTA 1 of the pair
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, 1;" : "=r"(r) : "r"(own));
+  return r;
+}
+constexpr int TQ = 4;
+constexpr int TQ_READERS_PAIR = 2 + 2 * EPI_WARPS; // leader MMA thread, peer producer, epilogue warps of both CTAs
+constexpr int DYN_MIN_K = 2048;                    // shortest reduction length that takes tiles from the counter
+struct TileQueue {
+  uint32_t full0, empty0, val0;      // shared::cta addresses of full[TQ], empty[TQ] (leader's used), tile[TQ]
+  uint32_t rank;                     // CTA rank in the pair
+  volatile int* abort_flag;
+  __device__ __forceinline__ uint32_t full(int q) const { return full0 + 8u * (uint32_t)(q & (TQ - 1)); }
+  __device__ __forceinline__ uint32_t empty(int q) const { return empty0 + 8u * (uint32_t)(q & (TQ - 1)); }
+  __device__ __forceinline__ uint32_t val(int q) const { return val0 + 4u * (uint32_t)(q & (TQ - 1)); }
+  // leader's producer thread: publish tile (or -1 = no more) as entry q; false if a wait ran out
+  __device__ __forceinline__ bool put(int q, int tile) const {
+    const uint32_t par = (((uint32_t)q / TQ) & 1u) ^ 1u;
+    if (!mbar_wait(empty(q), par, abort_flag)) return false;     // only the count matters here
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(val(q)), "r"((uint32_t)tile) : "memory");
+    mbar_arrive(full(q));
+    st_cluster_u32(peer_addr(val(q)), (uint32_t)tile);           // the peer CTA's copy
+    mbar_arrive_cluster_release(peer_addr(full(q)));
+    return true;
+  }
+  // any other role (one thread, or one whole warp): entry q, or -2 if the wait ran out
+  __device__ __forceinline__ int get(int q, bool whole_warp) const {
+    const uint32_t par = ((uint32_t)q / TQ) & 1u;
+    // only the peer's copy was written from another CTA and needs the cluster-scope acquire
+    bool ok = rank != 0 ? mbar_wait_cluster(full(q), par, abort_flag) : mbar_wait(full(q), par, abort_flag);
+    if (whole_warp) ok = __all_sync(0xffffffffu, ok);
+    if (!ok) return -2;
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(val(q)) : "memory");
+    if (whole_warp) __syncwarp();
+    if (!whole_warp || (threadIdx.x & 31) == 0) {
+      if (rank == 0) mbar_arrive(empty(q));
+      else mbar_arrive_cluster(empty(q) & PEER_MASK);
+    }
+    return (int)v;
+  }
+};
+
 // ---------------------------------------------------------------- tile enumeration
 struct Tile { int e, row0, rows, n0; };
 
@@ -268,7 +356,6 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(MAX_STAGES + s); };
   auto tfull_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 + b); };
-
   if (tid == 0) {
     for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), nthreads - 64); }
@@ -606,7 +693,6 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
 constexpr int STAGES2 = 6;
 constexpr int HALF_B_BYTES = 128 * BK * 2;                 // 16 KB
 constexpr int STAGE2_BYTES = A_BYTES + HALF_B_BYTES;       // 32 KB per CTA
-constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;                // shared::cluster address of the even CTA's copy
 static_assert(STAGES2 * STAGE2_BYTES == STAGES * STAGE_BYTES, "both variants share one smem layout");
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -648,16 +734,12 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
       ::"r"(bar), "h"((uint16_t)3)
       : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
 template <int MODE>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
           const __grid_constant__ CUtensorMap map_b1, const int32_t* __restrict__ expert_offsets, int E,
           int K, int Nout, __nv_bfloat16* __restrict__ out, int D_straggler, int32_t* __restrict__ dev_status,
-          int group /* consecutive tiles one pair takes before it strides on */) {
+          int32_t* __restrict__ sched /* tile counters, one per straggler group, zeroed; NULL = fixed lists */) {
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
   constexpr int N_TILE = SWIGLU ? 128 : 256;
   constexpr int BM2 = 2 * BM;                                   // rows of a pair's tile
@@ -680,10 +762,13 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(MAX_STAGES + s); };
   auto tfull_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 + b); };
+  // tile queue: barriers 40..47 and four ints behind them, inside the 512-byte barrier block
+  const TileQueue tq{bar0 + 8u * 40u, bar0 + 8u * 44u, bar0 + 8u * 48u, rank, abort_flag};
 
   if (tid == 0) {
     for (int s = 0; s < STAGES2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 2 * EPI_WARPS * 32); }
+    for (int i = 0; i < TQ; ++i) { mbar_init(tq.full(i), 1); mbar_init(tq.empty(i), TQ_READERS_PAIR); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -712,19 +797,29 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   const uint32_t tmem_base = *tmem_slot;
 
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-  int tile_hi, stride, first;
+  int tile_lo, tile_hi, stride, first;
+  int32_t* counter = sched;                                     // this pair's group counter
   if (D_straggler > 0) {
     const int per = npairs / D_straggler;
     const int g = pair / per;
-    if (g >= D_straggler) { tile_hi = 0; first = 0; stride = 1; }
+    if (g >= D_straggler) { tile_lo = tile_hi = 0; first = 0; stride = 1; counter = nullptr; }
     else {
       const int m = E / D_straggler;
+      tile_lo = tile_start[g * m];
       tile_hi = tile_start[(g + 1) * m];
-      first = tile_start[g * m] + (pair - g * per) * group; stride = per * group;
+      first = tile_lo + (pair - g * per); stride = per;
+      if (sched) counter = sched + g;
     }
   } else {
-    tile_hi = tile_start[E]; first = pair * group; stride = npairs * group;
+    tile_lo = 0; tile_hi = tile_start[E]; first = pair; stride = npairs;
   }
+  const bool dyn = sched != nullptr;
+  // Next tile of this pair for a role: the fixed list, or the queue (the leader's producer thread
+  // fills it).  Returns a negative number when there is no further tile or a wait ran out.
+  auto next_tile = [&](int j, bool whole_warp) -> int {   // every role but the scheduler
+    if (!dyn) { const int tile = first + j * stride; return tile < tile_hi ? tile : -1; }
+    return tq.get(j, whole_warp);
+  };
   const int num_kb = (K + BK - 1) / BK;
 
   if (warp == 0) {
@@ -734,9 +829,22 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       uint32_t ph = 0;
       Tile t;
       bool ok = true;
+      int ahead = 0;                                     // the scheduler's number for the tile after this one
       for (int j = 0; ok; ++j) {
-        const int tile = first + (j / group) * stride + (j % group);
-        if (tile >= tile_hi) break;
+        int tile;
+        if (!dyn || rank != 0) {
+          tile = next_tile(j, false);
+          if (tile < 0) break;
+        } else {
+          // Taken one tile ahead, so that the counter's round trip never sits between two tiles' loads.
+          tile = -1;
+          if (counter) {
+            tile = tile_lo + (j == 0 ? atomicAdd(counter, 1) : ahead);
+            if (tile >= tile_hi) tile = -1;
+          }
+          if (!tq.put(j, tile) || tile < 0) break;
+          ahead = atomicAdd(counter, 1);
+        }
         if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
         const int my_row0 = t.row0 + (int)rank * BM;
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -764,8 +872,8 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       Tile t;
       bool ok = true;
       for (int j = 0; ok; ++j, ++it) {
-        const int tile = first + (j / group) * stride + (j % group);
-        if (tile >= tile_hi) break;
+        const int tile = next_tile(j, false);
+        if (tile < 0) break;
         if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
         const uint32_t b = it & 1u, use = it >> 1;
         if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -794,8 +902,8 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     uint32_t it = 0;
     Tile t;
     for (int j = 0;; ++j, ++it) {
-      const int tile = first + (j / group) * stride + (j % group);
-      if (tile >= tile_hi) break;
+      const int tile = next_tile(j, true);
+      if (tile < 0) break;
       if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
       const uint32_t b = it & 1u, use = it >> 1;
       bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
@@ -946,9 +1054,18 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     if (err != cudaSuccess) return note_cuda(err);
     err = cudaFuncSetAttribute(k_ffn_tc2<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (err != cudaSuccess) return note_cuda(err);
-    // Consecutive tiles one pair takes before striding on.  1 is best: the reuse of weight tiles
-    // comes from pairs that work on them at the same time (measured: 2, 4, 8 raise DRAM reads).
-    const int group1 = 1, group2 = 1;
+    // Tile counters of the two launches (one per straggler group), in the caller's status block.
+    // Taking tiles from a counter pays where a pair works through many long tiles: it halved the
+    // DRAM reads of the Mixtral-shape gate/up GEMM and was 5 % faster on the DeepSeek shape, but
+    // GEMMs with a short reduction (the OLMoE-shape down GEMM, K = 1024) measured 9 % slower with
+    // it, so those keep the fixed lists.
+    int32_t *sched1 = nullptr, *sched2 = nullptr;
+    if (dev_status && D_straggler <= CAPMOE_FFN_SCHED_GROUPS) {
+      err = cudaMemsetAsync(dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st);
+      if (err != cudaSuccess) return note_cuda(err);
+      if (d >= DYN_MIN_K) sched1 = dev_status + 1;
+      if (F >= DYN_MIN_K) sched2 = dev_status + 1 + CAPMOE_FFN_SCHED_GROUPS;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.blockDim = dim3(TC_THREADS);
@@ -960,13 +1077,13 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_GATE_UP>, a1, bg, bu, expert_offsets, E, d, F,
-                             (__nv_bfloat16*)h_ws, D_straggler, dev_status, group1);
+                             (__nv_bfloat16*)h_ws, D_straggler, dev_status, sched1);
     count_launch(1);
     if (err != cudaSuccess) return note_cuda(err);
     int rc2;
     if (mid && (rc2 = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc2;
     err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_DOWN>, a2, bd128, bd128, expert_offsets, E, F, d,
-                             (__nv_bfloat16*)y_perm, D_straggler, dev_status, group2);
+                             (__nv_bfloat16*)y_perm, D_straggler, dev_status, sched2);
     count_launch(1);
     return note_cuda(err);
   }
