@@ -36,7 +36,7 @@ UNIT = "tokens/s"
 # captures of the current kernel (profiles/launch_list_mixtral_expanded_drop.md,
 # profiles/k_ffn_tc2_olmoe_ncu_full.md); key = (config, N, F, mode, gamma)
 NCU_TRAFFIC_GATE_UP = {
-    ("mixtral", 8192, 14336, "expanded_drop", 1.0): 5541300000 + 462400000,
+    ("mixtral", 8192, 14336, "expanded_drop", 1.0): 2377500000 + 460200000,
     ("olmoe", 4096, 1024, "expanded_drop", 1.0): 671821056 + 60885248,
 }
 
