@@ -249,7 +249,8 @@ __device__ __forceinline__ uint32_t peer_addr(uint32_t own) {   // same offset i
 }
 constexpr int TQ = 4;
 constexpr int TQ_READERS_PAIR = 2 + 2 * EPI_WARPS; // leader MMA thread, peer producer, epilogue warps of both CTAs
-constexpr int DYN_MIN_K = 2048;                    // shortest reduction length that takes tiles from the counter
+// A GEMM takes its tiles from the counter if K >= DYN_MIN_K and (a pair gets >= DYN_MIN_TILES tiles or K >= DYN_LONG_K)
+constexpr int DYN_MIN_K = 2048, DYN_LONG_K = 8192, DYN_MIN_TILES = 24;
 struct TileQueue {
   uint32_t full0, empty0, val0;      // shared::cta addresses of full[TQ], empty[TQ] (leader's used), tile[TQ]
   uint32_t rank;                     // CTA rank in the pair
@@ -1055,16 +1056,23 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     err = cudaFuncSetAttribute(k_ffn_tc2<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (err != cudaSuccess) return note_cuda(err);
     // Tile counters of the two launches (one per straggler group), in the caller's status block.
-    // Taking tiles from a counter pays where a pair works through many long tiles: it halved the
-    // DRAM reads of the Mixtral-shape gate/up GEMM and was 5 % faster on the DeepSeek shape, but
-    // GEMMs with a short reduction (the OLMoE-shape down GEMM, K = 1024) measured 9 % slower with
-    // it, so those keep the fixed lists.
+    // Taking tiles from a counter pays where a pair works through many tiles or very long ones: it
+    // halved the DRAM reads of the Mixtral-shape gate/up GEMM (97 tiles per pair) and was 5 % faster
+    // on the DeepSeek shape (57 per pair), but measured 9 % slower on a short reduction (OLMoE-shape
+    // down GEMM, K = 1024) and 2 % slower on a short run (OLMoE shape, 14 tiles per pair), so those
+    // keep the fixed lists.
     int32_t *sched1 = nullptr, *sched2 = nullptr;
     if (dev_status && D_straggler <= CAPMOE_FFN_SCHED_GROUPS) {
       err = cudaMemsetAsync(dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st);
       if (err != cudaSuccess) return note_cuda(err);
-      if (d >= DYN_MIN_K) sched1 = dev_status + 1;
-      if (F >= DYN_MIN_K) sched2 = dev_status + 1 + CAPMOE_FFN_SCHED_GROUPS;
+      // (rows are bounded by A_max, so the tile counts are upper bounds)
+      const int64_t row_blocks = ceil_div(A_max, 2 * BM) + E;
+      auto pays = [&](int K, int64_t col_blocks) {
+        const int64_t per_pair = row_blocks * col_blocks / pairs;
+        return K >= DYN_MIN_K && (per_pair >= DYN_MIN_TILES || K >= DYN_LONG_K);
+      };
+      if (pays(d, ceil_div(F, 128))) sched1 = dev_status + 1;
+      if (pays(F, ceil_div(d, 256))) sched2 = dev_status + 1 + CAPMOE_FFN_SCHED_GROUPS;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));

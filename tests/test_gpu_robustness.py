@@ -162,3 +162,42 @@ def test_cuda_graph_replay_matches_direct_launches(cm, name, mode):
         torch.cuda.synchronize()
         assert torch.equal(y, y0) and torch.equal(layer.t["keep_mask"], keep0) and torch.equal(layer.t["slot_row"], rows0)
     layer.check_device_status()
+
+
+def test_ffn_result_does_not_depend_on_how_tiles_are_handed_out(cm):
+    """Long expert segments run on CTA pairs that take their tiles from a device counter when the
+    caller lends a status block, and walk fixed lists without one: same bits either way, run after run."""
+    E, d, F, rows = 4, 8192, 256, 1536
+    A = E * rows
+    g = torch.Generator().manual_seed(5)
+    x_perm = torch.randn((A, d), generator=g).to(torch.bfloat16).cuda()
+    wg = (torch.randn((E, F, d), generator=g) * 0.02).to(torch.bfloat16).cuda()
+    wu = (torch.randn((E, F, d), generator=g) * 0.02).to(torch.bfloat16).cuda()
+    wd = (torch.randn((E, d, F), generator=g) * 0.02).to(torch.bfloat16).cuda()
+    offsets = torch.arange(0, A + 1, rows, dtype=torch.int32).cuda()
+    L = cm.lib()
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    st = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    def run(status, D_straggler):
+        h = torch.empty((A, F), device="cuda", dtype=torch.bfloat16)
+        y = torch.zeros((A, d), device="cuda", dtype=torch.bfloat16)
+        rc = L.capmoe_grouped_ffn(p(x_perm), p(offsets), E, d, F, cm.BF16, p(wg), p(wu), p(wd), p(h), p(y),
+                                  ctypes.c_int64(A), D_straggler, None if status is None else p(status), st)
+        assert rc == cm.OK
+        torch.cuda.synchronize()
+        return y
+
+    for D_straggler in (0, 2):
+        fixed = run(None, D_straggler)
+        status = torch.zeros((cm.FFN_STATUS_WORDS,), device="cuda", dtype=torch.int32)
+        for _ in range(3):
+            assert torch.equal(run(status, D_straggler), fixed)
+            assert int(status[0].item()) == cm.OK
+        # the counters handed out every tile of the gate/up GEMM (K = d = 8192 takes the counter) and then
+        # ran past the end once per pair and group; the down GEMM (K = F = 256) kept its fixed lists
+        n_tiles = (A // 256) * (F // 128)
+        groups = max(D_straggler, 1)
+        taken = int(status[1:1 + groups].sum().item())
+        assert taken >= n_tiles and int(status[64:64 + groups].sum().item()) == 0
+    assert torch.isfinite(fixed.float()).all() and float(fixed.float().abs().max()) > 0
