@@ -173,6 +173,7 @@ def run_table(args):
     base = _pick_config(args)
     Ns = synth.QWEN_SWEEP_N if (base.name == "qwen" and args.N is None) else (base.N,)
     steps, warmup = max(3, min(args.steps, 30)), max(3, min(args.warmup, 5))
+    md_head = False
     for N in Ns:
         cfg = base.with_(N=N)
         inp = synth.make_layer_inputs(cfg)
@@ -196,7 +197,7 @@ def run_table(args):
                 A = int(lay.t["expert_offsets"][-1].item())
                 nbar = N * cfg.k / cfg.E
                 m = cfg.E // cfg.D
-                print(json.dumps({
+                row = {
                     "config": cfg.name, "N": N, "mode": mode, "gamma": gamma, "straggler_emulation": strag,
                     "C": int(lay.C), "ms_per_layer": ms, "ms_per_layer_graph": graph_ms, "tokens_per_s": N / (ms * 1e-3),
                     "speedup_vs_nodrop": nodrop_ms[strag] / ms,
@@ -204,7 +205,19 @@ def run_table(args):
                     "max_device_kept_over_mean": float(kept.reshape(cfg.D, m).sum(1).max() / (nbar * m)),
                     "A": A, "kept_over_Nk": A / (N * cfg.k),
                     "dropped_fraction_of_topk": float(1.0 - min(A, N * cfg.k) / (N * cfg.k)) if "expanded" not in mode
-                    else None}), flush=True)
+                    else None}
+                if args.markdown:
+                    if not md_head:
+                        md_head = True
+                        print("| N | mode | γ | strag | C | A | A/(N·k) | max load | max kept | max dev | ms/layer | as one graph "
+                              "| tokens/s | speedup |\n|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+                    print("| %d | %s | %s | %s | %d | %d | %.2f | %.2f | %.2f | %.2f | %.3f | %.3f | %.2e | %.2f |" % (
+                        N, mode, "∞" if gamma is None else gamma, "on" if strag else "off", row["C"], A,
+                        row["kept_over_Nk"], row["max_load_over_mean"], row["max_kept_over_mean"],
+                        row["max_device_kept_over_mean"], ms, graph_ms, row["tokens_per_s"], row["speedup_vs_nodrop"]),
+                        flush=True)
+                else:
+                    print(json.dumps(row), flush=True)
                 del lay
         del g, inp
 
@@ -277,6 +290,7 @@ def main():
     ap.add_argument("--table", action="store_true",
                     help="instead of the benchmark line, print one JSON line per (N, gamma, mode) point of the "
                          "chosen config (for the Qwen-shape sweep: N in 128..65536, gamma in 0.5..2.0)")
+    ap.add_argument("--markdown", action="store_true", help="with --table: print a markdown table instead of JSON lines")
     ap.add_argument("--no-cpu", dest="cpu", action="store_false", help="skip the CPU baseline")
     ap.add_argument("--impl", default="capmoe", choices=["capmoe", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=None,
@@ -356,6 +370,10 @@ def main():
     ms_step = max_over_ranks(e0.elapsed_time(e1) / K)
     value = distrib.job_throughput(cfg.N, ms_step, info)
 
+    # per-step device time from each step's first to its last stage event: spread of the K steps
+    per_step = sorted(events[i][0].elapsed_time(events[i][capmoe.N_STAGE_EVENTS - 1]) for i in range(K))
+    step_spread = {"median_ms": statistics.median(per_step), "min_ms": per_step[0], "max_ms": per_step[-1],
+                   "note": "first to last stage event of one step; ms_per_step also counts the gap between steps"}
     stage_ms = {}
     for si, name in enumerate(capmoe.STAGE_NAMES):
         stage_ms[name] = statistics.mean(events[i][si].elapsed_time(events[i][si + 1]) for i in range(K))
@@ -527,7 +545,7 @@ def main():
             "dtype": cfg.dtype, "data": "synthetic", "config": _config_dict(cfg, args),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu,
-            "stages_ms": stage_ms, "hbm_stages": hbm_stages, "hbm_kernels": hbm_kernels,
+            "step_spread": step_spread, "stages_ms": stage_ms, "hbm_stages": hbm_stages, "hbm_kernels": hbm_kernels,
             "workload_stats": {"A": A, "C": int(layer_C(cfg, args, capmoe)), "max_load_over_mean": max(load) / nbar,
                                "kept_fraction_of_Nk": A / (cfg.N * cfg.k), "kept_per_expert": kept,
                                "load_per_expert": load},
