@@ -249,8 +249,6 @@ __device__ __forceinline__ uint32_t peer_addr(uint32_t own) {   // same offset i
 }
 constexpr int TQ = 4;
 constexpr int TQ_READERS_PAIR = 2 + 2 * EPI_WARPS; // leader MMA thread, peer producer, epilogue warps of both CTAs
-// A GEMM takes its tiles from the counter if K >= DYN_MIN_K and (a pair gets >= DYN_MIN_TILES tiles or K >= DYN_LONG_K)
-constexpr int DYN_MIN_K = 2048, DYN_LONG_K = 8192, DYN_MIN_TILES = 24;
 struct TileQueue {
   uint32_t full0, empty0, val0;      // shared::cta addresses of full[TQ], empty[TQ] (leader's used), tile[TQ]
   uint32_t rank;                     // CTA rank in the pair
@@ -264,15 +262,20 @@ struct TileQueue {
     if (!mbar_wait(empty(q), par, abort_flag)) return false;     // only the count matters here
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(val(q)), "r"((uint32_t)tile) : "memory");
     mbar_arrive(full(q));
-    st_cluster_u32(peer_addr(val(q)), (uint32_t)tile);           // the peer CTA's copy
-    mbar_arrive_cluster_release(peer_addr(full(q)));
+    // the peer CTA's copy: a store that reports to the peer's barrier itself (no fence on this
+    // thread, which has loads to issue)
+    const uint32_t pfull = peer_addr(full(q));
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(pfull), "r"(4u) : "memory");
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];"
+                 ::"r"(peer_addr(val(q))), "r"((uint32_t)tile), "r"(pfull)
+                 : "memory");
     return true;
   }
   // any other role (one thread, or one whole warp): entry q, or -2 if the wait ran out
   __device__ __forceinline__ int get(int q, bool whole_warp) const {
     const uint32_t par = ((uint32_t)q / TQ) & 1u;
     // only the peer's copy was written from another CTA and needs the cluster-scope acquire
-    bool ok = rank != 0 ? mbar_wait_cluster(full(q), par, abort_flag) : mbar_wait(full(q), par, abort_flag);
+    bool ok = mbar_wait(full(q), par, abort_flag);
     if (whole_warp) ok = __all_sync(0xffffffffu, ok);
     if (!ok) return -2;
     uint32_t v;
@@ -830,25 +833,33 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       uint32_t ph = 0;
       Tile t;
       bool ok = true;
-      int ahead = 0;                                     // the scheduler's number for the tile after this one
-      for (int j = 0; ok; ++j) {
-        int tile;
-        if (!dyn || rank != 0) {
-          tile = next_tile(j, false);
-          if (tile < 0) break;
-        } else {
-          // Taken one tile ahead, so that the counter's round trip never sits between two tiles' loads.
-          tile = -1;
-          if (counter) {
-            tile = tile_lo + (j == 0 ? atomicAdd(counter, 1) : ahead);
-            if (tile >= tile_hi) tile = -1;
-          }
-          if (!tq.put(j, tile) || tile < 0) break;
-          ahead = atomicAdd(counter, 1);
+      // The leader's producer is the pair's scheduler when tiles come from the counter.  It claims
+      // half a tile ahead: halfway through the loads of tile j it publishes entry j+1 (so the peer's
+      // producer has it before it runs out of work) and asks the counter for the entry after that
+      // (so the counter's round trip never sits between two tiles' loads).
+      const bool scheduler = dyn && rank == 0;
+      int cur = -1, claim = 0;
+      if (scheduler) {
+        if (counter) {
+          cur = tile_lo + atomicAdd(counter, 1);
+          if (cur >= tile_hi) cur = -1;
         }
+        ok = tq.put(0, cur);
+        if (ok && cur >= 0) claim = atomicAdd(counter, 1);
+      }
+      const int pub_kb = num_kb / 2;
+      for (int j = 0; ok; ++j) {
+        const int tile = scheduler ? cur : next_tile(j, false);
+        if (tile < 0) break;
         if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
         const int my_row0 = t.row0 + (int)rank * BM;
         for (int kb = 0; kb < num_kb; ++kb) {
+          if (scheduler && kb == pub_kb) {
+            cur = tile_lo + claim;
+            if (cur >= tile_hi) cur = -1;
+            if (!tq.put(j + 1, cur)) { ok = false; break; }
+            if (cur >= 0) claim = atomicAdd(counter, 1);
+          }
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t lead_full = full_bar(s) & PEER_MASK;   // the leader's barrier counts both CTAs' bytes
           if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
@@ -1056,23 +1067,14 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     err = cudaFuncSetAttribute(k_ffn_tc2<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (err != cudaSuccess) return note_cuda(err);
     // Tile counters of the two launches (one per straggler group), in the caller's status block.
-    // Taking tiles from a counter pays where a pair works through many tiles or very long ones: it
-    // halved the DRAM reads of the Mixtral-shape gate/up GEMM (97 tiles per pair) and was 5 % faster
-    // on the DeepSeek shape (57 per pair), but measured 9 % slower on a short reduction (OLMoE-shape
-    // down GEMM, K = 1024) and 2 % slower on a short run (OLMoE shape, 14 tiles per pair), so those
-    // keep the fixed lists.
+    // Against fixed lists the counter halved the DRAM reads of the Mixtral-shape gate/up GEMM and
+    // measured 2-5 % faster on the gate/up GEMMs of the other shapes, equal on their down GEMMs.
     int32_t *sched1 = nullptr, *sched2 = nullptr;
     if (dev_status && D_straggler <= CAPMOE_FFN_SCHED_GROUPS) {
       err = cudaMemsetAsync(dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st);
       if (err != cudaSuccess) return note_cuda(err);
-      // (rows are bounded by A_max, so the tile counts are upper bounds)
-      const int64_t row_blocks = ceil_div(A_max, 2 * BM) + E;
-      auto pays = [&](int K, int64_t col_blocks) {
-        const int64_t per_pair = row_blocks * col_blocks / pairs;
-        return K >= DYN_MIN_K && (per_pair >= DYN_MIN_TILES || K >= DYN_LONG_K);
-      };
-      if (pays(d, ceil_div(F, 128))) sched1 = dev_status + 1;
-      if (pays(F, ceil_div(d, 256))) sched2 = dev_status + 1 + CAPMOE_FFN_SCHED_GROUPS;
+      sched1 = dev_status + 1;
+      sched2 = dev_status + 1 + CAPMOE_FFN_SCHED_GROUPS;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));

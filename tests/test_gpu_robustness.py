@@ -167,7 +167,7 @@ def test_cuda_graph_replay_matches_direct_launches(cm, name, mode):
 def test_ffn_result_does_not_depend_on_how_tiles_are_handed_out(cm):
     """Long expert segments run on CTA pairs that take their tiles from a device counter when the
     caller lends a status block, and walk fixed lists without one: same bits either way, run after run."""
-    E, d, F, rows = 4, 8192, 256, 1536
+    E, d, F, rows = 4, 2048, 256, 1536
     A = E * rows
     g = torch.Generator().manual_seed(5)
     x_perm = torch.randn((A, d), generator=g).to(torch.bfloat16).cuda()
@@ -194,10 +194,8 @@ def test_ffn_result_does_not_depend_on_how_tiles_are_handed_out(cm):
         for _ in range(3):
             assert torch.equal(run(status, D_straggler), fixed)
             assert int(status[0].item()) == cm.OK
-        # the counters handed out every tile of the gate/up GEMM (K = d = 8192 takes the counter) and then
-        # ran past the end once per pair and group; the down GEMM (K = F = 256) kept its fixed lists
-        n_tiles = (A // 256) * (F // 128)
+        # each GEMM's counters handed out every one of its tiles, then ran past the end once per pair
         groups = max(D_straggler, 1)
-        taken = int(status[1:1 + groups].sum().item())
-        assert taken >= n_tiles and int(status[64:64 + groups].sum().item()) == 0
+        for base, n_tiles in ((1, (A // 256) * (F // 128)), (64, (A // 256) * (d // 256))):
+            assert int(status[base:base + groups].sum().item()) >= n_tiles
     assert torch.isfinite(fixed.float()).all() and float(fixed.float().abs().max()) > 0
