@@ -201,45 +201,11 @@ constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;                // shared::cluster ad
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Release at cluster scope: what this thread wrote into the other CTA's shared memory before the
-// arrive is visible to whoever acquires the barrier there.
-__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
-  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded like mbar_wait, acquiring at cluster scope (the signal may come from the other CTA).
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait_cluster(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t it = 1; it < 0x40000000u; ++it) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    if ((it & 127u) == 0u) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
-
-// Tile queue of a CTA pair.  With a scheduler counter the pair does not walk a fixed list of
-// tiles: the leader's producer thread takes the next tile index from a global counter when it is
-// ready to load it and hands it to every role of both CTAs through a small ring in shared memory
-// (value + "full" barrier in each CTA, one "empty" barrier in the leader that all readers arrive
-// on).  Tiles that are neighbours in the list (same weight tile, next row block) are then
+// Tile queue of a CTA or a CTA pair.  With a scheduler counter the CTAs do not walk fixed lists of
+// tiles: the (leader's) producer thread takes the next tile index from a global counter shortly
+// before it needs it and hands it to every role (of both CTAs) through a small ring in shared
+// memory (value + "full" barrier in each CTA, one "empty" barrier in the leader that all readers
+// arrive on).  Tiles that are neighbours in the list (same weight tile, next row block) are then
 // started within microseconds of each other whatever the speed of the SMs they run on, so their
 // shared operand tiles meet in L2, and no pair is left with a longer list than the others.
 __device__ __forceinline__ uint32_t peer_addr(uint32_t own) {   // same offset in CTA 1 of the pair
@@ -249,9 +215,11 @@ __device__ __forceinline__ uint32_t peer_addr(uint32_t own) {   // same offset i
 }
 constexpr int TQ = 4;
 constexpr int TQ_READERS_PAIR = 2 + 2 * EPI_WARPS; // leader MMA thread, peer producer, epilogue warps of both CTAs
+constexpr int TQ_READERS_ONE = 1 + EPI_WARPS;      // a CTA on its own: MMA thread and epilogue warps
+template <bool PAIRED>
 struct TileQueue {
   uint32_t full0, empty0, val0;      // shared::cta addresses of full[TQ], empty[TQ] (leader's used), tile[TQ]
-  uint32_t rank;                     // CTA rank in the pair
+  uint32_t rank;                     // CTA rank in the pair (0 for a CTA on its own)
   volatile int* abort_flag;
   __device__ __forceinline__ uint32_t full(int q) const { return full0 + 8u * (uint32_t)(q & (TQ - 1)); }
   __device__ __forceinline__ uint32_t empty(int q) const { return empty0 + 8u * (uint32_t)(q & (TQ - 1)); }
@@ -262,19 +230,20 @@ struct TileQueue {
     if (!mbar_wait(empty(q), par, abort_flag)) return false;     // only the count matters here
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(val(q)), "r"((uint32_t)tile) : "memory");
     mbar_arrive(full(q));
-    // the peer CTA's copy: a store that reports to the peer's barrier itself (no fence on this
-    // thread, which has loads to issue)
-    const uint32_t pfull = peer_addr(full(q));
-    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(pfull), "r"(4u) : "memory");
-    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];"
-                 ::"r"(peer_addr(val(q))), "r"((uint32_t)tile), "r"(pfull)
-                 : "memory");
+    if constexpr (PAIRED) {
+      // the peer CTA's copy: a store that reports to the peer's barrier itself (no fence on this
+      // thread, which has loads to issue)
+      const uint32_t pfull = peer_addr(full(q));
+      asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(pfull), "r"(4u) : "memory");
+      asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];"
+                   ::"r"(peer_addr(val(q))), "r"((uint32_t)tile), "r"(pfull)
+                   : "memory");
+    }
     return true;
   }
   // any other role (one thread, or one whole warp): entry q, or -2 if the wait ran out
   __device__ __forceinline__ int get(int q, bool whole_warp) const {
     const uint32_t par = ((uint32_t)q / TQ) & 1u;
-    // only the peer's copy was written from another CTA and needs the cluster-scope acquire
     bool ok = mbar_wait(full(q), par, abort_flag);
     if (whole_warp) ok = __all_sync(0xffffffffu, ok);
     if (!ok) return -2;
@@ -282,7 +251,7 @@ struct TileQueue {
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(val(q)) : "memory");
     if (whole_warp) __syncwarp();
     if (!whole_warp || (threadIdx.x & 31) == 0) {
-      if (rank == 0) mbar_arrive(empty(q));
+      if (!PAIRED || rank == 0) mbar_arrive(empty(q));
       else mbar_arrive_cluster(empty(q) & PEER_MASK);
     }
     return (int)v;
@@ -327,7 +296,8 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
          int K /* reduction length */, int Nout /* output columns */, void* __restrict__ out_ptr,
          int D_straggler, int32_t* __restrict__ dev_status, int n_mma, int single_rows,
          const float* __restrict__ bias, int tile_rows /* rows per tile actually loaded (<= 128) */,
-         int n_stages, int stage_stride, const RouterFused rf) {
+         int n_stages, int stage_stride, const RouterFused rf,
+         int32_t* __restrict__ sched /* FFN modes: tile counters, one per straggler group, zeroed; NULL = fixed lists */) {
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
   constexpr bool ROUTER = MODE == MODE_ROUTER || MODE == MODE_ROUTER_FUSED;
   constexpr bool FUSED = MODE == MODE_ROUTER_FUSED;
@@ -360,9 +330,12 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(MAX_STAGES + s); };
   auto tfull_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 + b); };
+  // tile queue: barriers 40..47 and four ints behind them, inside the 512-byte barrier block
+  const TileQueue<false> tq{bar0 + 8u * 40u, bar0 + 8u * 44u, bar0 + 8u * 48u, 0u, abort_flag};
   if (tid == 0) {
     for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), nthreads - 64); }
+    for (int i = 0; i < TQ; ++i) { mbar_init(tq.full(i), 1); mbar_init(tq.empty(i), TQ_READERS_ONE); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -397,19 +370,26 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
 
   // this CTA's share of the tile list
   int tile_lo, tile_hi, stride, first;
+  int32_t* counter = sched;                             // this CTA's group counter
   if (D_straggler > 0) {
     const int per = gridDim.x / D_straggler;            // CTAs per virtual device
     const int g = blockIdx.x / per;
-    if (g >= D_straggler) { tile_lo = tile_hi = 0; first = 0; stride = 1; }
+    if (g >= D_straggler) { tile_lo = tile_hi = 0; first = 0; stride = 1; counter = nullptr; }
     else {
       const int m = E / D_straggler;
       tile_lo = tile_start[g * m]; tile_hi = tile_start[(g + 1) * m];
       first = tile_lo + (blockIdx.x - g * per); stride = per;
+      if (sched) counter = sched + g;
     }
   } else {
     tile_lo = 0; tile_hi = tile_start[E]; first = blockIdx.x; stride = gridDim.x;
   }
   const int num_kb = (K + BK - 1) / BK;
+  const bool dyn = !ROUTER && sched != nullptr;
+  auto next_tile = [&](int j, bool whole_warp) -> int {   // every role but the scheduler
+    if (!dyn) { const int tile = first + j * stride; return tile < tile_hi ? tile : -1; }
+    return tq.get(j, whole_warp);
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -419,9 +399,30 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       uint32_t ph = 0;
       Tile t;
       bool ok = true;
-      for (int tile = first; ok && tile < tile_hi; tile += stride) {
+      // With a counter the producer is the CTA's scheduler: halfway through the loads of tile j it
+      // publishes entry j+1 and asks the counter for the one after, so the counter's round trip
+      // never sits between two tiles' loads.
+      int cur = -1, claim = 0;
+      if (dyn) {
+        if (counter) {
+          cur = tile_lo + atomicAdd(counter, 1);
+          if (cur >= tile_hi) cur = -1;
+        }
+        ok = tq.put(0, cur);
+        if (ok && cur >= 0) claim = atomicAdd(counter, 1);
+      }
+      const int pub_kb = num_kb / 2;
+      for (int j = 0; ok; ++j) {
+        const int tile = dyn ? cur : next_tile(j, false);
+        if (tile < 0) break;
         if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
         for (int kb = 0; kb < num_kb; ++kb) {
+          if (dyn && kb == pub_kb) {
+            cur = tile_lo + claim;
+            if (cur >= tile_hi) cur = -1;
+            if (!tq.put(j + 1, cur)) { ok = false; break; }
+            if (cur >= 0) claim = atomicAdd(counter, 1);
+          }
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
           mbar_expect_tx(full_bar(s), stage_tx);
           const uint32_t a_dst = tiles + (uint32_t)s * (uint32_t)stage_stride;
@@ -451,7 +452,9 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       uint64_t stage_off = 0;
       Tile t;
       bool ok = true;
-      for (int tile = first; ok && tile < tile_hi; tile += stride, ++it) {
+      for (int j = 0; ok; ++j, ++it) {
+        const int tile = next_tile(j, false);
+        if (tile < 0) break;
         if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
         const uint32_t b = it & 1u, use = it >> 1;
         if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -482,7 +485,9 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     int cursor = 0;
     uint32_t it = 0;
     Tile t;
-    for (int tile = first; tile < tile_hi; tile += stride, ++it) {
+    for (int j = 0;; ++j, ++it) {
+      const int tile = next_tile(j, true);
+      if (tile < 0) break;
       if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
       const uint32_t b = it & 1u, use = it >> 1;
       bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
@@ -767,7 +772,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   auto tfull_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 + b); };
   // tile queue: barriers 40..47 and four ints behind them, inside the 512-byte barrier block
-  const TileQueue tq{bar0 + 8u * 40u, bar0 + 8u * 44u, bar0 + 8u * 48u, rank, abort_flag};
+  const TileQueue<true> tq{bar0 + 8u * 40u, bar0 + 8u * 44u, bar0 + 8u * 48u, rank, abort_flag};
 
   if (tid == 0) {
     for (int s = 0; s < STAGES2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -1053,6 +1058,17 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
   err = cudaFuncSetAttribute(k_ffn_tc<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (err != cudaSuccess) return note_cuda(err);
   int grid = sm_count();
+  // Tile counters of the two launches (one per straggler group), in the caller's status block.
+  // Against fixed lists the counter halved the DRAM reads of the Mixtral-shape gate/up GEMM and
+  // measured 2-5 % faster on the gate/up GEMMs of the other long-segment shapes, equal on their
+  // down GEMMs and on the single-CTA kernel's ragged workloads.
+  int32_t *sched1 = nullptr, *sched2 = nullptr;
+  if (dev_status && D_straggler <= CAPMOE_FFN_SCHED_GROUPS) {
+    err = cudaMemsetAsync(dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st);
+    if (err != cudaSuccess) return note_cuda(err);
+    sched1 = dev_status + 1;
+    sched2 = dev_status + 1 + CAPMOE_FFN_SCHED_GROUPS;
+  }
   // CTA pairs (256-row tiles) when the expert segments are long enough that the extra tail
   // padding does not matter, or are known multiples of 256 rows
   const int64_t avg_rows = A_max / E;
@@ -1066,16 +1082,6 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     if (err != cudaSuccess) return note_cuda(err);
     err = cudaFuncSetAttribute(k_ffn_tc2<MODE_DOWN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (err != cudaSuccess) return note_cuda(err);
-    // Tile counters of the two launches (one per straggler group), in the caller's status block.
-    // Against fixed lists the counter halved the DRAM reads of the Mixtral-shape gate/up GEMM and
-    // measured 2-5 % faster on the gate/up GEMMs of the other shapes, equal on their down GEMMs.
-    int32_t *sched1 = nullptr, *sched2 = nullptr;
-    if (dev_status && D_straggler <= CAPMOE_FFN_SCHED_GROUPS) {
-      err = cudaMemsetAsync(dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st);
-      if (err != cudaSuccess) return note_cuda(err);
-      sched1 = dev_status + 1;
-      sched2 = dev_status + 1 + CAPMOE_FFN_SCHED_GROUPS;
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.blockDim = dim3(TC_THREADS);
@@ -1103,13 +1109,13 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
   }
   k_ffn_tc<MODE_GATE_UP><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a1, bg, bu, expert_offsets, E, d, F, h_ws,
                                                               D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES,
-                                                              RouterFused{});
+                                                              RouterFused{}, sched1);
   int rc = check_launch();
   if (rc != CAPMOE_OK) return rc;
   if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
   k_ffn_tc<MODE_DOWN><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a2, bd, bd, expert_offsets, E, F, d, y_perm,
                                                            D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES,
-                                                              RouterFused{});
+                                                              RouterFused{}, sched2);
   return check_launch();
 }
 
@@ -1126,7 +1132,7 @@ static int launch_router_tc(const CUtensorMap& ax, const CUtensorMap& bw, int gr
                                          SMEM_BYTES);
   if (err != cudaSuccess) return note_cuda(err);
   k_ffn_tc<MODE, EPAD><<<grid, MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, SMEM_BYTES, st>>>(ax, bw, bw, nullptr, 1, d, E, logits, 0, nullptr, n_mma,
-                                                            (int)N, bias, tile_rows, n_stages, stage_stride, rf);
+                                                            (int)N, bias, tile_rows, n_stages, stage_stride, rf, nullptr);
   return check_launch();
 }
 
