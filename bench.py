@@ -457,6 +457,60 @@ def main():
                        for k, v in hbm_kernels.items()}
         del xs, p_outs, ys, y_outs
 
+    # The drop stage moves a few MB: it is bound by launch and dependency latency, not by bandwidth.
+    # Reported against the measured device time of a launch that does (almost) nothing: a one-element
+    # capmoe_drop_keys call, the smallest kernel the library has (both replayed from CUDA graphs).
+    latency_stages = {}
+    if rank == 0 and args.mode != "nodrop":
+        t = layer.t
+
+        def timed_graph(fn, inner=16, graph_reps=10):
+            """ms per call of fn, replayed from a CUDA graph of `inner` calls: device time without the
+            host's per-call cost (which exceeds these kernels' duration)."""
+            fn(0)
+            torch.cuda.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.graph(gr, stream=side):
+                for i in range(inner):
+                    fn(i)
+            gr.replay()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(graph_reps):
+                gr.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / (graph_reps * inner)
+
+        one = torch.zeros((1, cfg.E), device=dev, dtype=torch.float32)
+        one_keys = torch.empty_like(one)
+        L_ = capmoe.lib()
+        import ctypes as _ct
+        st_ = lambda: _ct.c_void_p(torch.cuda.current_stream().cuda_stream)
+        floor_ms = timed_graph(lambda i: L_.capmoe_drop_keys(0, _ct.c_uint64(0), _ct.c_void_p(one.data_ptr()), None,
+                                                             _ct.c_int64(1), cfg.E, cfg.E,
+                                                             _ct.c_void_p(one_keys.data_ptr()), st_()))
+        l0 = capmoe.launch_count()
+        if args.mode == "token_drop":
+            fn = lambda i: capmoe.token_drop(t["topk_score"], t["topk_idx"], cfg.E, layer.C, ws=t["drop_ws"])
+            drop_bytes = 16 * cfg.N * cfg.k + 8 * cfg.N
+        elif args.mode == "expanded_drop":
+            fn = lambda i: capmoe.expanded_drop(t["scores"], t["topk_idx"], layer.C, cfg.D, ws=t["drop_ws"])
+            drop_bytes = 4 * cfg.N * cfg.E + 4 * cfg.N * cfg.k + 8 * cfg.N + 4 * cfg.N * layer.slots
+        else:
+            fn = lambda i: capmoe.device_drop(t["scores"], t["topk_idx"], layer.C, cfg.D,
+                                              args.mode == "device_expanded_drop", ws=t["drop_ws"])
+            drop_bytes = 4 * cfg.N * cfg.E + 4 * cfg.N * cfg.k + 8 * cfg.N + 4 * cfg.N * layer.slots
+        fn(0)
+        n_launch = capmoe.launch_count() - l0
+        ms = timed_graph(fn)
+        latency_stages["drop"] = {"ms": ms, "kernel_launches": int(n_launch), "bytes": drop_bytes,
+                                  "near_empty_launch_us": floor_ms * 1e3,
+                                  "launch_floor_ms": floor_ms * n_launch,
+                                  "times_launch_floor": ms / (floor_ms * n_launch) if n_launch else None}
+
     # ------------------------------------------------------------------ e2e through the host-buffer entry point
     # Every step copies its activations in from pinned host memory and its output back out, inside
     # the timed region.  Two layer instances (own activation buffers, shared weights) alternate on
@@ -545,7 +599,7 @@ def main():
             "dtype": cfg.dtype, "data": "synthetic", "config": _config_dict(cfg, args),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu,
-            "step_spread": step_spread, "stages_ms": stage_ms, "hbm_stages": hbm_stages, "hbm_kernels": hbm_kernels,
+            "step_spread": step_spread, "stages_ms": stage_ms, "hbm_stages": hbm_stages, "hbm_kernels": hbm_kernels, "latency_stages": latency_stages,
             "workload_stats": {"A": A, "C": int(layer_C(cfg, args, capmoe)), "max_load_over_mean": max(load) / nbar,
                                "kept_fraction_of_Nk": A / (cfg.N * cfg.k), "kept_per_expert": kept,
                                "load_per_expert": load},
