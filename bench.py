@@ -180,14 +180,19 @@ def run_table(args):
         g = {k: getattr(inp, k).cuda() for k in ("x", "w_router", "bias", "w_gate", "w_up", "w_down")}
         shared = None if inp.shared is None else tuple(s.cuda() for s in inp.shared)
         nodrop_ms = {}
-        points = [("nodrop", None)] + [(m, gm) for gm in cfg.gammas
-                                       for m in ("token_drop", "expanded_drop", "device_token_drop",
-                                                 "device_expanded_drop")]
-        for mode, gamma in points:
+        points = [("nodrop", None, "", {})] + [(m, gm, "", {}) for gm in cfg.gammas
+                                               for m in ("token_drop", "expanded_drop", "device_token_drop",
+                                                         "device_expanded_drop")]
+        # variants of the drop at the first capacity factor
+        g0 = cfg.gammas[0]
+        points += [("token_drop", g0, "+random", dict(metric="random", seed=1)),
+                   ("expanded_drop", g0, "+topk_first", dict(topk_first=True)),
+                   ("expanded_drop", g0, "+max_k", dict(max_experts=cfg.k))]
+        for mode, gamma, tag, variant in points:
             for strag in ([False, True] if cfg.straggler else [False]):
                 lay = capmoe.MoELayer(g["x"], g["w_router"], g["bias"], g["w_gate"], g["w_up"], g["w_down"], cfg.k,
                                       cfg.D, mode, gamma=1.0 if gamma is None else gamma, straggler=strag,
-                                      shared=shared)
+                                      shared=shared, **variant)
                 ms = time_layer(lay, steps, warmup, torch)
                 graph_ms = time_graph(lay, steps, torch)
                 if mode == "nodrop":
@@ -198,7 +203,7 @@ def run_table(args):
                 nbar = N * cfg.k / cfg.E
                 m = cfg.E // cfg.D
                 row = {
-                    "config": cfg.name, "N": N, "mode": mode, "gamma": gamma, "straggler_emulation": strag,
+                    "config": cfg.name, "N": N, "mode": mode + tag, "gamma": gamma, "straggler_emulation": strag,
                     "C": int(lay.C), "ms_per_layer": ms, "ms_per_layer_graph": graph_ms, "tokens_per_s": N / (ms * 1e-3),
                     "speedup_vs_nodrop": nodrop_ms[strag] / ms,
                     "max_load_over_mean": float(load.max() / nbar), "max_kept_over_mean": float(kept.max() / nbar),
@@ -212,7 +217,7 @@ def run_table(args):
                         print("| N | mode | γ | strag | C | A | A/(N·k) | max load | max kept | max dev | ms/layer | as one graph "
                               "| tokens/s | speedup |\n|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
                     print("| %d | %s | %s | %s | %d | %d | %.2f | %.2f | %.2f | %.2f | %.3f | %.3f | %.2e | %.2f |" % (
-                        N, mode, "∞" if gamma is None else gamma, "on" if strag else "off", row["C"], A,
+                        N, mode + tag, "∞" if gamma is None else gamma, "on" if strag else "off", row["C"], A,
                         row["kept_over_Nk"], row["max_load_over_mean"], row["max_kept_over_mean"],
                         row["max_device_kept_over_mean"], ms, graph_ms, row["tokens_per_s"], row["speedup_vs_nodrop"]),
                         flush=True)

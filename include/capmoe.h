@@ -291,6 +291,17 @@ typedef struct {
    * [4] after the gate/up GEMM + SwiGLU, [5] after the down GEMM, [6] after the shared expert,
    * [7] after combine. */
   void** stage_events;
+  /* Variants of the drop for modes 1 and 2 (all zero / NULL = the default reading: Score metric,
+   * equal competition, no limit on experts per token).  See capmoe_drop_keys,
+   * capmoe_priority_keys, capmoe_limit_experts. */
+  int metric;                  /* capmoe_metric */
+  uint64_t metric_seed;        /* CAPMOE_METRIC_RANDOM */
+  const uint8_t* token_class;  /* [N] or NULL: 1 = token of the protected modality (modality-first dropping) */
+  int topk_first;              /* mode 2: a token's top-k pairs outrank its home-device-only pairs */
+  int max_experts;             /* > 0: every token retains at most this many experts ("w/ max") */
+  float* drop_keys;            /* scratch for the keys, [N,k] (mode 1) or [N,E] (mode 2) 32-bit words; needed
+                                  unless metric is Score, token_class is NULL and topk_first is 0 */
+  int32_t* bad;                /* device int32, needed when max_experts > 0 (see capmoe_rows_from_mask) */
 } capmoe_layer;
 #define CAPMOE_N_STAGE_EVENTS 8
 

@@ -60,6 +60,9 @@ class _Layer(ctypes.Structure):
         ("drop_ws", ctypes.c_void_p), ("drop_ws_bytes", ctypes.c_size_t),
         ("dev_status", ctypes.c_void_p),
         ("stage_events", ctypes.POINTER(ctypes.c_void_p)),
+        ("metric", ctypes.c_int), ("metric_seed", ctypes.c_uint64), ("token_class", ctypes.c_void_p),
+        ("topk_first", ctypes.c_int), ("max_experts", ctypes.c_int), ("drop_keys", ctypes.c_void_p),
+        ("bad", ctypes.c_void_p),
     ]
 
 N_STAGE_EVENTS = 8
@@ -378,7 +381,12 @@ class MoELayer:
     capmoe_layer_forward; `forward_host()` enqueues the host-buffer variant."""
 
     def __init__(self, x, w_router, bias, w_gate, w_up, w_down, k: int, D: int, mode: str, gamma: float = 1.0,
-                 straggler: bool = False, shared=None, round_mode: str = "ceil", C: Optional[int] = None):
+                 straggler: bool = False, shared=None, round_mode: str = "ceil", C: Optional[int] = None,
+                 metric: str = "score", seed: int = 0, token_class=None, topk_first: bool = False,
+                 max_experts: int = 0):
+        """Variants of the drop (token_drop / expanded_drop modes): `metric` ranks candidates by Score, Order,
+        Reverse Order or Random; `token_class` (uint8 [N], 1 = protected modality) drops the other modality
+        first; `topk_first` lets the expansion only fill spare capacity; `max_experts` > 0 is 'w/ max'."""
         dev = x.device
         N, d = x.shape
         E, F, _ = w_gate.shape
@@ -430,7 +438,19 @@ class MoELayer:
             t["hs_ws"] = torch.empty((N, F_shared), **act)
             t["y_shared"] = torch.empty((N, d), **act)
             t["one_segment"] = torch.tensor([0, N], **i32)
+        keyed = metric != "score" or token_class is not None or (topk_first and mode == "expanded_drop")
+        if keyed or max_experts > 0:
+            if mode not in ("token_drop", "expanded_drop"):
+                raise ValueError("drop variants apply to the token_drop and expanded_drop modes")
+        if keyed:
+            t["drop_keys"] = torch.empty((N, E if expanded else k), **f32)
+        if token_class is not None:
+            assert token_class.dtype == torch.uint8 and token_class.shape == (N,)
+            t["token_class"] = token_class
+        if max_experts > 0:
+            t["bad"] = torch.zeros((1,), **i32)
         L = self.c = _Layer()
+        L.metric, L.metric_seed, L.topk_first, L.max_experts = METRICS[metric], seed, int(bool(topk_first)), max_experts
         L.N, L.d, L.E, L.k, L.F, L.D, L.dtype = N, d, E, k, F, D, _dt(x)
         L.mode, L.C, L.straggler = MODES[mode], C, int(bool(straggler))
         L.F_shared, L.A_max = F_shared, A_max

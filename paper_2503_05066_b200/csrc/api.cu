@@ -159,24 +159,52 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   int slots, Dp;
   if (L->mode >= 3) {                     // device-level capacity: L->C is the per-device bound
     if (L->D < 1 || L->E % L->D != 0) return CAPMOE_EINVAL;
+    if (L->metric != CAPMOE_METRIC_SCORE || L->token_class || L->topk_first || L->max_experts > 0)
+      return CAPMOE_EUNSUPPORTED;         // the variants are defined for the per-expert capacity
     const int expanded = L->mode == 4;
     rc = capmoe_device_drop(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, expanded, nullptr, L->keep_mask,
                             L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream);
     slots = expanded ? L->k + L->E / L->D : L->k;
     Dp = expanded ? L->D : 0;
-  } else if (L->mode == 2) {
-    if (L->D < 1 || L->E % L->D != 0) return CAPMOE_EINVAL;
-    rc = capmoe_expanded_drop(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, nullptr, L->keep_mask,
-                              L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes,
-                              stream);
-    slots = L->k + L->E / L->D;
-    Dp = L->D;
   } else {
-    rc = capmoe_token_drop(L->topk_score, L->topk_idx, L->N, L->E, L->k, L->mode == 0 ? L->N : L->C,
-                           L->keep_mask, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes,
-                           stream);
-    slots = L->k;
-    Dp = 0;
+    // drop keys: the scores themselves, or a metric / priority class worked into 32-bit keys
+    const bool expanded = L->mode == 2;
+    if (expanded && (L->D < 1 || L->E % L->D != 0)) return CAPMOE_EINVAL;
+    const bool keyed = L->mode != 0 && (L->metric != CAPMOE_METRIC_SCORE || L->token_class || (expanded && L->topk_first));
+    const float* sel = expanded ? L->scores : L->topk_score;
+    if (keyed) {
+      if (!L->drop_keys) return CAPMOE_EINVAL;
+      const int cols = expanded ? L->E : L->k;
+      const int32_t* idx = expanded ? nullptr : L->topk_idx;
+      uint32_t* keys = reinterpret_cast<uint32_t*>(L->drop_keys);
+      rc = capmoe_drop_keys(L->metric, L->metric_seed, sel, idx, L->N, cols, L->E, keys, stream);
+      if (rc != CAPMOE_OK) return rc;
+      if (L->token_class || (expanded && L->topk_first)) {
+        rc = capmoe_priority_keys(keys, idx, L->N, cols, L->E, L->metric == CAPMOE_METRIC_SCORE, L->token_class,
+                                  (expanded && L->topk_first) ? L->topk_idx : nullptr, L->k, keys, stream);
+        if (rc != CAPMOE_OK) return rc;
+      }
+      sel = L->drop_keys;
+    }
+    if (expanded) {
+      rc = capmoe_expanded_drop(sel, L->topk_idx, L->N, L->E, L->k, L->C, L->D, nullptr, L->keep_mask, L->cand,
+                                L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream);
+      slots = L->k + L->E / L->D;
+      Dp = L->D;
+    } else {
+      rc = capmoe_token_drop(sel, L->topk_idx, L->N, L->E, L->k, L->mode == 0 ? L->N : L->C, L->keep_mask,
+                             L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream);
+      slots = L->k;
+      Dp = 0;
+    }
+    if (rc == CAPMOE_OK && L->mode != 0 && L->max_experts > 0) {        // "w/ max": prune, then renumber the rows
+      if (!L->bad) return CAPMOE_EINVAL;
+      rc = capmoe_limit_experts(L->scores, L->N, L->E, L->max_experts, L->keep_mask, stream);
+      if (rc != CAPMOE_OK) return rc;
+      rc = capmoe_rows_from_mask(L->keep_mask, L->topk_idx, L->N, L->E, L->k, slots, expanded ? L->D : 1, nullptr,
+                                 L->kept, L->expert_offsets, L->slot_row, L->bad, L->drop_ws, L->drop_ws_bytes,
+                                 stream);
+    }
   }
   if (rc != CAPMOE_OK) return rc;
   if ((rc = mark(2)) != CAPMOE_OK) return rc;

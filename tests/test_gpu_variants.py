@@ -169,3 +169,64 @@ def test_layer_from_stage_calls(cm, variant):
     y_ref = oracle.layer_tokens(to_np(inp.x), tokens, scores, idx, ref_rows, D, to_np(inp.w_gate), to_np(inp.w_up),
                                 to_np(inp.w_down), cfg.dtype)
     assert rel_err(as_f64(y)[tokens], y_ref) <= TOL[cfg.dtype]
+
+
+@pytest.mark.parametrize("mode,kw", [
+    ("token_drop", dict(metric="order")),
+    ("token_drop", dict(metric="random", seed=11)),
+    ("token_drop", dict(image_first=True)),
+    ("expanded_drop", dict(topk_first=True)),
+    ("expanded_drop", dict(image_first=True, topk_first=True)),
+    ("expanded_drop", dict(max_experts=4)),
+    ("expanded_drop", dict(metric="reverse_order", max_experts=2)),
+])
+def test_layer_forward_with_variants(cm, mode, kw):
+    """The same variants selected through the layer struct: one capmoe_layer_forward call."""
+    cfg = synth.CONFIGS["olmoe"].with_(N=1500, d=256, F=192, E=16, k=4, D=4)
+    inp = synth.make_layer_inputs(cfg)
+    g = {n: getattr(inp, n).cuda() for n in ("x", "w_router", "bias", "w_gate", "w_up", "w_down")}
+    N, E, k, D, m = cfg.N, cfg.E, cfg.k, cfg.D, cfg.E // cfg.D
+    kw = dict(kw)
+    cls = None
+    if kw.pop("image_first", False):
+        cls = ((np.arange(N) % 5) < 2).astype(np.uint8)
+        kw["token_class"] = dev(cls)
+    layer = cm.MoELayer(g["x"], g["w_router"], g["bias"], g["w_gate"], g["w_up"], g["w_down"], k, D, mode, gamma=1.0,
+                        **kw)
+    y = layer.forward()
+    torch.cuda.synchronize()
+    layer.check_device_status()
+    scores, idx = layer.t["scores"].cpu().numpy(), layer.t["topk_idx"].cpu().numpy()
+    expanded = mode == "expanded_drop"
+    metric, seed = kw.get("metric", "score"), kw.get("seed", 0)
+    keys = oracle.drop_keys(metric, seed, scores, None, E)
+    if cls is not None or kw.get("topk_first"):
+        keys = oracle.priority_keys(keys, None, E, metric == "score", token_class=cls,
+                                    topk_idx=idx if (expanded and kw.get("topk_first")) else None)
+    ref = oracle.drop_keyed(keys, idx, layer.C, D, expanded)
+    rows, mask = ref["slot_row"], ref["keep_mask"]
+    if kw.get("max_experts", 0) > 0:
+        mask = oracle.limit_experts(scores, mask, kw["max_experts"])
+        rows = oracle.rows_from_mask(mask, idx, E, k + (m if expanded else 0), D)["slot_row"]
+        assert int(layer.t["bad"].item()) == 0
+    assert np.array_equal(host_mask(layer.t["keep_mask"]), mask)
+    assert np.array_equal(layer.t["slot_row"].cpu().numpy(), rows)
+    tokens = np.arange(0, N, 5, dtype=np.int32)
+    y_ref = oracle.layer_tokens(to_np(inp.x), tokens, scores, idx, rows, D if expanded else 0, to_np(inp.w_gate),
+                                to_np(inp.w_up), to_np(inp.w_down), cfg.dtype)
+    assert rel_err(as_f64(y)[tokens], y_ref) <= TOL[cfg.dtype]
+
+
+def test_layer_variants_are_refused_for_device_level_capacity(cm):
+    cfg = synth.CONFIGS["tiny_f32"]
+    inp = synth.make_layer_inputs(cfg)
+    g = {n: getattr(inp, n).cuda() for n in ("x", "w_router", "bias", "w_gate", "w_up", "w_down")}
+    with pytest.raises(ValueError):
+        cm.MoELayer(g["x"], g["w_router"], g["bias"], g["w_gate"], g["w_up"], g["w_down"], cfg.k, cfg.D,
+                    "device_token_drop", metric="order")
+    layer = cm.MoELayer(g["x"], g["w_router"], g["bias"], g["w_gate"], g["w_up"], g["w_down"], cfg.k, cfg.D,
+                        "device_token_drop")
+    layer.c.metric = cm.METRICS["order"]                   # bypass the binding's own check
+    with pytest.raises(cm.CapmoeError) as e:
+        layer.forward()
+    assert e.value.status == cm.EUNSUPPORTED
