@@ -406,8 +406,14 @@ def main():
         # the workloads that were captured
         "traffic": NCU_TRAFFIC_GATE_UP.get((cfg.name, cfg.N, cfg.F, args.mode, args.gamma)),
         "algorithmic_bytes": (2 * cfg.E * cfg.F * cfg.d + A * cfg.d + A * cfg.F) * elt,
+        # the same launch against the HBM roofline (it is the binding one when few rows are kept per
+        # expert and the weights are streamed for little work): algorithmic bytes / time / measured copy bandwidth
+        "hbm_frac": ((2 * cfg.E * cfg.F * cfg.d + A * cfg.d + A * cfg.F) * elt / t1 / 1e9 / peaks["hbm_gbs"])
+        if t1 > 0 else None,
         "down_gemm": {"achieved": gemm2_flops / t2 / 1e12 if t2 > 0 else None,
-                      "frac": (gemm2_flops / t2 / 1e12 / peak_tf) if (t2 > 0 and peak_tf) else None},
+                      "frac": (gemm2_flops / t2 / 1e12 / peak_tf) if (t2 > 0 and peak_tf) else None,
+                      "hbm_frac": ((cfg.E * cfg.F * cfg.d + A * cfg.d + A * cfg.F) * elt / t2 / 1e9 / peaks["hbm_gbs"])
+                      if t2 > 0 else None},
     }
     # HBM-bound stages: algorithmic bytes over stage time
     n_kept_tok = int((layer.t["keep_mask"] != 0).any(dim=1).sum().item())
