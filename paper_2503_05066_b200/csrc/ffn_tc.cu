@@ -1,22 +1,28 @@
 // Stage 5, tensor-core path: grouped SwiGLU expert FFN in bf16 on tcgen05 (5th-generation
-// tensor cores) with TMA-fed shared-memory tiles and fp32 accumulators in tensor memory.
+// tensor cores) with TMA-fed shared-memory tiles and fp32 accumulators in tensor memory; the
+// router (stage 1) for bf16 inputs with more than 16 experts runs on the same pipeline.
 //
-// Two persistent, warp-specialised kernels per layer:
+// Two persistent, warp-specialised launches per layer:
 //   GEMM1  H[r, f]  = silu(x_perm[r,:] . W_g[e,f,:]) * (x_perm[r,:] . W_u[e,f,:])
 //   GEMM2  y_perm[r, j] = H[r,:] . W_d[e,j,:]
 // Both operands of both GEMMs are K-major (row-major activations, [out,in] weights), so every
 // tile is loaded by TMA with the 128-byte swizzle and consumed by tcgen05.mma straight from
-// shared memory.  One CTA per SM:
-//   warp 0      TMA producer (one lane): ring of STAGES {A 128x64, B 256x64} bf16 tiles
-//   warp 1      MMA issuer (one lane): 128 x 256 x 16 tcgen05.mma, accumulators ping-pong
+// shared memory.  k_ffn_tc, one CTA per SM:
+//   warp 0      TMA producer (one elected lane): ring of STAGES {A 128x64, B 256x64} bf16 tiles
+//   warp 1      MMA issuer (one elected lane): 128 x 256 x 16 tcgen05.mma, accumulators ping-pong
 //               between two 256-column halves of the CTA's 512 TMEM columns
 //   warps 2-9   epilogue: tcgen05.ld the finished accumulator, SwiGLU / convert, 16-byte stores,
 //               overlapping the next tile's MMAs
 // GEMM1 puts 128 gate rows and 128 up rows of the same output columns into one 256-row B tile,
-// so one MMA yields both halves of the SwiGLU pair.  Tiles are enumerated on the device from
-// expert_offsets (no host synchronisation); within an expert the row-block index runs fastest
-// so that concurrently running CTAs share weight tiles through L2.  In straggler-emulation mode
-// the CTAs are split into D equal groups and group g only serves the experts of virtual device g.
+// so one MMA yields both halves of the SwiGLU pair.  k_ffn_tc2 is the same pipeline on CTA pairs
+// (cta_group::2, 256 x 256 tiles, each CTA loads half of B) and serves long expert segments.
+// Tiles are enumerated on the device from expert_offsets (no host synchronisation); within an
+// expert the row-block index runs fastest so that concurrently running CTAs share weight tiles
+// through L2.  With a status block from the caller the CTAs take their tiles from a device counter
+// (TileQueue below), else each walks a fixed list.  In straggler-emulation mode the CTAs are split
+// into D equal groups and group g only serves the experts of virtual device g.
+// MODE_ROUTER / MODE_ROUTER_FUSED reuse k_ffn_tc for logits = x . W_r^T + bias, the fused form with
+// softmax, top-k and the load histogram in a 16-warp epilogue.
 // Every mbarrier wait is bounded; on expiry the CTA raises a flag, all roles drain and the
 // kernel reports CAPMOE_ETIMEOUT through dev_status.
 #include <cuda.h>
