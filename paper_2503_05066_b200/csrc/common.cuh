@@ -25,6 +25,29 @@ __device__ __forceinline__ int home_group(int64_t t, int64_t N, int D, const int
   return token_group ? token_group[t] : (int)((t * (int64_t)D) / N);
 }
 
+// Kernels that form a dependent chain on one stream are launched with programmatic stream
+// serialisation: the launch of the next kernel is processed while its predecessor still runs, and
+// its threads wait in wait_for_previous_kernel(), before touching memory, until the predecessor has
+// finished and its writes are visible.  That removes most of the gap (about 3 us) between two
+// dependent launches.  Without the launch attribute the wait is a no-op.
+__device__ __forceinline__ void wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                                  cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <typename T> __device__ __forceinline__ T from_float(float v);

@@ -154,6 +154,7 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
          const int32_t* __restrict__ token_group, const int32_t* __restrict__ cand, DropWs ws,
          unsigned long long* __restrict__ keep_mask, int32_t* __restrict__ kept,
          int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
+  wait_for_previous_kernel();
   __shared__ int hist[RADIX_BINS];
   __shared__ uint32_t scan_sh[SEL_WARPS + 1];
   __shared__ uint32_t found[3];
@@ -326,9 +327,11 @@ int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, 
       topk_idx, N, E, k, D, token_group, cand, (unsigned long long*)keep_mask, slot_row);
   int rc = check_launch();
   if (rc != CAPMOE_OK) return rc;
-  k_select<EXPANDED><<<E, SEL_THREADS, 0, st>>>(score_src, topk_idx, N, E, k, C, D, token_group, cand, ws,
-                                                 (unsigned long long*)keep_mask, kept, expert_offsets, slot_row);
-  return check_launch();
+  rc = note_cuda(launch_chained(k_select<EXPANDED>, (unsigned)E, SEL_THREADS, 0, st, score_src, topk_idx, N, E, k, C, D,
+                                token_group, (const int32_t*)cand, ws, (unsigned long long*)keep_mask, kept,
+                                expert_offsets, slot_row));
+  count_launch(1);
+  return rc;
 }
 
 int validate(int64_t N, int E, int k, int64_t C) {

@@ -41,6 +41,7 @@ constexpr int MAX_SEG = 256;
 
 struct Level { int shift, bits; };
 
+
 struct SegState {                    // one per segment, in global memory
   unsigned long long prefix;         // key bits fixed so far (tau once done)
   uint32_t rank;                     // how many keys of the current bin are still to be kept
@@ -91,6 +92,7 @@ __device__ __forceinline__ bool pair_of(const PArgs& a, int64_t t, int s, const 
 
 __global__ void __launch_bounds__(PAIR_THREADS)
 pk_hist(PArgs a, PWs w, int level, Level lv, int first_level_counts_cand) {
+  wait_for_previous_kernel();
   __shared__ int cand_s[MAX_SEG];
   const int tid = threadIdx.x;
   if (level > 0 && __ldcg(&w.active[level - 1]) == 0u) return;       // every segment already has its tau
@@ -127,6 +129,7 @@ pk_hist(PArgs a, PWs w, int level, Level lv, int first_level_counts_cand) {
 // prefix, clear the counters.  Thread i owns 8 consecutive bins, highest bins first.
 __global__ void __launch_bounds__(CHUNK)
 pk_find(PWs w, unsigned long long C_seg, int level, Level lv, int n_levels) {
+  wait_for_previous_kernel();
   __shared__ uint32_t wtot[CHUNK / 32 + 1];
   __shared__ uint32_t res[3];
   const int sg = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -200,6 +203,7 @@ pk_find(PWs w, unsigned long long C_seg, int level, Level lv, int n_levels) {
 
 __global__ void __launch_bounds__(PAIR_THREADS)
 pk_count(PArgs a, PWs w) {
+  wait_for_previous_kernel();
   __shared__ int cnt_s[MAX_SEG];
   const int tid = threadIdx.x;
   for (int i = tid; i < a.E; i += PAIR_THREADS) cnt_s[i] = 0;
@@ -222,6 +226,7 @@ pk_count(PArgs a, PWs w) {
 // one CTA per expert: exclusive scan of its per-chunk counts
 __global__ void __launch_bounds__(CHUNK)
 pk_scan(PWs w, int E, int chunks, int32_t* __restrict__ kept, int32_t* __restrict__ cand_out) {
+  wait_for_previous_kernel();
   __shared__ int warp_tot[CHUNK / 32 + 1];
   const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   int running = 0;
@@ -255,6 +260,7 @@ pk_scan(PWs w, int E, int chunks, int32_t* __restrict__ kept, int32_t* __restric
 __global__ void __launch_bounds__(PAIR_THREADS)
 pk_place(PArgs a, PWs w, const int32_t* __restrict__ kept, unsigned long long* __restrict__ keep_mask,
          int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
+  wait_for_previous_kernel();
   __shared__ int off[MAX_SEG + 1];
   __shared__ uint32_t bitmap[MAX_SEG][CHUNK / 32];
   __shared__ unsigned long long mask_s[CHUNK][4];               // keep mask of the chunk's tokens (E <= 256)
@@ -382,17 +388,21 @@ int drop_parallel(const float* scores, const float* topk_score, const int32_t* t
   const unsigned chunks = (unsigned)ceil_div(N, CHUNK);
   int rc;
   for (int l = 0; l < nl; ++l) {
-    pk_hist<<<chunks, PAIR_THREADS, 0, st>>>(a, w, l, lv[l], l == 0 ? 1 : 0);
-    if ((rc = check_launch()) != CAPMOE_OK) return rc;
-    pk_find<<<S, CHUNK, 0, st>>>(w, a.C_seg, l, lv[l], nl);
-    if ((rc = check_launch()) != CAPMOE_OK) return rc;
+    if ((rc = note_cuda(launch_chained(pk_hist, chunks, PAIR_THREADS, 0, st, a, w, l, lv[l], l == 0 ? 1 : 0))) != CAPMOE_OK)
+      return rc;
+    count_launch(1);
+    if ((rc = note_cuda(launch_chained(pk_find, (unsigned)S, CHUNK, 0, st, w, a.C_seg, l, lv[l], nl))) != CAPMOE_OK) return rc;
+    count_launch(1);
   }
-  pk_count<<<chunks, PAIR_THREADS, 0, st>>>(a, w);
-  if ((rc = check_launch()) != CAPMOE_OK) return rc;
-  pk_scan<<<E, CHUNK, 0, st>>>(w, E, (int)chunks, kept, cand_out);
-  if ((rc = check_launch()) != CAPMOE_OK) return rc;
-  pk_place<<<chunks, PAIR_THREADS, 0, st>>>(a, w, kept, (unsigned long long*)keep_mask, expert_offsets, slot_row);
-  return check_launch();
+  if ((rc = note_cuda(launch_chained(pk_count, chunks, PAIR_THREADS, 0, st, a, w))) != CAPMOE_OK) return rc;
+  count_launch(1);
+  if ((rc = note_cuda(launch_chained(pk_scan, (unsigned)E, CHUNK, 0, st, w, E, (int)chunks, kept, cand_out))) != CAPMOE_OK)
+    return rc;
+  count_launch(1);
+  rc = note_cuda(launch_chained(pk_place, chunks, PAIR_THREADS, 0, st, a, w, (const int32_t*)kept,
+                                (unsigned long long*)keep_mask, expert_offsets, slot_row));
+  count_launch(1);
+  return rc;
 }
 
 }  // namespace capmoe

@@ -307,6 +307,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
   constexpr bool ROUTER = MODE == MODE_ROUTER || MODE == MODE_ROUTER_FUSED;
   constexpr bool FUSED = MODE == MODE_ROUTER_FUSED;
+  wait_for_previous_kernel();
   constexpr int N_TILE = SWIGLU ? 128 : 256;
   __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(out_ptr);
   const uint32_t idesc = make_idesc(n_mma);
@@ -758,6 +759,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
   constexpr int N_TILE = SWIGLU ? 128 : 256;
   constexpr int BM2 = 2 * BM;                                   // rows of a pair's tile
+  wait_for_previous_kernel();
   const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BNB >> 3) << 17) |
                          ((uint32_t)(BM2 >> 4) << 24);          // M = 256, N = 256
   extern __shared__ uint8_t smem_raw[];
@@ -1093,11 +1095,13 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     cfg.blockDim = dim3(TC_THREADS);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see wait_for_previous_kernel()
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_GATE_UP>, a1, bg, bu, expert_offsets, E, d, F,
                              (__nv_bfloat16*)h_ws, D_straggler, dev_status, sched1);
     count_launch(1);
@@ -1113,16 +1117,17 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     if (grid < D_straggler) return CAPMOE_EUNSUPPORTED;
     grid = (grid / D_straggler) * D_straggler;          // equal share of SMs per virtual device
   }
-  k_ffn_tc<MODE_GATE_UP><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a1, bg, bu, expert_offsets, E, d, F, h_ws,
-                                                              D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES,
-                                                              RouterFused{}, sched1);
-  int rc = check_launch();
+  int rc = note_cuda(launch_chained(k_ffn_tc<MODE_GATE_UP, 32>, (unsigned)grid, TC_THREADS, SMEM_BYTES, st, a1, bg, bu,
+                                    expert_offsets, E, d, F, h_ws, D_straggler, dev_status, BNB, 0,
+                                    (const float*)nullptr, BM, STAGES, STAGE_BYTES, RouterFused{}, sched1));
+  count_launch(1);
   if (rc != CAPMOE_OK) return rc;
   if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
-  k_ffn_tc<MODE_DOWN><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a2, bd, bd, expert_offsets, E, F, d, y_perm,
-                                                           D_straggler, dev_status, BNB, 0, nullptr, BM, STAGES, STAGE_BYTES,
-                                                              RouterFused{}, sched2);
-  return check_launch();
+  rc = note_cuda(launch_chained(k_ffn_tc<MODE_DOWN, 32>, (unsigned)grid, TC_THREADS, SMEM_BYTES, st, a2, bd, bd,
+                                expert_offsets, E, F, d, y_perm, D_straggler, dev_status, BNB, 0,
+                                (const float*)nullptr, BM, STAGES, STAGE_BYTES, RouterFused{}, sched2));
+  count_launch(1);
+  return rc;
 }
 
 // Router on the same pipeline: logits[N,E] = x[N,d] . w_router[E,d]^T + bias in fp32 and, when

@@ -18,6 +18,7 @@ k_permute(const uint4* __restrict__ x, int64_t N, int row_vecs /* 16-byte vector
           int k, int slots, int D, const float* __restrict__ scores, const int32_t* __restrict__ topk_idx,
           const int32_t* __restrict__ token_group, const int32_t* __restrict__ slot_row,
           uint4* __restrict__ x_perm, int32_t* __restrict__ perm_token, float* __restrict__ perm_weight) {
+  wait_for_previous_kernel();
   const int lane = threadIdx.x & 31;
   const int64_t unit = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
   const int64_t t = unit / chunks;
@@ -110,6 +111,7 @@ __global__ void __launch_bounds__(PC_WARPS * 32, 4)
 k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row,
           const float* __restrict__ perm_weight, int64_t N, int row_vecs, int chunks, int slots,
           const uint4* __restrict__ y_shared, uint4* __restrict__ y) {
+  wait_for_previous_kernel();
   constexpr int NV = Vec16<T>::n;
   const int lane = threadIdx.x & 31;
   const int64_t unit = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
@@ -178,10 +180,11 @@ extern "C" int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int
   const int chunks = (row_vecs + CHUNK_VECS - 1) / CHUNK_VECS;
   const int64_t blocks = ceil_div(N * chunks, PC_WARPS);
   if (blocks > 0x7fffffff) return CAPMOE_EUNSUPPORTED;
-  k_permute<<<(unsigned)blocks, PC_WARPS * 32, 0, as_stream(stream)>>>(
-      (const uint4*)x, N, row_vecs, chunks, E, k, slots, D, scores, topk_idx, token_group, slot_row,
-      (uint4*)x_perm, perm_token, perm_weight);
-  return check_launch();
+  const int rc = note_cuda(launch_chained(k_permute, (unsigned)blocks, PC_WARPS * 32, 0, as_stream(stream),
+                                          (const uint4*)x, N, row_vecs, chunks, E, k, slots, D, scores, topk_idx,
+                                          token_group, slot_row, (uint4*)x_perm, perm_token, perm_weight));
+  count_launch(1);
+  return rc;
 }
 
 extern "C" int capmoe_combine(const void* y_perm, const int32_t* slot_row, const float* perm_weight, int64_t N,
@@ -198,12 +201,13 @@ extern "C" int capmoe_combine(const void* y_perm, const int32_t* slot_row, const
   const int64_t blocks = ceil_div(N * chunks, PC_WARPS);
   if (blocks > 0x7fffffff) return CAPMOE_EUNSUPPORTED;
   cudaStream_t st = as_stream(stream);
+  cudaError_t err;
   if (dtype == CAPMOE_F32)
-    k_combine<float><<<(unsigned)blocks, PC_WARPS * 32, 0, st>>>((const uint4*)y_perm, slot_row, perm_weight, N,
-                                                                row_vecs, chunks, slots, (const uint4*)y_shared,
-                                                                (uint4*)y);
+    err = launch_chained(k_combine<float>, (unsigned)blocks, PC_WARPS * 32, 0, st, (const uint4*)y_perm, slot_row,
+                         perm_weight, N, row_vecs, chunks, slots, (const uint4*)y_shared, (uint4*)y);
   else
-    k_combine<__nv_bfloat16><<<(unsigned)blocks, PC_WARPS * 32, 0, st>>>(
-        (const uint4*)y_perm, slot_row, perm_weight, N, row_vecs, chunks, slots, (const uint4*)y_shared, (uint4*)y);
-  return check_launch();
+    err = launch_chained(k_combine<__nv_bfloat16>, (unsigned)blocks, PC_WARPS * 32, 0, st, (const uint4*)y_perm,
+                         slot_row, perm_weight, N, row_vecs, chunks, slots, (const uint4*)y_shared, (uint4*)y);
+  count_launch(1);
+  return note_cuda(err);
 }
