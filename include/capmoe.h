@@ -239,8 +239,10 @@ int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int slots, int
  * that overlap on the GPU need a block each.
  * bf16 with d % 64 == 0 and F % 128 == 0 runs on tcgen05 tensor cores with TMA-fed tiles;
  * everything else (fp32, odd shapes) runs a plain fp32-FMA kernel. */
-#define CAPMOE_FFN_SCHED_GROUPS 63
-#define CAPMOE_FFN_STATUS_WORDS (1 + 2 * CAPMOE_FFN_SCHED_GROUPS + 1)   /* 128 */
+#define CAPMOE_FFN_SCHED_GROUPS 62
+#define CAPMOE_FFN_STATUS_WORDS (1 + 2 * CAPMOE_FFN_SCHED_GROUPS + 3)   /* 128: status, counters of the routed
+                                                                           experts' two GEMMs, two counters for
+                                                                           the layer's shared expert, one spare */
 int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F,
                        int dtype, const void* w_gate, const void* w_up, const void* w_down,
                        void* h_ws, void* y_perm, int64_t A_max, int D_straggler,

@@ -43,12 +43,13 @@ int ffn_simt(const void* x_perm, const int32_t* expert_offsets, int E, int d, in
 bool ffn_tc_supported(int d, int F, int dtype);
 int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
            const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
-           int32_t* dev_status, cudaEvent_t mid, cudaStream_t st);
+           int32_t* dev_status, int sched_slot, bool counters_cleared, cudaEvent_t mid, cudaStream_t st);
 int wait_probe(long long limit_cycles, int32_t* dev_status, cudaStream_t st);
 
 static int grouped_ffn_impl(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
                             const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
-                            int64_t A_max, int D_straggler, int32_t* dev_status, cudaEvent_t mid, void* stream) {
+                            int64_t A_max, int D_straggler, int32_t* dev_status, cudaEvent_t mid, void* stream,
+                            int sched_slot = 0, bool counters_cleared = false) {
   if (E < 1 || d < 1 || F < 1 || A_max < 0 || D_straggler < 0) return CAPMOE_EINVAL;
   if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
   if (D_straggler > 0 && E % D_straggler != 0) return CAPMOE_EINVAL;
@@ -61,7 +62,7 @@ static int grouped_ffn_impl(const void* x_perm, const int32_t* expert_offsets, i
     return CAPMOE_EINVAL;
   if (ffn_tc_supported(d, F, dtype))
     return ffn_tc(x_perm, expert_offsets, E, d, F, w_gate, w_up, w_down, h_ws, y_perm, A_max, D_straggler,
-                  dev_status, mid, as_stream(stream));
+                  dev_status, sched_slot, counters_cleared, mid, as_stream(stream));
   if (D_straggler > 0) return CAPMOE_EUNSUPPORTED;   // SM partitioning exists only in the tensor-core kernel
   return ffn_simt(x_perm, expert_offsets, E, d, F, dtype, w_gate, w_up, w_down, h_ws, y_perm, A_max, mid,
                   as_stream(stream));
@@ -152,6 +153,12 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   };
   int rc = mark(0);
   if (rc != CAPMOE_OK) return rc;
+  // The tile counters of all FFN launches of this forward are cleared here, away from the kernels
+  // that use them, so that no memset sits between the permute and the first GEMM.
+  if (L->dev_status) {
+    rc = note_cuda(cudaMemsetAsync(L->dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st));
+    if (rc != CAPMOE_OK) return rc;
+  }
   rc = capmoe_route(L->x, L->w_router, L->bias, nullptr, L->N, L->d, L->E, L->k, L->dtype, L->logits,
                     L->scores, L->topk_idx, L->topk_score, L->load, stream);
   if (rc != CAPMOE_OK) return rc;
@@ -214,7 +221,7 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if ((rc = mark(3)) != CAPMOE_OK) return rc;
   rc = grouped_ffn_impl(L->x_perm, L->expert_offsets, L->E, L->d, L->F, L->dtype, L->w_gate, L->w_up, L->w_down,
                         L->h_ws, L->y_perm, L->A_max, L->straggler ? L->D : 0, L->dev_status,
-                        L->stage_events ? (cudaEvent_t)L->stage_events[4] : nullptr, stream);
+                        L->stage_events ? (cudaEvent_t)L->stage_events[4] : nullptr, stream, 0, true);
   if (rc != CAPMOE_OK) return rc;
   if (L->A_max == 0 && (rc = mark(4)) != CAPMOE_OK) return rc;
   if ((rc = mark(5)) != CAPMOE_OK) return rc;
@@ -223,7 +230,7 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
     if (!L->ws_gate || !L->ws_up || !L->ws_down || !L->hs_ws || !L->y_shared || !L->one_segment)
       return CAPMOE_EINVAL;
     rc = grouped_ffn_impl(L->x, L->one_segment, 1, L->d, L->F_shared, L->dtype, L->ws_gate, L->ws_up, L->ws_down,
-                          L->hs_ws, L->y_shared, L->N, 0, L->dev_status, nullptr, stream);
+                          L->hs_ws, L->y_shared, L->N, 0, L->dev_status, nullptr, stream, 1, true);
     if (rc != CAPMOE_OK) return rc;
     y_shared = L->y_shared;
   }

@@ -1051,7 +1051,7 @@ bool ffn_tc_supported(int d, int F, int dtype) {
 
 int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
            const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
-           int32_t* dev_status, cudaEvent_t mid, cudaStream_t st) {
+           int32_t* dev_status, int sched_slot, bool counters_cleared, cudaEvent_t mid, cudaStream_t st) {
   if (E > MAX_E) return CAPMOE_EUNSUPPORTED;
   alignas(64) CUtensorMap a1, bg, bu, a2, bd;
   if (!make_map(&a1, x_perm, (uint64_t)d, (uint64_t)A_max, 0, BM) ||
@@ -1071,11 +1071,16 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
   // measured 2-5 % faster on the gate/up GEMMs of the other long-segment shapes, equal on their
   // down GEMMs and on the single-CTA kernel's ragged workloads.
   int32_t *sched1 = nullptr, *sched2 = nullptr;
-  if (dev_status && D_straggler <= CAPMOE_FFN_SCHED_GROUPS) {
-    err = cudaMemsetAsync(dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st);
-    if (err != cudaSuccess) return note_cuda(err);
+  if (dev_status && sched_slot == 0 && D_straggler <= CAPMOE_FFN_SCHED_GROUPS) {
     sched1 = dev_status + 1;
     sched2 = dev_status + 1 + CAPMOE_FFN_SCHED_GROUPS;
+  } else if (dev_status && sched_slot == 1 && D_straggler == 0) {   // a layer's shared expert: one group
+    sched1 = dev_status + 1 + 2 * CAPMOE_FFN_SCHED_GROUPS;
+    sched2 = sched1 + 1;
+  }
+  if (sched1 && !counters_cleared) {
+    err = cudaMemsetAsync(dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st);
+    if (err != cudaSuccess) return note_cuda(err);
   }
   // CTA pairs (256-row tiles) when the expert segments are long enough that the extra tail
   // padding does not matter, or are known multiples of 256 rows
