@@ -7,6 +7,8 @@
 #include "common.cuh"
 
 namespace capmoe {
+thread_local bool t_stage_counters_cleared = false;
+
 
 static std::atomic<uint64_t> g_launches{0};
 static thread_local char g_cuda_err[256] = "";
@@ -159,6 +161,16 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
     rc = note_cuda(cudaMemsetAsync(L->dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st));
     if (rc != CAPMOE_OK) return rc;
   }
+  // Likewise the load histogram and the drop stage's counters (see t_stage_counters_cleared).
+  if (!L->load || L->E < 1) return CAPMOE_EINVAL;
+  if ((rc = note_cuda(cudaMemsetAsync(L->load, 0, sizeof(int32_t) * L->E, st))) != CAPMOE_OK) return rc;
+  if ((rc = drop_clear_counters(L->mode, L->N, L->E, L->k, L->D < 1 ? 1 : L->D, L->cand, L->drop_ws, L->drop_ws_bytes,
+                                st)) != CAPMOE_OK)
+    return rc;
+  struct Cleared {                       // the flag is up only while this forward issues its stages
+    Cleared() { t_stage_counters_cleared = true; }
+    ~Cleared() { t_stage_counters_cleared = false; }
+  } cleared_scope;
   rc = capmoe_route(L->x, L->w_router, L->bias, nullptr, L->N, L->d, L->E, L->k, L->dtype, L->logits,
                     L->scores, L->topk_idx, L->topk_score, L->load, stream);
   if (rc != CAPMOE_OK) return rc;

@@ -15,6 +15,14 @@ int note_cuda(cudaError_t err);            // records the text, returns CAPMOE_E
 int check_launch();                        // cudaPeekAtLastError -> status, counts one launch
 int sm_count();                            // SMs of the current device (cached per device)
 
+// Set by capmoe_layer_forward around its stage calls once it has itself issued, at the start of
+// the forward, the small memsets those stages begin with (load histogram, drop counters): the
+// stages then skip them, and their first kernels chain onto the previous stage's last one.
+extern thread_local bool t_stage_counters_cleared;
+// The memsets of the drop stage that would run for these arguments (mode as in capmoe_layer).
+int drop_clear_counters(int mode, int64_t N, int E, int k, int D, int32_t* cand, void* ws, size_t ws_bytes,
+                        cudaStream_t st);
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t elt_size(int dtype) { return dtype == CAPMOE_F32 ? 4 : 2; }
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }

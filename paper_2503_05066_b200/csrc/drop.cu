@@ -19,6 +19,7 @@ namespace capmoe {
 
 // token-parallel select (drop_parallel.cu): large batches and device-level capacity
 size_t drop_parallel_ws_bytes(int64_t N, int E);
+int drop_parallel_clear(void* ws_ptr, int64_t N, int E, int S, cudaStream_t st);
 int drop_parallel(const float* scores, const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
                   int64_t C_seg, int D, int seg_m, int expanded, const int32_t* token_group, uint64_t* keep_mask,
                   int32_t* cand_out, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr,
@@ -70,6 +71,7 @@ __global__ void __launch_bounds__(CNT_THREADS)
 k_count_candidates(const int32_t* __restrict__ topk_idx, int64_t N, int E, int k, int D,
                    const int32_t* __restrict__ token_group, int32_t* __restrict__ cand,
                    unsigned long long* __restrict__ keep_mask, int32_t* __restrict__ slot_row) {
+  wait_for_previous_kernel();
   extern __shared__ int hist[];
   for (int i = threadIdx.x; i < E; i += CNT_THREADS) hist[i] = 0;
   __syncthreads();
@@ -322,10 +324,12 @@ int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, 
   if (ws_bytes < ws_bytes_needed(N, E, k, D, EXPANDED ? 1 : 0)) return CAPMOE_EWORKSPACE;
   DropWs ws = carve(ws_ptr, N, E, k, D, EXPANDED ? 1 : 0);
   int32_t* cand = cand_out ? cand_out : ws.cand;
-  if ((err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
-  k_count_candidates<EXPANDED><<<(unsigned)ceil_div(N, CNT_TOKENS), CNT_THREADS, sizeof(int) * E, st>>>(
-      topk_idx, N, E, k, D, token_group, cand, (unsigned long long*)keep_mask, slot_row);
-  int rc = check_launch();
+  if (!t_stage_counters_cleared && (err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess)
+    return note_cuda(err);
+  int rc = note_cuda(launch_chained(k_count_candidates<EXPANDED>, (unsigned)ceil_div(N, CNT_TOKENS), CNT_THREADS,
+                                    sizeof(int) * E, st, topk_idx, N, E, k, D, token_group, cand,
+                                    (unsigned long long*)keep_mask, slot_row));
+  count_launch(1);
   if (rc != CAPMOE_OK) return rc;
   rc = note_cuda(launch_chained(k_select<EXPANDED>, (unsigned)E, SEL_THREADS, 0, st, score_src, topk_idx, N, E, k, C, D,
                                 token_group, (const int32_t*)cand, ws, (unsigned long long*)keep_mask, kept,
@@ -353,6 +357,20 @@ extern "C" int capmoe_drop_workspace_bytes(int64_t N, int E, int k, int D, int e
   const size_t b = drop_parallel_ws_bytes(N, E);
   *bytes = a > b ? a : b;
   return CAPMOE_OK;
+}
+
+int capmoe::drop_clear_counters(int mode, int64_t N, int E, int k, int D, int32_t* cand, void* ws, size_t ws_bytes,
+                                cudaStream_t st) {
+  if (N <= 0 || !ws) return CAPMOE_OK;                        // the stage handles (and checks) these itself
+  const bool device_level = mode >= 3, expanded = mode == 2 || mode == 4;
+  const bool parallel = device_level || (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32));
+  if (parallel) {
+    if (ws_bytes < drop_parallel_ws_bytes(N, E)) return CAPMOE_EWORKSPACE;
+    return drop_parallel_clear(ws, N, E, device_level ? D : E, st);
+  }
+  if (ws_bytes < ws_bytes_needed(N, E, k, D, expanded ? 1 : 0)) return CAPMOE_EWORKSPACE;
+  int32_t* c = (expanded && cand) ? cand : carve(ws, N, E, k, D, expanded ? 1 : 0).cand;
+  return note_cuda(cudaMemsetAsync(c, 0, sizeof(int32_t) * E, st));
 }
 
 extern "C" int capmoe_token_drop(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,

@@ -353,6 +353,11 @@ size_t drop_parallel_ws_bytes(int64_t N, int E) {
          al256(sizeof(SegState) * (size_t)E) + 2 * al256(sizeof(int32_t) * (size_t)chunks * E);
 }
 
+int drop_parallel_clear(void* ws_ptr, int64_t N, int E, int S, cudaStream_t st) {
+  PWs w = carve_p(ws_ptr, N, E, S);
+  return note_cuda(cudaMemsetAsync(w.hist, 0, (size_t)((char*)w.seg - (char*)w.hist), st));
+}
+
 // C_seg: capacity of one segment (expert: C; device: C_dev).  seg_m: experts per segment.
 int drop_parallel(const float* scores, const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
                   int64_t C_seg, int D, int seg_m, int expanded, const int32_t* token_group, uint64_t* keep_mask,
@@ -382,9 +387,10 @@ int drop_parallel(const float* scores, const float* topk_score, const int32_t* t
     left -= b;
   }
   // hist, tickets and candidate counters start at zero
-  const size_t zero_bytes = (size_t)((char*)w.seg - (char*)w.hist);
-  cudaError_t err = cudaMemsetAsync(w.hist, 0, zero_bytes, st);
-  if (err != cudaSuccess) return note_cuda(err);
+  if (!t_stage_counters_cleared) {
+    const int rc0 = drop_parallel_clear(ws_ptr, N, E, S, st);
+    if (rc0 != CAPMOE_OK) return rc0;
+  }
   const unsigned chunks = (unsigned)ceil_div(N, CHUNK);
   int rc;
   for (int l = 0; l < nl; ++l) {

@@ -362,7 +362,8 @@ extern "C" int capmoe_route(const void* x, const void* w_router, const float* bi
   if (!logits_in && (!x || !w_router || !logits || d < 1)) return CAPMOE_EINVAL;
   if (N * (int64_t)E >= (int64_t)1 << 40) return CAPMOE_EUNSUPPORTED;
   cudaStream_t st = as_stream(stream);
-  cudaError_t err = cudaMemsetAsync(load, 0, sizeof(int32_t) * E, st);
+  cudaError_t err = cudaSuccess;
+  if (!t_stage_counters_cleared) err = cudaMemsetAsync(load, 0, sizeof(int32_t) * E, st);
   if (err != cudaSuccess) return note_cuda(err);
   if (N == 0) return CAPMOE_OK;
   const float* lg = logits_in;
