@@ -234,6 +234,8 @@ def _pick_config(args):
         cfg = cfg.with_(N=args.N)
     if args.F is not None:
         cfg = cfg.with_(F=args.F)
+    if args.D is not None:
+        cfg = cfg.with_(D=args.D)
     return cfg
 
 
@@ -288,6 +290,9 @@ def main():
     ap.add_argument("--config", default="mixtral")
     ap.add_argument("--N", type=int, default=None, help="override the number of tokens (sweeps, small ncu cases)")
     ap.add_argument("--F", type=int, default=None, help="override the expert FFN width (small ncu cases)")
+    ap.add_argument("--D", type=int, default=None,
+                    help="override the number of virtual expert-parallel devices (E %% D == 0), e.g. the paper's "
+                         "one or two experts per GPU for the Mixtral shape: --D 8, --D 4")
     ap.add_argument("--mode", default="expanded_drop", choices=["nodrop", "token_drop", "expanded_drop", "device_token_drop", "device_expanded_drop"])
     ap.add_argument("--gamma", type=float, default=1.0)
     ap.add_argument("--no-straggler", dest="straggler", action="store_false")
