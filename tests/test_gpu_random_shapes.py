@@ -1,0 +1,89 @@
+"""Seeded random shapes through the routing stages on the GPU against the CPU checker, bit for bit:
+sizes that are not multiples of any tile, chunk or warp size, every number of experts from 2 to
+130, both selection paths (one CTA per expert below 16384 tokens, token-parallel above) and both
+capacity levels."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_05066_b200 import synth
+from tests.test_gpu_parity import ROUTER_TOL, bias_for, cm, dev, host_mask  # noqa: F401
+from tests.util import rel_err, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def _cases(n, seed, big):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        D = int(rng.choice([1, 2, 3, 4, 5, 8]))
+        m = int(rng.integers(1, 17))
+        E = D * m
+        if E < 2 or E > 130:
+            continue
+        k = int(rng.integers(1, min(E, 8) + 1))
+        N = int(rng.integers(16384, 40000)) if big else int(rng.integers(1, 6000))
+        gamma = float(rng.choice([0.25, 0.5, 1.0, 1.0, 1.5, 3.0]))
+        q = float(rng.choice([0.0, 0.0, 0.25, 1.0]))
+        out.append((N, E, k, D, gamma, q))
+    return out
+
+
+CASES = _cases(28, 2024, False) + _cases(8, 2025, True)
+
+
+@pytest.mark.parametrize("N,E,k,D,gamma,q", CASES)
+def test_drops_on_random_shapes(cm, N, E, k, D, gamma, q):
+    lg = synth.synthetic_logits(N, E, 1000 + N, bias=bias_for(E, 0.8), quantum=q)
+    r = cm.route(None, None, None, k, logits_in=dev(lg))
+    scores, idx = r["scores"].cpu().numpy(), r["topk_idx"].cpu().numpy()
+    assert np.array_equal(scores.view(np.uint32), oracle.softmax(lg).view(np.uint32))
+    C = cm.capacity(N, E, k, gamma)
+    got, ref = cm.token_drop(r["topk_score"], r["topk_idx"], E, C), oracle.token_drop(scores, idx, C)
+    for key in ("kept", "offsets", "slot_row"):
+        assert np.array_equal(got[key].cpu().numpy(), ref[key]), ("token", key)
+    assert np.array_equal(host_mask(got["keep_mask"]), ref["keep_mask"])
+    got, ref = cm.expanded_drop(r["scores"], r["topk_idx"], C, D), oracle.expanded_drop(scores, idx, C, D)
+    for key in ("cand", "kept", "offsets", "slot_row"):
+        assert np.array_equal(got[key].cpu().numpy(), ref[key]), ("expanded", key)
+    assert np.array_equal(host_mask(got["keep_mask"]), ref["keep_mask"])
+    Cd = cm.device_capacity(N, E, k, D, gamma)
+    for expanded in (False, True):
+        got = cm.device_drop(r["scores"], r["topk_idx"], Cd, D, expanded)
+        ref = oracle.device_drop(scores, idx, Cd, D, expanded)
+        for key in ("cand", "kept", "offsets", "slot_row"):
+            assert np.array_equal(got[key].cpu().numpy(), ref[key]), ("device", expanded, key)
+        assert np.array_equal(host_mask(got["keep_mask"]), ref["keep_mask"])
+
+
+def _router_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        E = int(rng.integers(2, 131))
+        k = int(rng.integers(1, min(E, 16) + 1))
+        d = 64 * int(rng.integers(1, 9))
+        N = int(rng.integers(1, 9000))
+        out.append((N, d, E, k))
+    return out
+
+
+@pytest.mark.parametrize("N,d,E,k", _router_cases(16, 7))
+def test_router_on_random_shapes(cm, N, d, E, k):
+    g = torch.Generator().manual_seed(N * 131 + E)
+    x = torch.randn((N, d), generator=g).to(torch.bfloat16)
+    w = (torch.randn((E, d), generator=g) * (2.0 / d ** 0.5)).to(torch.bfloat16)
+    b = torch.randn((E,), generator=g) * 0.5
+    out = cm.route(dev(x), dev(w), dev(b), k)
+    torch.cuda.synchronize()
+    got_logits = out["logits"].cpu().numpy()
+    ref_logits = oracle.router_logits(to_np(x), to_np(w), b.numpy(), "bf16")
+    assert rel_err(got_logits.astype(np.float64), ref_logits.astype(np.float64)) <= ROUTER_TOL["bf16"]
+    s_ref = oracle.softmax(got_logits)
+    assert np.array_equal(out["scores"].cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    idx, val, load = oracle.topk(s_ref, k)
+    assert np.array_equal(out["topk_idx"].cpu().numpy(), idx)
+    assert np.array_equal(out["topk_score"].cpu().numpy().view(np.uint32), val.view(np.uint32))
+    assert np.array_equal(out["load"].cpu().numpy(), load)
