@@ -87,3 +87,53 @@ def test_router_on_random_shapes(cm, N, d, E, k):
     assert np.array_equal(out["topk_idx"].cpu().numpy(), idx)
     assert np.array_equal(out["topk_score"].cpu().numpy().view(np.uint32), val.view(np.uint32))
     assert np.array_equal(out["load"].cpu().numpy(), load)
+
+
+def _ffn_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        E = int(rng.integers(1, 9))
+        d = 64 * int(rng.integers(1, 7))
+        F = 64 * int(rng.integers(1, 7))
+        style = i % 4
+        if style == 0:      # ragged, some experts empty
+            rows = [int(rng.choice([0, 1, 17, 127, 128, 129, 300, 511])) for _ in range(E)]
+        elif style == 1:    # long segments: CTA pairs
+            rows = [int(rng.integers(1024, 1400)) for _ in range(E)]
+        elif style == 2:    # multiples of 256: CTA pairs with exact tiles
+            rows = [256 * int(rng.integers(1, 4)) for _ in range(E)]
+        else:               # one expert holds nearly everything
+            rows = [int(rng.integers(0, 40)) for _ in range(E)]
+            rows[int(rng.integers(0, E))] = int(rng.integers(1500, 2500))
+        D = int(rng.choice([0, 0, 1, E])) if style != 0 else 0
+        out.append((E, d, F, tuple(rows), D))
+    return out
+
+
+@pytest.mark.parametrize("E,d,F,rows,D_straggler", _ffn_cases(16, 99))
+def test_grouped_ffn_on_random_segments(cm, E, d, F, rows, D_straggler):
+    """bf16 tensor-core FFN over random expert segments against the double-precision SwiGLU of the
+    CPU checker on sampled rows; rows past the last segment stay untouched."""
+    A = int(sum(rows))
+    A_max = A + 5
+    g = torch.Generator().manual_seed(E * 1000 + d + F + A)
+    x_perm = torch.randn((A_max, d), generator=g).to(torch.bfloat16)
+    wg = (torch.randn((E, F, d), generator=g) * 0.05).to(torch.bfloat16)
+    wu = (torch.randn((E, F, d), generator=g) * 0.05).to(torch.bfloat16)
+    wd = (torch.randn((E, d, F), generator=g) * 0.05).to(torch.bfloat16)
+    offsets = np.concatenate([[0], np.cumsum(rows)]).astype(np.int32)
+    y = torch.full((A_max, d), 7.0, dtype=torch.bfloat16).cuda()
+    out = cm.grouped_ffn(dev(x_perm), dev(offsets), dev(wg), dev(wu), dev(wd), D_straggler=D_straggler, y_perm=y)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert (got[A:] == 7.0).all()                               # never written
+    if A == 0:
+        return
+    rng = np.random.default_rng(A)
+    sample = np.unique(np.concatenate([rng.integers(0, A, size=min(A, 96)), offsets[:-1][np.array(rows) > 0],
+                                       offsets[1:][np.array(rows) > 0] - 1]))
+    row_expert = (np.searchsorted(offsets, sample, side="right") - 1).astype(np.int32)
+    ref = oracle.expert_ffn(np.ascontiguousarray(to_np(x_perm)[sample]), row_expert, to_np(wg), to_np(wu), to_np(wd),
+                            "bf16")
+    assert rel_err(got[sample], ref) <= 2e-2
