@@ -704,8 +704,8 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
 // tcgen05.mma.cta_group::2 (M = 256) for both, and each CTA's tensor memory receives the 128
 // accumulator rows it loaded A for.  Per k-block a CTA now fills 32 KB of shared memory instead of
 // 48 KB for the same MMA work, which cuts L2->SM traffic by a third, and the ring is six deep.
-// No multicast loads are used; tcgen05.commit multicasts the "stage free" and "accumulator
-// ready" signals to both CTAs.
+// Every TMA load goes to the shared memory of the CTA that issued it; only the "stage free" and
+// "accumulator ready" barrier signals of tcgen05.commit reach both CTAs.
 constexpr int STAGES2 = 6;
 constexpr int HALF_B_BYTES = 128 * BK * 2;                 // 16 KB
 constexpr int STAGE2_BYTES = A_BYTES + HALF_B_BYTES;       // 32 KB per CTA
