@@ -199,3 +199,31 @@ def test_ffn_result_does_not_depend_on_how_tiles_are_handed_out(cm):
         for base, n_tiles in ((1, (A // 256) * (F // 128)), (63, (A // 256) * (d // 256))):
             assert int(status[base:base + groups].sum().item()) >= n_tiles
     assert torch.isfinite(fixed.float()).all() and float(fixed.float().abs().max()) > 0
+
+
+@pytest.mark.parametrize("name,mode,over", [
+    ("olmoe", "expanded_drop", dict(N=4096, d=512, F=256)),          # CTA pairs, tile counters, per-expert select
+    ("qwen", "device_expanded_drop", dict(N=6000, d=256, F=128)),    # token-parallel select, ragged segments
+])
+def test_two_layers_on_two_streams_do_not_disturb_each_other(cm, name, mode, over):
+    """Two instances (own buffers and status blocks, shared weights) running at the same time on two
+    streams give, step after step, the bits a lone forward gives."""
+    cfg = synth.CONFIGS[name].with_(**over)
+    g = _inputs(cfg)
+    mk = lambda: cm.MoELayer(g["x"], g["w_router"], g["bias"], g["w_gate"], g["w_up"], g["w_down"], cfg.k, cfg.D,
+                             mode, gamma=1.0)
+    a, b = mk(), mk()
+    ref = a.forward().clone()
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    for it in range(60):
+        with torch.cuda.stream(s1):
+            ya = a.forward()
+        with torch.cuda.stream(s2):
+            yb = b.forward()
+        if it % 20 == 19:
+            torch.cuda.synchronize()
+            assert torch.equal(ya, ref) and torch.equal(yb, ref), it
+    torch.cuda.synchronize()
+    a.check_device_status()
+    b.check_device_status()
