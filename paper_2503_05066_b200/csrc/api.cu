@@ -7,7 +7,6 @@
 #include "common.cuh"
 
 namespace capmoe {
-thread_local bool t_stage_counters_cleared = false;
 
 
 static std::atomic<uint64_t> g_launches{0};
@@ -161,18 +160,14 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
     rc = note_cuda(cudaMemsetAsync(L->dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st));
     if (rc != CAPMOE_OK) return rc;
   }
-  // Likewise the load histogram and the drop stage's counters (see t_stage_counters_cleared).
+  // Likewise the load histogram and the drop stage's counters; the stages are told so below.
   if (!L->load || L->E < 1) return CAPMOE_EINVAL;
   if ((rc = note_cuda(cudaMemsetAsync(L->load, 0, sizeof(int32_t) * L->E, st))) != CAPMOE_OK) return rc;
   if ((rc = drop_clear_counters(L->mode, L->N, L->E, L->k, L->D < 1 ? 1 : L->D, L->cand, L->drop_ws, L->drop_ws_bytes,
                                 st)) != CAPMOE_OK)
     return rc;
-  struct Cleared {                       // the flag is up only while this forward issues its stages
-    Cleared() { t_stage_counters_cleared = true; }
-    ~Cleared() { t_stage_counters_cleared = false; }
-  } cleared_scope;
-  rc = capmoe_route(L->x, L->w_router, L->bias, nullptr, L->N, L->d, L->E, L->k, L->dtype, L->logits,
-                    L->scores, L->topk_idx, L->topk_score, L->load, stream);
+  rc = route_impl(L->x, L->w_router, L->bias, nullptr, L->N, L->d, L->E, L->k, L->dtype, L->logits, L->scores,
+                  L->topk_idx, L->topk_score, L->load, stream, true);
   if (rc != CAPMOE_OK) return rc;
   if ((rc = mark(1)) != CAPMOE_OK) return rc;
   int slots, Dp;
@@ -181,8 +176,9 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
     if (L->metric != CAPMOE_METRIC_SCORE || L->token_class || L->topk_first || L->max_experts > 0)
       return CAPMOE_EUNSUPPORTED;         // the variants are defined for the per-expert capacity
     const int expanded = L->mode == 4;
-    rc = capmoe_device_drop(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, expanded, nullptr, L->keep_mask,
-                            L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream);
+    rc = device_drop_impl(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, expanded, nullptr, L->keep_mask,
+                          L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream,
+                          true);
     slots = expanded ? L->k + L->E / L->D : L->k;
     Dp = expanded ? L->D : 0;
   } else {
@@ -206,13 +202,13 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
       sel = L->drop_keys;
     }
     if (expanded) {
-      rc = capmoe_expanded_drop(sel, L->topk_idx, L->N, L->E, L->k, L->C, L->D, nullptr, L->keep_mask, L->cand,
-                                L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream);
+      rc = expanded_drop_impl(sel, L->topk_idx, L->N, L->E, L->k, L->C, L->D, nullptr, L->keep_mask, L->cand,
+                              L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream, true);
       slots = L->k + L->E / L->D;
       Dp = L->D;
     } else {
-      rc = capmoe_token_drop(sel, L->topk_idx, L->N, L->E, L->k, L->mode == 0 ? L->N : L->C, L->keep_mask,
-                             L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream);
+      rc = token_drop_impl(sel, L->topk_idx, L->N, L->E, L->k, L->mode == 0 ? L->N : L->C, L->keep_mask, L->kept,
+                           L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream, true);
       slots = L->k;
       Dp = 0;
     }

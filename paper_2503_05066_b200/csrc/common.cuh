@@ -15,10 +15,24 @@ int note_cuda(cudaError_t err);            // records the text, returns CAPMOE_E
 int check_launch();                        // cudaPeekAtLastError -> status, counts one launch
 int sm_count();                            // SMs of the current device (cached per device)
 
-// Set by capmoe_layer_forward around its stage calls once it has itself issued, at the start of
-// the forward, the small memsets those stages begin with (load histogram, drop counters): the
-// stages then skip them, and their first kernels chain onto the previous stage's last one.
-extern thread_local bool t_stage_counters_cleared;
+// The stages as capmoe_layer_forward calls them.  With the last argument true the caller has
+// itself issued, earlier on the stream, the small memsets the stage begins with (load histogram,
+// drop counters: see drop_clear_counters): the stage skips them, and its first kernel chains onto
+// the previous stage's last one.  Argument lists as in capmoe.h.
+int route_impl(const void* x, const void* w_router, const float* bias, const float* logits_in, int64_t N, int d, int E,
+               int k, int dtype, float* logits, float* scores, int32_t* topk_idx, float* topk_score, int32_t* load,
+               void* stream, bool load_cleared);
+int token_drop_impl(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C,
+                    uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row, void* ws,
+                    size_t ws_bytes, void* stream, bool counters_cleared);
+int expanded_drop_impl(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C, int D,
+                       const int32_t* token_group, uint64_t* keep_mask, int32_t* cand, int32_t* kept,
+                       int32_t* expert_offsets, int32_t* slot_row, void* ws, size_t ws_bytes, void* stream,
+                       bool counters_cleared);
+int device_drop_impl(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C_dev, int D,
+                     int expanded, const int32_t* token_group, uint64_t* keep_mask, int32_t* cand, int32_t* kept,
+                     int32_t* expert_offsets, int32_t* slot_row, void* ws, size_t ws_bytes, void* stream,
+                     bool counters_cleared);
 // The memsets of the drop stage that would run for these arguments (mode as in capmoe_layer).
 int drop_clear_counters(int mode, int64_t N, int E, int k, int D, int32_t* cand, void* ws, size_t ws_bytes,
                         cudaStream_t st);

@@ -23,7 +23,7 @@ int drop_parallel_clear(void* ws_ptr, int64_t N, int E, int S, cudaStream_t st);
 int drop_parallel(const float* scores, const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
                   int64_t C_seg, int D, int seg_m, int expanded, const int32_t* token_group, uint64_t* keep_mask,
                   int32_t* cand_out, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr,
-                  size_t ws_bytes, cudaStream_t st);
+                  size_t ws_bytes, cudaStream_t st, bool counters_cleared);
 
 namespace {
 
@@ -313,7 +313,8 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
 template <bool EXPANDED>
 int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C, int D,
              const int32_t* token_group, uint64_t* keep_mask, int32_t* cand_out, int32_t* kept,
-             int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr, size_t ws_bytes, cudaStream_t st) {
+             int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr, size_t ws_bytes, cudaStream_t st,
+             bool counters_cleared = false) {
   cudaError_t err;
   if (N == 0) {
     if ((err = cudaMemsetAsync(kept, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
@@ -324,7 +325,7 @@ int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, 
   if (ws_bytes < ws_bytes_needed(N, E, k, D, EXPANDED ? 1 : 0)) return CAPMOE_EWORKSPACE;
   DropWs ws = carve(ws_ptr, N, E, k, D, EXPANDED ? 1 : 0);
   int32_t* cand = cand_out ? cand_out : ws.cand;
-  if (!t_stage_counters_cleared && (err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess)
+  if (!counters_cleared && (err = cudaMemsetAsync(cand, 0, sizeof(int32_t) * E, st)) != cudaSuccess)
     return note_cuda(err);
   int rc = note_cuda(launch_chained(k_count_candidates<EXPANDED>, (unsigned)ceil_div(N, CNT_TOKENS), CNT_THREADS,
                                     sizeof(int) * E, st, topk_idx, N, E, k, D, token_group, cand,
@@ -373,9 +374,9 @@ int capmoe::drop_clear_counters(int mode, int64_t N, int E, int k, int D, int32_
   return note_cuda(cudaMemsetAsync(c, 0, sizeof(int32_t) * E, st));
 }
 
-extern "C" int capmoe_token_drop(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
+int capmoe::token_drop_impl(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
                                  int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
-                                 int32_t* slot_row, void* ws, size_t ws_bytes, void* stream) {
+                                 int32_t* slot_row, void* ws, size_t ws_bytes, void* stream, bool counters_cleared) {
   int rc = validate(N, E, k, C);
   if (rc != CAPMOE_OK) return rc;
   if (!kept || !expert_offsets) return CAPMOE_EINVAL;
@@ -383,15 +384,15 @@ extern "C" int capmoe_token_drop(const float* topk_score, const int32_t* topk_id
   if (N * (int64_t)k >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
   if (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32))
     return drop_parallel(nullptr, topk_score, topk_idx, N, E, k, C, 1, 1, 0, nullptr, keep_mask, nullptr, kept,
-                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream));
+                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream), counters_cleared);
   return run_drop<false>(topk_score, topk_idx, N, E, k, C, 1, nullptr, keep_mask, nullptr, kept,
-                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream));
+                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream), counters_cleared);
 }
 
-extern "C" int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
+int capmoe::expanded_drop_impl(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
                                     int64_t C, int D, const int32_t* token_group, uint64_t* keep_mask,
                                     int32_t* cand, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row,
-                                    void* ws, size_t ws_bytes, void* stream) {
+                                    void* ws, size_t ws_bytes, void* stream, bool counters_cleared) {
   int rc = validate(N, E, k, C);
   if (rc != CAPMOE_OK) return rc;
   if (D < 1 || E % D != 0) return CAPMOE_EINVAL;
@@ -400,15 +401,15 @@ extern "C" int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx
   if (N * (int64_t)(k + E / D) >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
   if (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32))
     return drop_parallel(scores, nullptr, topk_idx, N, E, k, C, D, 1, 1, token_group, keep_mask, cand, kept,
-                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream));
+                         expert_offsets, slot_row, ws, ws_bytes, as_stream(stream), counters_cleared);
   return run_drop<true>(scores, topk_idx, N, E, k, C, D, token_group, keep_mask, cand, kept, expert_offsets,
-                        slot_row, ws, ws_bytes, as_stream(stream));
+                        slot_row, ws, ws_bytes, as_stream(stream), counters_cleared);
 }
 
-extern "C" int capmoe_device_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
+int capmoe::device_drop_impl(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
                                   int64_t C_dev, int D, int expanded, const int32_t* token_group,
                                   uint64_t* keep_mask, int32_t* cand, int32_t* kept, int32_t* expert_offsets,
-                                  int32_t* slot_row, void* ws, size_t ws_bytes, void* stream) {
+                                  int32_t* slot_row, void* ws, size_t ws_bytes, void* stream, bool counters_cleared) {
   if (N < 0 || E < 1 || k < 1 || k > E || D < 1 || E % D != 0 || C_dev < 0) return CAPMOE_EINVAL;
   if (C_dev > N * (int64_t)(E / D)) return CAPMOE_EINVAL;
   if (E > 256 || k > 32) return CAPMOE_EUNSUPPORTED;
@@ -424,7 +425,7 @@ extern "C" int capmoe_device_drop(const float* scores, const int32_t* topk_idx, 
     return CAPMOE_OK;
   }
   return drop_parallel(scores, nullptr, topk_idx, N, E, k, C_dev, D, E / D, expanded ? 1 : 0, token_group, keep_mask,
-                       cand, kept, expert_offsets, slot_row, ws, ws_bytes, st);
+                       cand, kept, expert_offsets, slot_row, ws, ws_bytes, st, counters_cleared);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -531,4 +532,27 @@ extern "C" int capmoe_drop_keys(int metric, uint64_t seed, const float* scores, 
   k_drop_keys<<<(unsigned)ceil_div(total, 256), 256, 0, as_stream(stream)>>>(
       metric, (unsigned long long)seed, scores, idx, total, cols, E, keys);
   return check_launch();
+}
+
+extern "C" int capmoe_token_drop(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
+                                 int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
+                                 int32_t* slot_row, void* ws, size_t ws_bytes, void* stream) {
+  return token_drop_impl(topk_score, topk_idx, N, E, k, C, keep_mask, kept, expert_offsets, slot_row, ws, ws_bytes,
+                         stream, false);
+}
+
+extern "C" int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
+                                    int64_t C, int D, const int32_t* token_group, uint64_t* keep_mask,
+                                    int32_t* cand, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row,
+                                    void* ws, size_t ws_bytes, void* stream) {
+  return expanded_drop_impl(scores, topk_idx, N, E, k, C, D, token_group, keep_mask, cand, kept, expert_offsets,
+                            slot_row, ws, ws_bytes, stream, false);
+}
+
+extern "C" int capmoe_device_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
+                                  int64_t C_dev, int D, int expanded, const int32_t* token_group,
+                                  uint64_t* keep_mask, int32_t* cand, int32_t* kept, int32_t* expert_offsets,
+                                  int32_t* slot_row, void* ws, size_t ws_bytes, void* stream) {
+  return device_drop_impl(scores, topk_idx, N, E, k, C_dev, D, expanded, token_group, keep_mask, cand, kept,
+                          expert_offsets, slot_row, ws, ws_bytes, stream, false);
 }

@@ -362,7 +362,7 @@ int drop_parallel_clear(void* ws_ptr, int64_t N, int E, int S, cudaStream_t st) 
 int drop_parallel(const float* scores, const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
                   int64_t C_seg, int D, int seg_m, int expanded, const int32_t* token_group, uint64_t* keep_mask,
                   int32_t* cand_out, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr,
-                  size_t ws_bytes, cudaStream_t st) {
+                  size_t ws_bytes, cudaStream_t st, bool counters_cleared) {
   if (E > MAX_SEG) return CAPMOE_EUNSUPPORTED;
   if ((unsigned long long)N * (unsigned)E >= (1ull << 32)) return CAPMOE_EUNSUPPORTED;   // position word
   if (ws_bytes < drop_parallel_ws_bytes(N, E)) return CAPMOE_EWORKSPACE;
@@ -387,7 +387,7 @@ int drop_parallel(const float* scores, const float* topk_score, const int32_t* t
     left -= b;
   }
   // hist, tickets and candidate counters start at zero
-  if (!t_stage_counters_cleared) {
+  if (!counters_cleared) {
     const int rc0 = drop_parallel_clear(ws_ptr, N, E, S, st);
     if (rc0 != CAPMOE_OK) return rc0;
   }

@@ -352,9 +352,9 @@ int launch_router_mma(const __nv_bfloat16* x, const __nv_bfloat16* w, const floa
 
 using namespace capmoe;
 
-extern "C" int capmoe_route(const void* x, const void* w_router, const float* bias, const float* logits_in,
+int capmoe::route_impl(const void* x, const void* w_router, const float* bias, const float* logits_in,
                             int64_t N, int d, int E, int k, int dtype, float* logits, float* scores,
-                            int32_t* topk_idx, float* topk_score, int32_t* load, void* stream) {
+                            int32_t* topk_idx, float* topk_score, int32_t* load, void* stream, bool load_cleared) {
   if (N < 0 || E < 1 || k < 1 || k > E || d < 0) return CAPMOE_EINVAL;
   if (E > 256 || k > 32) return CAPMOE_EUNSUPPORTED;
   if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
@@ -363,7 +363,7 @@ extern "C" int capmoe_route(const void* x, const void* w_router, const float* bi
   if (N * (int64_t)E >= (int64_t)1 << 40) return CAPMOE_EUNSUPPORTED;
   cudaStream_t st = as_stream(stream);
   cudaError_t err = cudaSuccess;
-  if (!t_stage_counters_cleared) err = cudaMemsetAsync(load, 0, sizeof(int32_t) * E, st);
+  if (!load_cleared) err = cudaMemsetAsync(load, 0, sizeof(int32_t) * E, st);
   if (err != cudaSuccess) return note_cuda(err);
   if (N == 0) return CAPMOE_OK;
   const float* lg = logits_in;
@@ -395,4 +395,11 @@ extern "C" int capmoe_route(const void* x, const void* w_router, const float* bi
   if (epl <= 2) return launch_softmax_warp<2>(lg, N, E, k, scores, topk_idx, topk_score, load, st);
   if (epl <= 4) return launch_softmax_warp<4>(lg, N, E, k, scores, topk_idx, topk_score, load, st);
   return launch_softmax_warp<8>(lg, N, E, k, scores, topk_idx, topk_score, load, st);
+}
+
+extern "C" int capmoe_route(const void* x, const void* w_router, const float* bias, const float* logits_in,
+                            int64_t N, int d, int E, int k, int dtype, float* logits, float* scores,
+                            int32_t* topk_idx, float* topk_score, int32_t* load, void* stream) {
+  return route_impl(x, w_router, bias, logits_in, N, d, E, k, dtype, logits, scores, topk_idx, topk_score, load, stream,
+                    false);
 }
