@@ -49,7 +49,12 @@ constexpr int RF_SUBS = 4;
 constexpr int RF_THREADS = 64 + 4 * RF_SUBS * 32;
 constexpr int RF_XCH_FLOATS = RF_SUBS * 128 + 128 + 4 * RF_SUBS * 128;   // max, sum relay, top-k candidates
 constexpr int MAX_E = 256;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/ +
+// Epilogue staging: each FFN epilogue warp packs a 32-row x 32-column bf16 piece of the output into
+// 2 KB of shared memory (64-byte rows, 64-byte swizzle) and one lane hands it to TMA to store.
+constexpr int STG_WARP_BYTES = 32 * 64;
+constexpr int STG_BYTES = EPI_WARPS * STG_WARP_BYTES;      // 16 KB, right behind the operand ring
+constexpr int TAIL_OFF = STAGES * STAGE_BYTES + STG_BYTES; // barriers and tables start here
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STG_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/ +
                            2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/ + RF_XCH_FLOATS * 4;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
 
@@ -118,6 +123,51 @@ __device__ __forceinline__ bool elect_one() {
       : "=r"(pred));
   return pred != 0;
 }
+// Store of a shared-memory box through TMA (bulk async group of the issuing thread).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all but the newest 0 groups of this thread have finished READING their shared-memory source
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// makes this thread's shared-memory writes visible to the async proxy (TMA) that will read them
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// One 32 x 32 bf16 piece of the output: lane r holds row r as 16 packed words.  With all 32 rows
+// inside the segment the piece goes out as one TMA store (full 64-byte runs per row instead of 32
+// scattered 16-byte stores per instruction, which made short-K GEMMs wait on their epilogue);
+// otherwise the rows that exist are written directly.
+__device__ __forceinline__ void store_piece(const uint32_t* packed, bool full_rows, bool row_ok, uint8_t* stg,
+                                            const CUtensorMap* map_out, int col, int row0_of_warp,
+                                            __nv_bfloat16* orow_c, int cols_left) {
+  const int lane = threadIdx.x & 31;
+  if (full_rows) {
+    if (lane == 0) bulk_wait_read_all();                 // the previous piece has left the staging buffer
+    __syncwarp();
+    const uint32_t base = smem_u32(stg) + (uint32_t)lane * 64u;
+#pragma unroll
+    for (int v = 0; v < 4; ++v)
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + (uint32_t)((v ^ ((lane >> 1) & 3)) * 16)),
+                   "r"(packed[4 * v]), "r"(packed[4 * v + 1]), "r"(packed[4 * v + 2]), "r"(packed[4 * v + 3])
+                   : "memory");
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      tma_store_2d(map_out, col, row0_of_warp, smem_u32(stg));
+      bulk_commit();
+    }
+  } else if (row_ok) {
+#pragma unroll
+    for (int v = 0; v < 4; ++v)
+      if (v * 8 + 8 <= cols_left)
+        *reinterpret_cast<uint4*>(orow_c + v * 8) =
+            make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+  }
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -298,7 +348,8 @@ struct RouterFused { float* scores; int32_t* topk_idx; float* topk_score; int32_
 template <int MODE, int EPAD = 32>
 __global__ void __launch_bounds__(MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, 1)
 k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
-         const __grid_constant__ CUtensorMap map_b1, const int32_t* __restrict__ expert_offsets, int E,
+         const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_out /* FFN modes: the
+         output as 32 x 32 boxes */, const int32_t* __restrict__ expert_offsets, int E,
          int K /* reduction length */, int Nout /* output columns */, void* __restrict__ out_ptr,
          int D_straggler, int32_t* __restrict__ dev_status, int n_mma, int single_rows,
          const float* __restrict__ bias, int tile_rows /* rows per tile actually loaded (<= 128) */,
@@ -320,11 +371,11 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (tiles - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + STAGES * STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + TAIL_OFF);
   // bars[0..16) full, [16..32) empty, [32..34) tmem_full, [34..36) tmem_empty
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* offs = reinterpret_cast<int*>(gen + STAGES * STAGE_BYTES + 512);
+  int* offs = reinterpret_cast<int*>(gen + TAIL_OFF + 512);
   int* tile_start = offs + (MAX_E + 1);
   float* bias_s = reinterpret_cast<float*>(tile_start + (MAX_E + 1) + 2);   // [256], router mode only
   int* hist = tile_start + 8;                          // [<= 128] load histogram, fused router only
@@ -647,6 +698,8 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
         continue;
       }
       __nv_bfloat16* orow = out + (int64_t)(t.row0 + row_in_tile) * Nout + t.n0;
+      const bool full_rows = quarter * 32 + 32 <= t.rows;      // all 32 rows of this warp are inside the segment
+      uint8_t* stg = gen + STAGES * STAGE_BYTES + (warp - 2) * STG_WARP_BYTES;
 #pragma unroll 1
       for (int c = half * (N_TILE / 2); c < (half + 1) * (N_TILE / 2); c += 32) {
         uint32_t g[32];
@@ -671,18 +724,13 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
           for (int j = 0; j < 16; ++j)
             packed[j] = pack_bf16(__uint_as_float(g[2 * j]), __uint_as_float(g[2 * j + 1]));
         }
-        if (row_ok) {
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            if (t.n0 + c + v * 8 + 8 <= Nout)
-              *reinterpret_cast<uint4*>(orow + c + v * 8) =
-                  make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-          }
-        }
+        store_piece(packed, full_rows, row_ok, stg, &map_out, t.n0 + c, t.row0 + quarter * 32, orow + c,
+                    Nout - (t.n0 + c));
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(b));
     }
+    if (!ROUTER && lane == 0) bulk_wait_all();           // this lane's stores have landed before the CTA ends
   }
 
   // ------------------------------------------------------------ teardown
@@ -753,7 +801,8 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 template <int MODE>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
-          const __grid_constant__ CUtensorMap map_b1, const int32_t* __restrict__ expert_offsets, int E,
+          const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_out /* the output as
+          32 x 32 boxes */, const int32_t* __restrict__ expert_offsets, int E,
           int K, int Nout, __nv_bfloat16* __restrict__ out, int D_straggler, int32_t* __restrict__ dev_status,
           int32_t* __restrict__ sched /* tile counters, one per straggler group, zeroed; NULL = fixed lists */) {
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
@@ -766,10 +815,10 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (tiles - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + STAGES * STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + TAIL_OFF);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* offs = reinterpret_cast<int*>(gen + STAGES * STAGE_BYTES + 512);
+  int* offs = reinterpret_cast<int*>(gen + TAIL_OFF + 512);
   int* tile_start = offs + (MAX_E + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -939,6 +988,9 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       const int row_in_tile = (int)rank * BM + row_in_half;
       const bool row_ok = row_in_tile < t.rows;
       __nv_bfloat16* orow = out + (int64_t)(t.row0 + row_in_tile) * Nout + t.n0;
+      const int warp_row0 = (int)rank * BM + quarter * 32;     // first of this warp's 32 rows in the pair's tile
+      const bool full_rows = warp_row0 + 32 <= t.rows;
+      uint8_t* stg = gen + STAGES * STAGE_BYTES + (warp - 2) * STG_WARP_BYTES;
 #pragma unroll 1
       for (int c = half * (N_TILE / 2); c < (half + 1) * (N_TILE / 2); c += 32) {
         uint32_t g[32];
@@ -963,18 +1015,13 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           for (int j = 0; j < 16; ++j)
             packed[j] = pack_bf16(__uint_as_float(g[2 * j]), __uint_as_float(g[2 * j + 1]));
         }
-        if (row_ok) {
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            if (t.n0 + c + v * 8 + 8 <= Nout)
-              *reinterpret_cast<uint4*>(orow + c + v * 8) =
-                  make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-          }
-        }
+        store_piece(packed, full_rows, row_ok, stg, &map_out, t.n0 + c, t.row0 + warp_row0, orow + c,
+                    Nout - (t.n0 + c));
       }
       tc_fence_before();
       mbar_arrive_cluster(tempty_bar(b) & PEER_MASK);   // the leader waits for both CTAs' epilogues
     }
+    if (lane == 0) bulk_wait_all();                      // this lane's stores have landed before the CTA ends
   }
 
   // ------------------------------------------------------------ teardown
@@ -1021,6 +1068,20 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, ui
   return r == CUDA_SUCCESS;
 }
 
+// bf16 matrix [rows, cols] as 32 x 32 boxes with the 64-byte swizzle: the epilogue's TMA stores.
+bool make_store_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Exercises the bounded wait on a barrier that nothing ever signals: the wait must run out, the
 // kernel must return, and the status word must say so.  One warp, no tensor memory.
 __global__ void k_wait_probe(long long limit_cycles, int32_t* __restrict__ dev_status) {
@@ -1053,8 +1114,10 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
            const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
            int32_t* dev_status, int sched_slot, bool counters_cleared, cudaEvent_t mid, cudaStream_t st) {
   if (E > MAX_E) return CAPMOE_EUNSUPPORTED;
-  alignas(64) CUtensorMap a1, bg, bu, a2, bd;
-  if (!make_map(&a1, x_perm, (uint64_t)d, (uint64_t)A_max, 0, BM) ||
+  alignas(64) CUtensorMap a1, bg, bu, a2, bd, o1, o2;
+  if (!make_store_map(&o1, h_ws, (uint64_t)F, (uint64_t)A_max) ||
+      !make_store_map(&o2, y_perm, (uint64_t)d, (uint64_t)A_max) ||
+      !make_map(&a1, x_perm, (uint64_t)d, (uint64_t)A_max, 0, BM) ||
       !make_map(&bg, w_gate, (uint64_t)d, (uint64_t)F, (uint64_t)E, 128) ||
       !make_map(&bu, w_up, (uint64_t)d, (uint64_t)F, (uint64_t)E, 128) ||
       !make_map(&a2, h_ws, (uint64_t)F, (uint64_t)A_max, 0, BM) ||
@@ -1107,13 +1170,13 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_GATE_UP>, a1, bg, bu, expert_offsets, E, d, F,
+    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_GATE_UP>, a1, bg, bu, o1, expert_offsets, E, d, F,
                              (__nv_bfloat16*)h_ws, D_straggler, dev_status, sched1);
     count_launch(1);
     if (err != cudaSuccess) return note_cuda(err);
     int rc2;
     if (mid && (rc2 = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc2;
-    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_DOWN>, a2, bd128, bd128, expert_offsets, E, F, d,
+    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_DOWN>, a2, bd128, bd128, o2, expert_offsets, E, F, d,
                              (__nv_bfloat16*)y_perm, D_straggler, dev_status, sched2);
     count_launch(1);
     return note_cuda(err);
@@ -1122,13 +1185,13 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     if (grid < D_straggler) return CAPMOE_EUNSUPPORTED;
     grid = (grid / D_straggler) * D_straggler;          // equal share of SMs per virtual device
   }
-  int rc = note_cuda(launch_chained(k_ffn_tc<MODE_GATE_UP, 32>, (unsigned)grid, TC_THREADS, SMEM_BYTES, st, a1, bg, bu,
+  int rc = note_cuda(launch_chained(k_ffn_tc<MODE_GATE_UP, 32>, (unsigned)grid, TC_THREADS, SMEM_BYTES, st, a1, bg, bu, o1,
                                     expert_offsets, E, d, F, h_ws, D_straggler, dev_status, BNB, 0,
                                     (const float*)nullptr, BM, STAGES, STAGE_BYTES, RouterFused{}, sched1));
   count_launch(1);
   if (rc != CAPMOE_OK) return rc;
   if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
-  rc = note_cuda(launch_chained(k_ffn_tc<MODE_DOWN, 32>, (unsigned)grid, TC_THREADS, SMEM_BYTES, st, a2, bd, bd,
+  rc = note_cuda(launch_chained(k_ffn_tc<MODE_DOWN, 32>, (unsigned)grid, TC_THREADS, SMEM_BYTES, st, a2, bd, bd, o2,
                                 expert_offsets, E, F, d, y_perm, D_straggler, dev_status, BNB, 0,
                                 (const float*)nullptr, BM, STAGES, STAGE_BYTES, RouterFused{}, sched2));
   count_launch(1);
@@ -1147,8 +1210,10 @@ static int launch_router_tc(const CUtensorMap& ax, const CUtensorMap& bw, int gr
   cudaError_t err = cudaFuncSetAttribute(k_ffn_tc<MODE, EPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          SMEM_BYTES);
   if (err != cudaSuccess) return note_cuda(err);
-  k_ffn_tc<MODE, EPAD><<<grid, MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, SMEM_BYTES, st>>>(ax, bw, bw, nullptr, 1, d, E, logits, 0, nullptr, n_mma,
-                                                            (int)N, bias, tile_rows, n_stages, stage_stride, rf, nullptr);
+  // (the fourth tensor map is the FFN modes' output map: unused here)
+  k_ffn_tc<MODE, EPAD><<<grid, MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, SMEM_BYTES, st>>>(
+      ax, bw, bw, bw, nullptr, 1, d, E, logits, 0, nullptr, n_mma, (int)N, bias, tile_rows, n_stages, stage_stride, rf,
+      nullptr);
   return check_launch();
 }
 
