@@ -60,6 +60,10 @@ int capmoe_capacity(int64_t N, int E, int k, double gamma, int round, int64_t* C
  * min(E*C, N*k) for Token Drop, min(E*C, N*(k+E/D)) for Expanded Drop.  Host pointer out. */
 int capmoe_max_rows(int64_t N, int E, int k, int D, int64_t C, int expanded, int64_t* A_max);
 
+/* The same bound under device-level capacity (capmoe_device_drop with a per-device bound C_dev):
+ * min(D*C_dev, N*k) or, with the expanded candidate set, min(D*C_dev, N*(k+E/D)).  Host pointer out. */
+int capmoe_device_max_rows(int64_t N, int E, int k, int D, int64_t C_dev, int expanded, int64_t* A_max);
+
 /* Scratch needed by capmoe_token_drop (expanded = 0) / capmoe_expanded_drop (expanded = 1). */
 int capmoe_drop_workspace_bytes(int64_t N, int E, int k, int D, int expanded, size_t* bytes);
 
@@ -118,7 +122,10 @@ int capmoe_token_drop(const float* topk_score, const int32_t* topk_idx, int64_t 
  *     call outside of any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents: the
  *     call clears the part that has to start at zero itself, but two calls that overlap on the
- *     GPU (different streams, or several host threads) race on it.  Serialise them. */
+ *     GPU (different streams, or several host threads) race on it.  Serialise them.
+ *   - Whatever the batch size it runs the select with one thread block per expert, which walks
+ *     all N tokens; from a few ten thousand tokens on capmoe_token_drop, which spreads the select
+ *     over the whole GPU, is several times faster. */
 #define CAPMOE_STATIC_DROP_MAX_PAIRS (1 << 20)
 int capmoe_token_drop_static(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
                              int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
@@ -237,8 +244,10 @@ int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int slots, int
  * operand run at the same time whatever the speed of their SMs); with NULL, or more than
  * CAPMOE_FFN_SCHED_GROUPS straggler groups, every CTA walks a fixed list of tiles instead.  Calls
  * that overlap on the GPU need a block each.
- * bf16 with d % 64 == 0 and F % 128 == 0 runs on tcgen05 tensor cores with TMA-fed tiles;
- * everything else (fp32, odd shapes) runs a plain fp32-FMA kernel. */
+ * bf16 with d % 64 == 0 and F % 64 == 0 runs on tcgen05 tensor cores with TMA-fed tiles (the last
+ * 128-column block of the gate/up GEMM is half filled when F is an odd multiple of 64); everything
+ * else (fp32, odd shapes) runs a plain fp32-FMA kernel, which has no straggler emulation
+ * (D_straggler > 0 then returns CAPMOE_EUNSUPPORTED).  capmoe_ffn_uses_tensor_cores tells which. */
 #define CAPMOE_FFN_SCHED_GROUPS 62
 #define CAPMOE_FFN_STATUS_WORDS (1 + 2 * CAPMOE_FFN_SCHED_GROUPS + 3)   /* 128: status, counters of the routed
                                                                            experts' two GEMMs, two counters for
@@ -307,7 +316,12 @@ typedef struct {
 } capmoe_layer;
 #define CAPMOE_N_STAGE_EVENTS 8
 
-/* Runs the stages above in order on `stream` (route, drop, permute, FFN, [shared FFN], combine). */
+/* Runs the stages above in order on `stream` (route, drop, permute, FFN, [shared FFN], combine).
+ * Every field is checked before the first event record, memset or launch: missing pointers for the
+ * chosen mode and variants (CAPMOE_EINVAL), E % D, capacities out of range, a drop workspace below
+ * what the mode needs or A_max below the row bound of the mode (capmoe_max_rows /
+ * capmoe_device_max_rows; N*k without dropping) (CAPMOE_EWORKSPACE), straggler emulation off the
+ * tensor-core path (CAPMOE_EUNSUPPORTED).  x_perm, h_ws and y_perm must hold A_max rows. */
 int capmoe_layer_forward(const capmoe_layer* L, void* stream);
 
 /* Same, with the activations on the HOST: copies x_host [N,d] (pinned) to L->x, runs the layer,

@@ -23,7 +23,7 @@ F32, BF16 = 0, 1
 MODE_NODROP, MODE_TOKEN_DROP, MODE_EXPANDED_DROP = 0, 1, 2
 MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2, "device_token_drop": 3, "device_expanded_drop": 4}
 
-EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_drop_workspace_bytes", "capmoe_status_str",
+EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_device_max_rows", "capmoe_drop_workspace_bytes", "capmoe_status_str",
            "capmoe_last_cuda_error", "capmoe_launch_count", "capmoe_ffn_uses_tensor_cores", "capmoe_route",
            "capmoe_token_drop", "capmoe_token_drop_static", "capmoe_expanded_drop", "capmoe_device_capacity",
            "capmoe_device_drop", "capmoe_drop_keys", "capmoe_priority_keys", "capmoe_limit_experts",
@@ -127,6 +127,13 @@ def max_rows(N: int, E: int, k: int, D: int, C: int, expanded: bool) -> int:
     out = ctypes.c_int64(0)
     _check(lib().capmoe_max_rows(_i64(N), int(E), int(k), int(D), _i64(C), int(bool(expanded)),
                                  ctypes.byref(out)), "capmoe_max_rows")
+    return out.value
+
+
+def device_max_rows(N: int, E: int, k: int, D: int, C_dev: int, expanded: bool) -> int:
+    out = ctypes.c_int64(0)
+    _check(lib().capmoe_device_max_rows(_i64(N), int(E), int(k), int(D), _i64(C_dev), int(bool(expanded)),
+                                        ctypes.byref(out)), "capmoe_device_max_rows")
     return out.value
 
 
@@ -404,7 +411,7 @@ class MoELayer:
                 C = capacity(N, E, k, gamma, round_mode)
         self.C = C
         self.slots = k + m if expanded else k
-        A_max = min(D * C, N * self.slots) if device_level else max_rows(N, E, k, D, C, expanded)
+        A_max = device_max_rows(N, E, k, D, C, expanded) if device_level else max_rows(N, E, k, D, C, expanded)
         self.A_max = A_max
         W = (E + 63) // 64
         f32 = dict(device=dev, dtype=torch.float32)

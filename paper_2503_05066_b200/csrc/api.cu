@@ -115,6 +115,15 @@ extern "C" int capmoe_max_rows(int64_t N, int E, int k, int D, int64_t C, int ex
   return CAPMOE_OK;
 }
 
+extern "C" int capmoe_device_max_rows(int64_t N, int E, int k, int D, int64_t C_dev, int expanded, int64_t* A_max) {
+  if (!A_max || N < 0 || E < 1 || k < 1 || k > E || D < 1 || E % D != 0 || C_dev < 0) return CAPMOE_EINVAL;
+  const int64_t cands = N * (int64_t)(expanded ? k + E / D : k);
+  const int64_t most = N * (int64_t)(E / D);
+  const int64_t cap = (int64_t)D * (C_dev > most ? most : C_dev);
+  *A_max = cands < cap ? cands : cap;
+  return CAPMOE_OK;
+}
+
 extern "C" const char* capmoe_status_str(int status) {
   switch (status) {
     case CAPMOE_OK: return "ok";
@@ -144,9 +153,87 @@ extern "C" int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offs
                           D_straggler, dev_status, nullptr, stream);
 }
 
+namespace capmoe {
+namespace {
+
+// Rows of the permuted matrix that a forward with these settings can produce at most.
+int64_t layer_row_bound(const capmoe_layer* L, int slots) {
+  const int64_t cands = L->N * (int64_t)slots;
+  int64_t cap;
+  if (L->mode == 0) cap = cands;
+  else if (L->mode <= 2) cap = (int64_t)L->E * (L->C > L->N ? L->N : L->C);
+  else cap = (int64_t)L->D * L->C;
+  return cands < cap ? cands : cap;
+}
+
+// Every check of capmoe_layer_forward, made before the first event record, memset or launch, so
+// that a non-zero return (other than CAPMOE_ECUDA) leaves the stream untouched.
+int validate_layer(const capmoe_layer* L) {
+  if (L->mode < 0 || L->mode > 4) return CAPMOE_EINVAL;
+  if (L->N < 0 || L->d < 1 || L->E < 1 || L->k < 1 || L->k > L->E || L->F < 1 || L->A_max < 0) return CAPMOE_EINVAL;
+  if (L->dtype != CAPMOE_F32 && L->dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
+  if (L->E > 256 || L->k > 32) return CAPMOE_EUNSUPPORTED;
+  if (L->N >= ((int64_t)1 << 31) || L->N * (int64_t)L->E >= ((int64_t)1 << 40)) return CAPMOE_EUNSUPPORTED;
+  const bool expanded = L->mode == 2 || L->mode == 4, device_level = L->mode >= 3;
+  const bool needs_D = expanded || device_level || L->straggler;
+  if (needs_D && (L->D < 1 || L->E % L->D != 0)) return CAPMOE_EINVAL;
+  const int slots = expanded ? L->k + L->E / L->D : L->k;
+  if (slots > 288) return CAPMOE_EUNSUPPORTED;
+  if (L->N * (int64_t)slots >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  if (((size_t)L->d * elt_size(L->dtype)) % 16 != 0) return CAPMOE_EUNSUPPORTED;
+  if (L->mode == 1 || L->mode == 2) {
+    if (L->C < 0 || L->C > L->N) return CAPMOE_EINVAL;
+  } else if (device_level) {
+    if (L->C < 0 || L->C > L->N * (int64_t)(L->E / L->D)) return CAPMOE_EINVAL;
+  }
+  // variants of the drop
+  if (L->metric < CAPMOE_METRIC_SCORE || L->metric > CAPMOE_METRIC_RANDOM || L->max_experts < 0) return CAPMOE_EINVAL;
+  const bool variant = L->metric != CAPMOE_METRIC_SCORE || L->token_class || L->topk_first || L->max_experts > 0;
+  if (device_level && variant) return CAPMOE_EUNSUPPORTED;      // defined for the per-expert capacity
+  const bool keyed = (L->mode == 1 || L->mode == 2) &&
+                     (L->metric != CAPMOE_METRIC_SCORE || L->token_class || (L->mode == 2 && L->topk_first));
+  if (keyed && !L->drop_keys) return CAPMOE_EINVAL;
+  if (L->mode != 0 && L->max_experts > 0 && !L->bad) return CAPMOE_EINVAL;
+  // buffers
+  if (!L->logits || !L->scores || !L->topk_idx || !L->topk_score || !L->load || !L->kept || !L->expert_offsets)
+    return CAPMOE_EINVAL;
+  if ((expanded || device_level) && !L->cand) return CAPMOE_EINVAL;
+  if (L->stage_events)
+    for (int i = 0; i < CAPMOE_N_STAGE_EVENTS; ++i)
+      if (!L->stage_events[i]) return CAPMOE_EINVAL;
+  if (L->F_shared < 0) return CAPMOE_EINVAL;
+  if (L->F_shared > 0 &&
+      (!L->ws_gate || !L->ws_up || !L->ws_down || !L->hs_ws || !L->y_shared || !L->one_segment ||
+       !aligned16(L->ws_gate) || !aligned16(L->ws_up) || !aligned16(L->ws_down) || !aligned16(L->hs_ws) ||
+       !aligned16(L->y_shared)))
+    return CAPMOE_EINVAL;
+  if (L->straggler && !ffn_tc_supported(L->d, L->F, L->dtype)) return CAPMOE_EUNSUPPORTED;
+  if (L->A_max < layer_row_bound(L, slots)) return CAPMOE_EWORKSPACE;   // the permute and the FFN write by row index
+  if (L->N > 0) {
+    if (!L->x || !L->w_router || !L->keep_mask || !L->slot_row || !L->y || !L->drop_ws) return CAPMOE_EINVAL;
+    if (!aligned16(L->x) || !aligned16(L->w_router) || !aligned16(L->y)) return CAPMOE_EINVAL;
+    if (L->drop_ws_bytes < drop_ws_required(L->mode, L->N, L->E, L->k, needs_D ? L->D : 1)) return CAPMOE_EWORKSPACE;
+  }
+  if (L->A_max > 0) {
+    if (!L->x_perm || !L->perm_token || !L->perm_weight || !L->h_ws || !L->y_perm || !L->w_gate || !L->w_up ||
+        !L->w_down)
+      return CAPMOE_EINVAL;
+    if (!aligned16(L->x_perm) || !aligned16(L->h_ws) || !aligned16(L->y_perm) || !aligned16(L->w_gate) ||
+        !aligned16(L->w_up) || !aligned16(L->w_down))
+      return CAPMOE_EINVAL;
+  }
+  return CAPMOE_OK;
+}
+
+}  // namespace
+}  // namespace capmoe
+
 extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if (!L) return CAPMOE_EINVAL;
-  if (L->mode < 0 || L->mode > 4) return CAPMOE_EINVAL;
+  {
+    const int bad_args = validate_layer(L);
+    if (bad_args != CAPMOE_OK) return bad_args;
+  }
   cudaStream_t st = as_stream(stream);
   auto mark = [&](int i) -> int {
     if (!L->stage_events) return CAPMOE_OK;
@@ -161,7 +248,6 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
     if (rc != CAPMOE_OK) return rc;
   }
   // Likewise the load histogram and the drop stage's counters; the stages are told so below.
-  if (!L->load || L->E < 1) return CAPMOE_EINVAL;
   if ((rc = note_cuda(cudaMemsetAsync(L->load, 0, sizeof(int32_t) * L->E, st))) != CAPMOE_OK) return rc;
   if ((rc = drop_clear_counters(L->mode, L->N, L->E, L->k, L->D < 1 ? 1 : L->D, L->cand, L->drop_ws, L->drop_ws_bytes,
                                 st)) != CAPMOE_OK)
@@ -172,9 +258,6 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if ((rc = mark(1)) != CAPMOE_OK) return rc;
   int slots, Dp;
   if (L->mode >= 3) {                     // device-level capacity: L->C is the per-device bound
-    if (L->D < 1 || L->E % L->D != 0) return CAPMOE_EINVAL;
-    if (L->metric != CAPMOE_METRIC_SCORE || L->token_class || L->topk_first || L->max_experts > 0)
-      return CAPMOE_EUNSUPPORTED;         // the variants are defined for the per-expert capacity
     const int expanded = L->mode == 4;
     rc = device_drop_impl(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, expanded, nullptr, L->keep_mask,
                           L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream,
@@ -184,11 +267,9 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   } else {
     // drop keys: the scores themselves, or a metric / priority class worked into 32-bit keys
     const bool expanded = L->mode == 2;
-    if (expanded && (L->D < 1 || L->E % L->D != 0)) return CAPMOE_EINVAL;
     const bool keyed = L->mode != 0 && (L->metric != CAPMOE_METRIC_SCORE || L->token_class || (expanded && L->topk_first));
     const float* sel = expanded ? L->scores : L->topk_score;
     if (keyed) {
-      if (!L->drop_keys) return CAPMOE_EINVAL;
       const int cols = expanded ? L->E : L->k;
       const int32_t* idx = expanded ? nullptr : L->topk_idx;
       uint32_t* keys = reinterpret_cast<uint32_t*>(L->drop_keys);
@@ -213,7 +294,6 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
       Dp = 0;
     }
     if (rc == CAPMOE_OK && L->mode != 0 && L->max_experts > 0) {        // "w/ max": prune, then renumber the rows
-      if (!L->bad) return CAPMOE_EINVAL;
       rc = capmoe_limit_experts(L->scores, L->N, L->E, L->max_experts, L->keep_mask, stream);
       if (rc != CAPMOE_OK) return rc;
       rc = capmoe_rows_from_mask(L->keep_mask, L->topk_idx, L->N, L->E, L->k, slots, expanded ? L->D : 1, nullptr,
@@ -235,8 +315,6 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if ((rc = mark(5)) != CAPMOE_OK) return rc;
   const void* y_shared = nullptr;
   if (L->F_shared > 0) {
-    if (!L->ws_gate || !L->ws_up || !L->ws_down || !L->hs_ws || !L->y_shared || !L->one_segment)
-      return CAPMOE_EINVAL;
     rc = grouped_ffn_impl(L->x, L->one_segment, 1, L->d, L->F_shared, L->dtype, L->ws_gate, L->ws_up, L->ws_down,
                           L->hs_ws, L->y_shared, L->N, 0, L->dev_status, nullptr, stream, 1, true);
     if (rc != CAPMOE_OK) return rc;

@@ -33,6 +33,9 @@ int device_drop_impl(const float* scores, const int32_t* topk_idx, int64_t N, in
                      int expanded, const int32_t* token_group, uint64_t* keep_mask, int32_t* cand, int32_t* kept,
                      int32_t* expert_offsets, int32_t* slot_row, void* ws, size_t ws_bytes, void* stream,
                      bool counters_cleared);
+// Workspace bytes the drop stage of a layer forward in this mode will ask for (mode as in capmoe_layer).
+size_t drop_ws_required(int mode, int64_t N, int E, int k, int D);
+bool ffn_tc_supported(int d, int F, int dtype);
 // The memsets of the drop stage that would run for these arguments (mode as in capmoe_layer).
 int drop_clear_counters(int mode, int64_t N, int E, int k, int D, int32_t* cand, void* ws, size_t ws_bytes,
                         cudaStream_t st);

@@ -360,6 +360,13 @@ extern "C" int capmoe_drop_workspace_bytes(int64_t N, int E, int k, int D, int e
   return CAPMOE_OK;
 }
 
+size_t capmoe::drop_ws_required(int mode, int64_t N, int E, int k, int D) {
+  if (N <= 0) return 0;
+  const bool device_level = mode >= 3, expanded = mode == 2 || mode == 4;
+  const bool parallel = device_level || (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32));
+  return parallel ? drop_parallel_ws_bytes(N, E) : ws_bytes_needed(N, E, k, D, expanded ? 1 : 0);
+}
+
 int capmoe::drop_clear_counters(int mode, int64_t N, int E, int k, int D, int32_t* cand, void* ws, size_t ws_bytes,
                                 cudaStream_t st) {
   if (N <= 0 || !ws) return CAPMOE_OK;                        // the stage handles (and checks) these itself

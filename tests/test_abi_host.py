@@ -101,3 +101,69 @@ def test_missing_library_fails_loudly(cm, monkeypatch):
     monkeypatch.setattr(cm, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         cm.capacity(8, 4, 2, 1.0)
+
+
+def _fake_layer(cm, **over):
+    """A capmoe_layer whose every field passes validation (pointers are aligned dummies that are
+    never dereferenced on the host); `over` then breaks one field."""
+    L = cm._Layer()
+    L.N, L.d, L.E, L.k, L.F, L.D, L.dtype = 64, 64, 8, 2, 64, 2, cm.BF16
+    L.mode, L.C, L.straggler = 2, 16, 0
+    L.A_max = cm.max_rows(64, 8, 2, 2, 16, True)
+    L.drop_ws_bytes = cm.drop_workspace_bytes(64, 8, 2, 2, True)
+    for name, typ in cm._Layer._fields_:
+        if typ is ctypes.c_void_p and name not in ("ws_gate", "ws_up", "ws_down", "hs_ws", "y_shared", "one_segment",
+                                                   "token_class", "drop_keys", "bad"):
+            setattr(L, name, 4096)
+    for key, v in over.items():
+        setattr(L, key, v)
+    return L
+
+
+def test_layer_forward_checks_every_field_before_it_enqueues_anything(cm):
+    """Each broken field is reported by the host-side checks: the call returns its status without
+    an event record, memset or launch (the launch counter does not move, and on a machine without
+    a GPU no CUDA call is reached, which would show as CAPMOE_ECUDA)."""
+    lib = cm.lib()
+    cases = [
+        (dict(mode=5), cm.EINVAL), (dict(k=9), cm.EINVAL), (dict(N=-1), cm.EINVAL), (dict(dtype=3), cm.EUNSUPPORTED),
+        (dict(E=512, k=2), cm.EUNSUPPORTED),
+        (dict(D=3), cm.EINVAL),                                   # E % D != 0 (Expanded Drop needs D)
+        (dict(mode=3, D=3), cm.EINVAL), (dict(mode=1, straggler=1, D=3), cm.EINVAL),
+        (dict(C=65), cm.EINVAL), (dict(C=-1), cm.EINVAL),
+        (dict(mode=4, C=64 * 4 + 1), cm.EINVAL),                  # device capacity beyond N * E/D
+        (dict(metric=7), cm.EINVAL),
+        (dict(metric=3), cm.EINVAL),                              # keyed drop without key scratch
+        (dict(topk_first=1), cm.EINVAL), (dict(token_class=4096), cm.EINVAL),
+        (dict(max_experts=2), cm.EINVAL),                         # "w/ max" without the bad flag
+        (dict(mode=3, metric=1, drop_keys=4096), cm.EUNSUPPORTED),
+        (dict(mode=4, max_experts=1, bad=4096), cm.EUNSUPPORTED),
+        (dict(load=0), cm.EINVAL), (dict(logits=0), cm.EINVAL), (dict(cand=0), cm.EINVAL),
+        (dict(kept=0), cm.EINVAL), (dict(expert_offsets=0), cm.EINVAL),
+        (dict(x=0), cm.EINVAL), (dict(keep_mask=0), cm.EINVAL), (dict(slot_row=0), cm.EINVAL),
+        (dict(y=0), cm.EINVAL), (dict(drop_ws=0), cm.EINVAL), (dict(x=4100), cm.EINVAL),
+        (dict(x_perm=0), cm.EINVAL), (dict(h_ws=0), cm.EINVAL), (dict(w_down=0), cm.EINVAL),
+        (dict(y_perm=4104), cm.EINVAL),
+        (dict(F_shared=64), cm.EINVAL),                           # shared expert without its buffers
+        (dict(F_shared=-1), cm.EINVAL),
+        (dict(d=60), cm.EUNSUPPORTED),                            # rows not a multiple of 16 bytes
+        (dict(dtype=cm.F32, straggler=1), cm.EUNSUPPORTED),       # SM partition exists only on the tensor-core path
+        (dict(A_max=16 * 8 - 1), cm.EWORKSPACE),                  # below min(E*C, N*(k+m))
+        (dict(mode=0, A_max=64 * 2 - 1), cm.EWORKSPACE),
+        (dict(mode=3, C=40, A_max=2 * 40 - 1), cm.EWORKSPACE),
+        (dict(drop_ws_bytes=64), cm.EWORKSPACE),
+    ]
+    before = cm.launch_count()
+    for over, want in cases:
+        L = _fake_layer(cm, **over)
+        got = lib.capmoe_layer_forward(ctypes.byref(L), ctypes.c_void_p(0))
+        assert got == want, (over, got, want)
+    assert cm.launch_count() == before
+
+
+def test_device_max_rows(cm):
+    assert cm.device_max_rows(4096, 64, 8, 8, 4096, False) == 32768
+    assert cm.device_max_rows(4096, 64, 8, 8, 100, False) == 800
+    assert cm.device_max_rows(4096, 64, 8, 8, 10 ** 9, True) == 4096 * 16
+    with pytest.raises(cm.CapmoeError):
+        cm.device_max_rows(4096, 64, 8, 7, 10, False)

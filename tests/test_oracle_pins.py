@@ -80,9 +80,12 @@ def test_softmax_special_rows():
     assert np.all(s[0] == np.float32(1.0) / np.float32(8.0))
     assert s[1, 3] == 1.0 and np.all(np.delete(s[1], 3) == 0.0)
     assert np.all(s[2] == np.float32(0.125))
-    # shift invariance is exact: the max is subtracted first
-    a = synth.synthetic_logits(50, E, 9)
-    assert np.array_equal(oracle.softmax(a), oracle.softmax(a))
+    # shift invariance is exact when the shift itself is: on a 1/64 grid a + 8 is representable,
+    # l - max is then the same number for both inputs, and the scores must agree bit for bit
+    a = synth.synthetic_logits(50, E, 9, quantum=1.0 / 64.0)
+    assert np.array_equal((a + np.float32(8.0)) - np.float32(8.0), a)
+    assert np.array_equal(oracle.softmax(a + np.float32(8.0)), oracle.softmax(a))
+    assert np.array_equal(oracle.softmax(a - np.float32(16.0)), oracle.softmax(a))
     lg2 = np.array([[0.0, -1.0, -2.0, -90.0]], np.float32)
     s2 = oracle.softmax(lg2)
     ref = np.exp(np.array([0.0, -1.0, -2.0])); ref /= ref.sum()
@@ -155,39 +158,38 @@ def test_token_drop_brute_force(N, E, k, C, q):
     assert np.array_equal(r["kept"], np.minimum(load, C))
 
 
-def _dense_mask_formulation(scores, row_mask, cap):
-    """The listings' formulation: mask the score matrix, take each column's `cap` largest
-    entries, intersect with the row mask."""
-    masked = scores * row_mask
+def _largest_per_expert(scores, eligible, C):
+    """Independent statement of Eq. 7-10 / Algorithm 1 on tie-free scores: for every expert the
+    kept set is the C largest scores among the tokens eligible for it (all of them if fewer)."""
     N, E = scores.shape
-    cap_mask = np.zeros_like(row_mask)
+    want = np.zeros((N, E), bool)
     for e in range(E):
-        order = np.argsort(-masked[:, e], kind="stable")[:cap]
-        cap_mask[order, e] = 1
-    final_map = row_mask * cap_mask
-    return final_map, masked * final_map
+        toks = np.nonzero(eligible[:, e])[0]
+        best = toks[np.argsort(-scores[toks, e], kind="stable")[:C]]
+        want[best, e] = True
+    return want
 
 
-def test_token_drop_matches_dense_mask_formulation():
-    # tie-free inputs, every selected score > 0: there the column top-`cap` is unique
+def test_token_drop_keeps_the_C_largest_of_each_expert():
+    # tie-free inputs: there the C largest of a column are unique
     for (N, E, k, gamma) in [(512, 8, 2, 1.0), (384, 64, 8, 1.5), (600, 60, 4, 0.5)]:
         bias = -np.log(np.arange(E) + 1.0)
         s = _scores(N, E, 21, bias=bias)
         idx, val, load = oracle.topk(s, k)
-        cap = min(int(gamma * (N * k) / E), N)
+        C = min(int(gamma * (N * k) / E), N)
         if len(np.unique(val)) != val.size or val.min() <= 0:
             pytest.skip("inputs not tie-free")
-        row_mask = np.zeros((N, E), np.float32)
-        np.put_along_axis(row_mask, idx, 1.0, axis=1)
-        fmap, fscores = _dense_mask_formulation(s, row_mask, cap)
-        r = oracle.token_drop(s, idx, cap)
-        dense = mask_to_dense(r["keep_mask"], E)
-        assert np.array_equal(dense, fmap.astype(np.uint8))
-        # final_scores = scores * final_map: the weights the permutation carries
+        chose = np.zeros((N, E), bool)
+        np.put_along_axis(chose, idx, True, axis=1)
+        want = _largest_per_expert(s, chose, C)
+        r = oracle.token_drop(s, idx, C)
+        assert np.array_equal(mask_to_dense(r["keep_mask"], E).astype(bool), want)
+        # the gate weight carried by a kept row is the score of that (token, expert) pair (Eq. 2
+        # with the kept set in place of the top-k set)
         A = int(r["offsets"][-1])
         p = oracle.permute(None, s, idx, r["slot_row"], A, 0, "f32")
-        assert np.array_equal(p["perm_weight"], fscores[p["perm_token"], p["perm_expert"]])
-        assert fscores.astype(bool).sum() == A
+        assert np.array_equal(p["perm_weight"], s[p["perm_token"], p["perm_expert"]])
+        assert want[p["perm_token"], p["perm_expert"]].all() and want.sum() == A
 
 
 def test_token_drop_invariants():
@@ -350,22 +352,21 @@ def test_expanded_drop_single_group_is_expert_choice():
         assert np.array_equal(np.sort(order), np.nonzero(dense[:, e])[0])
 
 
-def test_expanded_drop_matches_dense_mask_formulation():
+def test_expanded_drop_keeps_the_C_largest_among_topk_and_home_device_tokens():
+    # Algorithm 2 on tie-free scores: eligible = chose the expert, or lives on the expert's device
     N, E, k, D = 512, 8, 2, 2
     m = E // D
     s = _scores(N, E, 91, bias=-np.log(np.arange(E) + 1.0))
     idx, _, _ = oracle.topk(s, k)
     if len(np.unique(s)) != s.size or s.min() <= 0:
         pytest.skip("inputs not tie-free")
-    cap = int(1.0 * (N * k) / E)
+    C = int(1.0 * (N * k) / E)
     home = (np.arange(N) * D) // N
-    exp_mask = np.zeros((N, E), np.float32)
-    np.put_along_axis(exp_mask, idx, 1.0, axis=1)
-    for t in range(N):
-        exp_mask[t, home[t] * m:(home[t] + 1) * m] = 1.0          # the local expert ids of the token's device
-    fmap, _ = _dense_mask_formulation(s, exp_mask, cap)
-    r = oracle.expanded_drop(s, idx, cap, D)
-    assert np.array_equal(mask_to_dense(r["keep_mask"], E), fmap.astype(np.uint8))
+    eligible = np.zeros((N, E), bool)
+    np.put_along_axis(eligible, idx, True, axis=1)
+    eligible |= (np.arange(E)[None, :] // m) == home[:, None]
+    r = oracle.expanded_drop(s, idx, C, D)
+    assert np.array_equal(mask_to_dense(r["keep_mask"], E).astype(bool), _largest_per_expert(s, eligible, C))
 
 
 # ----------------------------------------------------------------------------- permutation
