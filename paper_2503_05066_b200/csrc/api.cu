@@ -257,7 +257,11 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if (rc != CAPMOE_OK) return rc;
   if ((rc = mark(1)) != CAPMOE_OK) return rc;
   int slots, Dp;
+  // The permute kernel can write the keep mask while it reads a token's rows, unless something
+  // between the drop and the permute needs the mask ("w/ max").
+  bool defer_mask = !(L->mode != 0 && L->max_experts > 0);
   if (L->mode >= 3) {                     // device-level capacity: L->C is the per-device bound
+    defer_mask = false;                   // the token-parallel select writes the mask itself
     const int expanded = L->mode == 4;
     rc = device_drop_impl(L->scores, L->topk_idx, L->N, L->E, L->k, L->C, L->D, expanded, nullptr, L->keep_mask,
                           L->cand, L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream,
@@ -284,12 +288,14 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
     }
     if (expanded) {
       rc = expanded_drop_impl(sel, L->topk_idx, L->N, L->E, L->k, L->C, L->D, nullptr, L->keep_mask, L->cand,
-                              L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream, true);
+                              L->kept, L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream, true,
+                              &defer_mask, L->load);
       slots = L->k + L->E / L->D;
       Dp = L->D;
     } else {
       rc = token_drop_impl(sel, L->topk_idx, L->N, L->E, L->k, L->mode == 0 ? L->N : L->C, L->keep_mask, L->kept,
-                           L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream, true);
+                           L->expert_offsets, L->slot_row, L->drop_ws, L->drop_ws_bytes, stream, true, &defer_mask,
+                           L->load);
       slots = L->k;
       Dp = 0;
     }
@@ -303,8 +309,8 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   }
   if (rc != CAPMOE_OK) return rc;
   if ((rc = mark(2)) != CAPMOE_OK) return rc;
-  rc = capmoe_permute(L->x, L->N, L->d, L->E, L->k, slots, Dp, L->dtype, L->scores, L->topk_idx, nullptr,
-                      L->slot_row, L->x_perm, L->perm_token, L->perm_weight, stream);
+  rc = permute_impl(L->x, L->N, L->d, L->E, L->k, slots, Dp, L->dtype, L->scores, L->topk_idx, nullptr, L->slot_row,
+                    L->x_perm, L->perm_token, L->perm_weight, defer_mask ? L->keep_mask : nullptr, stream);
   if (rc != CAPMOE_OK) return rc;
   if ((rc = mark(3)) != CAPMOE_OK) return rc;
   rc = grouped_ffn_impl(L->x_perm, L->expert_offsets, L->E, L->d, L->F, L->dtype, L->w_gate, L->w_up, L->w_down,

@@ -18,17 +18,20 @@ int sm_count();                            // SMs of the current device (cached 
 // The stages as capmoe_layer_forward calls them.  With the last argument true the caller has
 // itself issued, earlier on the stream, the small memsets the stage begins with (load histogram,
 // drop counters: see drop_clear_counters): the stage skips them, and its first kernel chains onto
-// the previous stage's last one.  Argument lists as in capmoe.h.
+// the previous stage's last one.  Argument lists as in capmoe.h.  defer_mask (may be NULL): on entry
+// true if the caller can derive keep_mask from slot_row itself later (permute_impl does); on return
+// true if the stage left keep_mask unwritten for that reason.  load (may be NULL): the router's load
+// histogram of the same top-k lists, which saves the stage a count.
 int route_impl(const void* x, const void* w_router, const float* bias, const float* logits_in, int64_t N, int d, int E,
                int k, int dtype, float* logits, float* scores, int32_t* topk_idx, float* topk_score, int32_t* load,
                void* stream, bool load_cleared);
 int token_drop_impl(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C,
                     uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row, void* ws,
-                    size_t ws_bytes, void* stream, bool counters_cleared);
+                    size_t ws_bytes, void* stream, bool counters_cleared, bool* defer_mask, const int32_t* load);
 int expanded_drop_impl(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C, int D,
                        const int32_t* token_group, uint64_t* keep_mask, int32_t* cand, int32_t* kept,
                        int32_t* expert_offsets, int32_t* slot_row, void* ws, size_t ws_bytes, void* stream,
-                       bool counters_cleared);
+                       bool counters_cleared, bool* defer_mask, const int32_t* load);
 int device_drop_impl(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C_dev, int D,
                      int expanded, const int32_t* token_group, uint64_t* keep_mask, int32_t* cand, int32_t* kept,
                      int32_t* expert_offsets, int32_t* slot_row, void* ws, size_t ws_bytes, void* stream,
@@ -39,6 +42,13 @@ bool ffn_tc_supported(int d, int F, int dtype);
 // The memsets of the drop stage that would run for these arguments (mode as in capmoe_layer).
 int drop_clear_counters(int mode, int64_t N, int E, int k, int D, int32_t* cand, void* ws, size_t ws_bytes,
                         cudaStream_t st);
+// keep_mask from slot_row (one thread per token); and the permute stage with the same derivation
+// folded into its per-token bookkeeping (keep_mask_out may be NULL).
+int drop_mask_from_rows(const int32_t* slot_row, const int32_t* topk_idx, int64_t N, int E, int k, int slots, int D,
+                        const int32_t* token_group, uint64_t* keep_mask, cudaStream_t st);
+int permute_impl(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype, const float* scores,
+                 const int32_t* topk_idx, const int32_t* token_group, const int32_t* slot_row, void* x_perm,
+                 int32_t* perm_token, float* perm_weight, uint64_t* keep_mask_out, void* stream);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t elt_size(int dtype) { return dtype == CAPMOE_F32 ? 4 : 2; }

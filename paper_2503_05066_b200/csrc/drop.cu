@@ -4,7 +4,10 @@
 // (non-negative floats order like unsigned integers), and keep everything above it plus the
 // first (C - #above) candidates equal to it, in token order.
 //
-// One small memset (the E candidate counters) and two launches:
+// Batches below the token-parallel threshold run the cluster select of drop_cluster.cu; the
+// per-expert kernel k_select of this file, which lists the candidates in scratch memory, serves
+// the entry point with built-in scratch and batches no other path takes:
+// one small memset (the E candidate counters) and two launches:
 //   k_count_candidates  one CTA per 256 tokens: per-expert candidate counts (shared-memory
 //                       histogram, then integer atomics: the totals do not depend on order), and
 //                       the initial state of the outputs that k_select only touches sparsely
@@ -14,6 +17,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "select.cuh"
 
 namespace capmoe {
 
@@ -25,18 +29,25 @@ int drop_parallel(const float* scores, const float* topk_score, const int32_t* t
                   int32_t* cand_out, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row, void* ws_ptr,
                   size_t ws_bytes, cudaStream_t st, bool counters_cleared);
 
+// cluster select (drop_cluster.cu): batches below the token-parallel threshold
+bool drop_cluster_takes(int64_t N, int E, bool expanded);
+template <bool EXPANDED>
+int drop_cluster(const float* score_src, const int32_t* topk_idx, int64_t N, int E, int k, int64_t C, int D,
+                 const int32_t* token_group, const int32_t* load, uint64_t* keep_mask, int32_t* cand_out, int32_t* kept,
+                 int32_t* expert_offsets, int32_t* slot_row, cudaStream_t st);
+
 namespace {
 
-// From this many tokens on, the token-parallel select is faster than one CTA per expert.
-constexpr int64_t PARALLEL_MIN_TOKENS = 16384;
+// Batches the cluster select does not take go to the token-parallel select, whose 64-bit keys
+// hold the pair's position t*E + e in 32 bits.
+inline bool use_parallel(int64_t N, int E, bool expanded) {
+  return !drop_cluster_takes(N, E, expanded) && (unsigned long long)N * (unsigned)E < (1ull << 32);
+}
 
 constexpr int CNT_THREADS = 256;
 constexpr int TPT = 4;                               // tokens (candidates) per thread per round in k_select
 constexpr int CNT_TOKENS = CNT_THREADS;              // tokens per counting CTA
-constexpr int SEL_THREADS = 1024;
-constexpr int SEL_WARPS = SEL_THREADS / 32;
 constexpr int SEL_TOKENS = SEL_THREADS * TPT;        // tokens per compaction round
-constexpr int RADIX_BINS = 2048;                     // 11 + 11 + 10 bits
 constexpr int E_STRIDE = 256;                        // E <= 256
 
 struct DropWs {
@@ -100,52 +111,6 @@ k_count_candidates(const int32_t* __restrict__ topk_idx, int64_t N, int E, int k
   __syncthreads();
   for (int i = threadIdx.x; i < E; i += CNT_THREADS)
     if (hist[i]) atomicAdd(&cand[i], hist[i]);
-}
-
-// Exclusive prefix sum over the block (SEL_THREADS threads).  total = sum of all v.
-__device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t* sh /*[SEL_WARPS+1]*/, uint32_t& total) {
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  uint32_t incl = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += n;
-  }
-  if (lane == 31) sh[wid] = incl;
-  __syncthreads();
-  if (wid == 0) {
-    uint32_t w = sh[lane];                       // SEL_WARPS == 32
-    uint32_t wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      uint32_t n = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += n;
-    }
-    sh[lane] = wi - w;
-    if (lane == 31) sh[SEL_WARPS] = wi;
-  }
-  __syncthreads();
-  const uint32_t res = incl - v + sh[wid];
-  total = sh[SEL_WARPS];
-  __syncthreads();                               // sh may be reused right away
-  return res;
-}
-
-// Among `nbins` histogram bins ordered from the highest digit down, find the bin that holds the
-// rank-th largest element (rank >= 1).  Result in out[0] = bin, out[1] = rank inside that bin.
-__device__ __forceinline__ void find_bin(const int* hist, int nbins, uint32_t rank, uint32_t* scan_sh,
-                                         uint32_t* out) {
-  const int p0 = 2 * threadIdx.x, p1 = p0 + 1;
-  const uint32_t h0 = p0 < nbins ? (uint32_t)hist[nbins - 1 - p0] : 0u;
-  const uint32_t h1 = p1 < nbins ? (uint32_t)hist[nbins - 1 - p1] : 0u;
-  uint32_t total;
-  const uint32_t before = block_scan(h0 + h1, scan_sh, total);
-  if (before < rank && rank <= before + h0) {
-    out[0] = (uint32_t)(nbins - 1 - p0); out[1] = rank - before;
-  } else if (before + h0 < rank && rank <= before + h0 + h1) {
-    out[0] = (uint32_t)(nbins - 1 - p1); out[1] = rank - before - h0;
-  }
-  __syncthreads();
 }
 
 // One CTA per expert.
@@ -339,6 +304,14 @@ int run_drop(const float* score_src, const int32_t* topk_idx, int64_t N, int E, 
   return rc;
 }
 
+int empty_batch(int E, int32_t* cand_out, int32_t* kept, int32_t* expert_offsets, cudaStream_t st) {
+  cudaError_t err;
+  if ((err = cudaMemsetAsync(kept, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
+  if ((err = cudaMemsetAsync(expert_offsets, 0, sizeof(int32_t) * (E + 1), st)) != cudaSuccess) return note_cuda(err);
+  if (cand_out && (err = cudaMemsetAsync(cand_out, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return note_cuda(err);
+  return CAPMOE_OK;
+}
+
 int validate(int64_t N, int E, int k, int64_t C) {
   if (N < 0 || E < 1 || k < 1 || k > E || C < 0 || C > N) return CAPMOE_EINVAL;
   if (E > 256 || k > 32) return CAPMOE_EUNSUPPORTED;
@@ -363,7 +336,7 @@ extern "C" int capmoe_drop_workspace_bytes(int64_t N, int E, int k, int D, int e
 size_t capmoe::drop_ws_required(int mode, int64_t N, int E, int k, int D) {
   if (N <= 0) return 0;
   const bool device_level = mode >= 3, expanded = mode == 2 || mode == 4;
-  const bool parallel = device_level || (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32));
+  const bool parallel = device_level || use_parallel(N, E, expanded);
   return parallel ? drop_parallel_ws_bytes(N, E) : ws_bytes_needed(N, E, k, D, expanded ? 1 : 0);
 }
 
@@ -371,27 +344,38 @@ int capmoe::drop_clear_counters(int mode, int64_t N, int E, int k, int D, int32_
                                 cudaStream_t st) {
   if (N <= 0 || !ws) return CAPMOE_OK;                        // the stage handles (and checks) these itself
   const bool device_level = mode >= 3, expanded = mode == 2 || mode == 4;
-  const bool parallel = device_level || (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32));
+  const bool parallel = device_level || use_parallel(N, E, expanded);
   if (parallel) {
     if (ws_bytes < drop_parallel_ws_bytes(N, E)) return CAPMOE_EWORKSPACE;
     return drop_parallel_clear(ws, N, E, device_level ? D : E, st);
   }
   if (ws_bytes < ws_bytes_needed(N, E, k, D, expanded ? 1 : 0)) return CAPMOE_EWORKSPACE;
+  if (drop_cluster_takes(N, E, expanded)) return CAPMOE_OK;  // the cluster select starts from nothing
   int32_t* c = (expanded && cand) ? cand : carve(ws, N, E, k, D, expanded ? 1 : 0).cand;
   return note_cuda(cudaMemsetAsync(c, 0, sizeof(int32_t) * E, st));
 }
 
 int capmoe::token_drop_impl(const float* topk_score, const int32_t* topk_idx, int64_t N, int E, int k,
                                  int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
-                                 int32_t* slot_row, void* ws, size_t ws_bytes, void* stream, bool counters_cleared) {
+                                 int32_t* slot_row, void* ws, size_t ws_bytes, void* stream, bool counters_cleared,
+                                 bool* defer_mask, const int32_t* load) {
+  const bool may_defer = defer_mask && *defer_mask;
+  if (defer_mask) *defer_mask = false;
   int rc = validate(N, E, k, C);
   if (rc != CAPMOE_OK) return rc;
   if (!kept || !expert_offsets) return CAPMOE_EINVAL;
   if (N > 0 && (!topk_score || !topk_idx || !keep_mask || !slot_row || !ws)) return CAPMOE_EINVAL;
   if (N * (int64_t)k >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
-  if (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32))
+  if (N == 0) return empty_batch(E, nullptr, kept, expert_offsets, as_stream(stream));
+  if (use_parallel(N, E, false))
     return drop_parallel(nullptr, topk_score, topk_idx, N, E, k, C, 1, 1, 0, nullptr, keep_mask, nullptr, kept,
                          expert_offsets, slot_row, ws, ws_bytes, as_stream(stream), counters_cleared);
+  if (ws_bytes < ws_bytes_needed(N, E, k, 1, 0)) return CAPMOE_EWORKSPACE;
+  if (drop_cluster_takes(N, E, false)) {
+    if (may_defer) *defer_mask = true;
+    return drop_cluster<false>(topk_score, topk_idx, N, E, k, C, 1, nullptr, load, may_defer ? nullptr : keep_mask, nullptr,
+                               kept, expert_offsets, slot_row, as_stream(stream));
+  }
   return run_drop<false>(topk_score, topk_idx, N, E, k, C, 1, nullptr, keep_mask, nullptr, kept,
                          expert_offsets, slot_row, ws, ws_bytes, as_stream(stream), counters_cleared);
 }
@@ -399,16 +383,26 @@ int capmoe::token_drop_impl(const float* topk_score, const int32_t* topk_idx, in
 int capmoe::expanded_drop_impl(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
                                     int64_t C, int D, const int32_t* token_group, uint64_t* keep_mask,
                                     int32_t* cand, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row,
-                                    void* ws, size_t ws_bytes, void* stream, bool counters_cleared) {
+                                    void* ws, size_t ws_bytes, void* stream, bool counters_cleared, bool* defer_mask,
+                                    const int32_t* load) {
+  const bool may_defer = defer_mask && *defer_mask;
+  if (defer_mask) *defer_mask = false;
   int rc = validate(N, E, k, C);
   if (rc != CAPMOE_OK) return rc;
   if (D < 1 || E % D != 0) return CAPMOE_EINVAL;
   if (!kept || !expert_offsets || !cand) return CAPMOE_EINVAL;
   if (N > 0 && (!scores || !topk_idx || !keep_mask || !slot_row || !ws)) return CAPMOE_EINVAL;
   if (N * (int64_t)(k + E / D) >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
-  if (N >= PARALLEL_MIN_TOKENS && (unsigned long long)N * (unsigned)E < (1ull << 32))
+  if (N == 0) return empty_batch(E, cand, kept, expert_offsets, as_stream(stream));
+  if (use_parallel(N, E, true))
     return drop_parallel(scores, nullptr, topk_idx, N, E, k, C, D, 1, 1, token_group, keep_mask, cand, kept,
                          expert_offsets, slot_row, ws, ws_bytes, as_stream(stream), counters_cleared);
+  if (ws_bytes < ws_bytes_needed(N, E, k, D, 1)) return CAPMOE_EWORKSPACE;
+  if (drop_cluster_takes(N, E, true)) {
+    if (may_defer) *defer_mask = true;
+    return drop_cluster<true>(scores, topk_idx, N, E, k, C, D, token_group, load, may_defer ? nullptr : keep_mask, cand, kept,
+                              expert_offsets, slot_row, as_stream(stream));
+  }
   return run_drop<true>(scores, topk_idx, N, E, k, C, D, token_group, keep_mask, cand, kept, expert_offsets,
                         slot_row, ws, ws_bytes, as_stream(stream), counters_cleared);
 }
@@ -545,7 +539,7 @@ extern "C" int capmoe_token_drop(const float* topk_score, const int32_t* topk_id
                                  int64_t C, uint64_t* keep_mask, int32_t* kept, int32_t* expert_offsets,
                                  int32_t* slot_row, void* ws, size_t ws_bytes, void* stream) {
   return token_drop_impl(topk_score, topk_idx, N, E, k, C, keep_mask, kept, expert_offsets, slot_row, ws, ws_bytes,
-                         stream, false);
+                         stream, false, nullptr, nullptr);
 }
 
 extern "C" int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,
@@ -553,7 +547,7 @@ extern "C" int capmoe_expanded_drop(const float* scores, const int32_t* topk_idx
                                     int32_t* cand, int32_t* kept, int32_t* expert_offsets, int32_t* slot_row,
                                     void* ws, size_t ws_bytes, void* stream) {
   return expanded_drop_impl(scores, topk_idx, N, E, k, C, D, token_group, keep_mask, cand, kept, expert_offsets,
-                            slot_row, ws, ws_bytes, stream, false);
+                            slot_row, ws, ws_bytes, stream, false, nullptr, nullptr);
 }
 
 extern "C" int capmoe_device_drop(const float* scores, const int32_t* topk_idx, int64_t N, int E, int k,

@@ -17,7 +17,8 @@ __global__ void __launch_bounds__(PC_WARPS * 32)
 k_permute(const uint4* __restrict__ x, int64_t N, int row_vecs /* 16-byte vectors per row */, int chunks, int E,
           int k, int slots, int D, const float* __restrict__ scores, const int32_t* __restrict__ topk_idx,
           const int32_t* __restrict__ token_group, const int32_t* __restrict__ slot_row,
-          uint4* __restrict__ x_perm, int32_t* __restrict__ perm_token, float* __restrict__ perm_weight) {
+          uint4* __restrict__ x_perm, int32_t* __restrict__ perm_token, float* __restrict__ perm_weight,
+          unsigned long long* __restrict__ keep_mask /* NULL, or [N, ceil(E/64)] to be derived from slot_row here */) {
   wait_for_previous_kernel();
   const int lane = threadIdx.x & 31;
   const int64_t unit = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
@@ -28,13 +29,27 @@ k_permute(const uint4* __restrict__ x, int64_t N, int row_vecs /* 16-byte vector
   if (chunk == 0) {                                    // bookkeeping once per token: lane s handles slot s, s+32, ...
     const int m = D > 0 ? E / D : 0;
     const int g = D > 0 ? home_group(t, N, D, token_group) : 0;
+    uint32_t bits[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};          // this lane's share of the token's keep mask (E <= 256)
     for (int s = lane; s < slots; s += 32) {
       const int32_t r = sr[s];
       if (r >= 0) {
         const int e = s < k ? topk_idx[t * k + s] : g * m + (s - k);
         perm_token[r] = (int32_t)t;
         perm_weight[r] = scores[t * E + e];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (i == (e >> 5)) bits[i] |= 1u << (e & 31);
       }
+    }
+    if (keep_mask) {                                   // bit e set iff the slot that stands for expert e holds a row
+      const int W = (E + 63) >> 6;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (i < W) {
+          const uint32_t lo32 = __reduce_or_sync(0xffffffffu, bits[2 * i]);
+          const uint32_t hi32 = __reduce_or_sync(0xffffffffu, bits[2 * i + 1]);
+          if (lane == 0) keep_mask[t * W + i] = ((unsigned long long)hi32 << 32) | lo32;
+        }
     }
   }
   const int v0 = chunk * CHUNK_VECS + lane;
@@ -163,10 +178,10 @@ k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row
 
 using namespace capmoe;
 
-extern "C" int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
-                              const float* scores, const int32_t* topk_idx, const int32_t* token_group,
-                              const int32_t* slot_row, void* x_perm, int32_t* perm_token, float* perm_weight,
-                              void* stream) {
+int capmoe::permute_impl(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
+                         const float* scores, const int32_t* topk_idx, const int32_t* token_group,
+                         const int32_t* slot_row, void* x_perm, int32_t* perm_token, float* perm_weight,
+                         uint64_t* keep_mask_out, void* stream) {
   if (N < 0 || d < 1 || E < 1 || k < 1 || k > E || slots < k || D < 0) return CAPMOE_EINVAL;
   if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
   if (D > 0 && (E % D != 0 || slots != k + E / D)) return CAPMOE_EINVAL;
@@ -182,9 +197,18 @@ extern "C" int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int
   if (blocks > 0x7fffffff) return CAPMOE_EUNSUPPORTED;
   const int rc = note_cuda(launch_chained(k_permute, (unsigned)blocks, PC_WARPS * 32, 0, as_stream(stream),
                                           (const uint4*)x, N, row_vecs, chunks, E, k, slots, D, scores, topk_idx,
-                                          token_group, slot_row, (uint4*)x_perm, perm_token, perm_weight));
+                                          token_group, slot_row, (uint4*)x_perm, perm_token, perm_weight,
+                                          reinterpret_cast<unsigned long long*>(keep_mask_out)));
   count_launch(1);
   return rc;
+}
+
+extern "C" int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
+                              const float* scores, const int32_t* topk_idx, const int32_t* token_group,
+                              const int32_t* slot_row, void* x_perm, int32_t* perm_token, float* perm_weight,
+                              void* stream) {
+  return permute_impl(x, N, d, E, k, slots, D, dtype, scores, topk_idx, token_group, slot_row, x_perm, perm_token,
+                      perm_weight, nullptr, stream);
 }
 
 extern "C" int capmoe_combine(const void* y_perm, const int32_t* slot_row, const float* perm_weight, int64_t N,

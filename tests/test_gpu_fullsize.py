@@ -1,7 +1,8 @@
 """Parity at the full workload sizes, in the launch configuration bench.py times (whole-layer
 entry point, straggler emulation where the workload asks for it).  Routing, drop and
 permutation outputs are compared with the CPU checker element by element over all N tokens;
-the layer output on a sample of tokens the checker computes one by one."""
+the layer output on a sample of tokens the checker computes one by one, chosen so that every
+128-row block of every expert's segment (every row tile of the two GEMMs) holds a checked row."""
 import numpy as np
 import pytest
 import torch
@@ -18,17 +19,17 @@ pytestmark = pytest.mark.gpu
 def test_mixtral_shape(cm, mode, gamma, straggler):
     cfg = synth.CONFIGS["mixtral"]
     assert cm.ffn_uses_tensor_cores(cfg.d, cfg.F, torch.bfloat16)
-    _layer_case(cm, cfg, mode, gamma, straggler=straggler, sample=12)
+    _layer_case(cm, cfg, mode, gamma, straggler=straggler, sample=12, cover_blocks=True)
 
 
 @pytest.mark.parametrize("mode,gamma", [("nodrop", 1.0), ("token_drop", 1.0), ("expanded_drop", 1.5)])
 def test_olmoe_shape(cm, mode, gamma):
-    _layer_case(cm, synth.CONFIGS["olmoe"], mode, gamma, sample=48)
+    _layer_case(cm, synth.CONFIGS["olmoe"], mode, gamma, sample=48, cover_blocks=True)
 
 
 @pytest.mark.parametrize("mode", ["token_drop", "expanded_drop"])
 def test_dsv2lite_shape_with_shared_experts(cm, mode):
-    _layer_case(cm, synth.CONFIGS["dsv2lite"], mode, 1.0, sample=48)
+    _layer_case(cm, synth.CONFIGS["dsv2lite"], mode, 1.0, sample=48, cover_blocks=True)
 
 
 @pytest.mark.parametrize("N,gamma,mode", [(128, 0.5, "token_drop"), (128, 2.0, "expanded_drop"),

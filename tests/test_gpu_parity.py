@@ -146,13 +146,21 @@ DROP_CASES = [
     (100, 8, 2, 2, float("inf"), 0.0),
     (1, 8, 2, 2, 1.0, 0.0),
     (7, 4, 1, 2, 1.0, 0.0),
-    # large batches take the token-parallel select
-    (20000, 8, 2, 2, 1.0, 0.5),      # ties at the threshold resolved by position
+    # cluster select with several tokens per thread (2, 4, 8) and clusters of 8, 4, 2 and 1 CTAs
+    (20000, 8, 2, 2, 1.0, 0.5),      # ties at the threshold
     (16384, 64, 8, 8, 1.0, 0.0),
-    (17001, 60, 4, 4, 0.5, 1.0),
-    (16400, 130, 6, 10, 1.0, 0.0),
+    (40000, 8, 2, 2, 1.0, 0.25),
     (16384, 8, 2, 2, 0.0, 0.0),
     (16384, 8, 2, 2, float("inf"), 0.0),
+    (3500, 130, 6, 10, 1.0, 0.0),
+    (4000, 200, 4, 8, 1.0, 1.0),
+    # larger batches take the token-parallel select
+    (17001, 60, 4, 4, 0.5, 1.0),     # ties at the threshold resolved by position
+    (16400, 130, 6, 10, 1.0, 0.0),
+    (40000, 64, 8, 8, 1.0, 0.0),
+    (70000, 8, 2, 2, 1.0, 0.5),
+    (70000, 8, 2, 2, 0.0, 0.0),
+    (70000, 8, 2, 2, float("inf"), 0.0),
 ]
 
 
@@ -259,8 +267,11 @@ def test_permute_and_combine(cm, dtype, d, mode):
 
 
 # ----------------------------------------------------------------------------- stage 5 and the layer
-def _layer_case(cm, cfg, mode, gamma, straggler=False, sample=None, std=0.02):
-    """Run the CUDA layer, then the checker from the GPU's own fp32 logits; compare."""
+def _layer_case(cm, cfg, mode, gamma, straggler=False, sample=None, std=0.02, cover_blocks=False):
+    """Run the CUDA layer, then the checker from the GPU's own fp32 logits; compare.
+    sample: compare the layer output on that many random tokens (None = all).  cover_blocks: also
+    on one token out of every 128-row block of every expert's row segment (and of every 128-token
+    block of the batch when there is a shared expert), so that every row tile of both GEMMs is checked."""
     inp = cached_inputs(cfg)
     wg, wu, wd = inp.w_gate, inp.w_up, inp.w_down
     shared = inp.shared
@@ -299,7 +310,18 @@ def _layer_case(cm, cfg, mode, gamma, straggler=False, sample=None, std=0.02):
         toks = np.arange(cfg.N, dtype=np.int32)
     else:
         rng = np.random.default_rng(0)
-        toks = np.unique(np.concatenate([[0, cfg.N - 1], rng.integers(0, cfg.N, sample)])).astype(np.int32)
+        picks = [np.array([0, cfg.N - 1]), rng.integers(0, cfg.N, sample)]
+        if cover_blocks:
+            off = ref["offsets"].astype(np.int64)
+            rows = []
+            for e in range(cfg.E):
+                for r0 in range(int(off[e]), int(off[e + 1]), 128):
+                    rows.append(r0 + int(rng.integers(0, min(128, int(off[e + 1]) - r0))))
+            picks.append(pref["perm_token"][np.array(rows, dtype=np.int64)] if rows else np.array([], np.int64))
+            if shared is not None:
+                starts = np.arange(0, cfg.N, 128)
+                picks.append(starts + rng.integers(0, np.minimum(128, cfg.N - starts)))
+        toks = np.unique(np.concatenate(picks)).astype(np.int32)
     yref = oracle.layer_tokens(xs, toks, scores, idx, ref["slot_row"], Dp, *args, cfg.dtype)
     if shared is not None:
         ysh = oracle.expert_ffn(np.ascontiguousarray(xs[toks]), None, *(to_np(s) for s in shared), cfg.dtype)
