@@ -66,6 +66,12 @@ __device__ __forceinline__ int home_group(int64_t t, int64_t N, int D, const int
 // finished and its writes are visible.  That removes most of the gap (about 3 us) between two
 // dependent launches.  Without the launch attribute the wait is a no-op.
 __device__ __forceinline__ void wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Called first thing in every kernel: once all CTAs of this grid have started, the next kernel on
+// the stream (if it was launched with the attribute above) may be scheduled onto free resources.  Its
+// CTAs run up to their own wait_for_previous_kernel(), which still returns only when this whole
+// grid has finished, so nothing it reads or writes moves ahead; what moves ahead is its launch
+// latency and whatever set-up it does before the wait.
+__device__ __forceinline__ void allow_next_kernel() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,

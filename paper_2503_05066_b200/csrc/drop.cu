@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(CNT_THREADS)
 k_count_candidates(const int32_t* __restrict__ topk_idx, int64_t N, int E, int k, int D,
                    const int32_t* __restrict__ token_group, int32_t* __restrict__ cand,
                    unsigned long long* __restrict__ keep_mask, int32_t* __restrict__ slot_row) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   extern __shared__ int hist[];
   for (int i = threadIdx.x; i < E; i += CNT_THREADS) hist[i] = 0;
@@ -121,6 +122,7 @@ k_select(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop)
          const int32_t* __restrict__ token_group, const int32_t* __restrict__ cand, DropWs ws,
          unsigned long long* __restrict__ keep_mask, int32_t* __restrict__ kept,
          int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   __shared__ int hist[RADIX_BINS];
   __shared__ uint32_t scan_sh[SEL_WARPS + 1];

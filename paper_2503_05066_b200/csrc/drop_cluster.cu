@@ -71,6 +71,7 @@ k_select_cluster(const float* __restrict__ score_src,   // topk_score [N,k] (Tok
                  const int32_t* __restrict__ token_group, const int32_t* __restrict__ load /* [E] or NULL */, int R,
                  int64_t T /* tokens per CTA */, int32_t* __restrict__ cand_out /* [E] or NULL */, int32_t* __restrict__ kept,
                  int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ int hist[3][RADIX_BINS];               // the leader's copies are the cluster's histograms
@@ -269,6 +270,7 @@ k_select_cluster(const float* __restrict__ score_src,   // topk_score [N,k] (Tok
 __global__ void __launch_bounds__(256)
 k_mask_from_rows(const int32_t* __restrict__ slot_row, const int32_t* __restrict__ topk_idx, int64_t N, int E, int k,
                  int slots, int D, const int32_t* __restrict__ token_group, unsigned long long* __restrict__ keep_mask) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (t >= N) return;

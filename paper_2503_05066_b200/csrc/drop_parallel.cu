@@ -92,6 +92,7 @@ __device__ __forceinline__ bool pair_of(const PArgs& a, int64_t t, int s, const 
 
 __global__ void __launch_bounds__(PAIR_THREADS)
 pk_hist(PArgs a, PWs w, int level, Level lv, int first_level_counts_cand) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   __shared__ int cand_s[MAX_SEG];
   const int tid = threadIdx.x;
@@ -129,6 +130,7 @@ pk_hist(PArgs a, PWs w, int level, Level lv, int first_level_counts_cand) {
 // prefix, clear the counters.  Thread i owns 8 consecutive bins, highest bins first.
 __global__ void __launch_bounds__(CHUNK)
 pk_find(PWs w, unsigned long long C_seg, int level, Level lv, int n_levels) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   __shared__ uint32_t wtot[CHUNK / 32 + 1];
   __shared__ uint32_t res[3];
@@ -203,6 +205,7 @@ pk_find(PWs w, unsigned long long C_seg, int level, Level lv, int n_levels) {
 
 __global__ void __launch_bounds__(PAIR_THREADS)
 pk_count(PArgs a, PWs w) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   __shared__ int cnt_s[MAX_SEG];
   const int tid = threadIdx.x;
@@ -226,6 +229,7 @@ pk_count(PArgs a, PWs w) {
 // one CTA per expert: exclusive scan of its per-chunk counts
 __global__ void __launch_bounds__(CHUNK)
 pk_scan(PWs w, int E, int chunks, int32_t* __restrict__ kept, int32_t* __restrict__ cand_out) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   __shared__ int warp_tot[CHUNK / 32 + 1];
   const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -260,6 +264,7 @@ pk_scan(PWs w, int E, int chunks, int32_t* __restrict__ kept, int32_t* __restric
 __global__ void __launch_bounds__(PAIR_THREADS)
 pk_place(PArgs a, PWs w, const int32_t* __restrict__ kept, unsigned long long* __restrict__ keep_mask,
          int32_t* __restrict__ expert_offsets, int32_t* __restrict__ slot_row) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   __shared__ int off[MAX_SEG + 1];
   __shared__ uint32_t bitmap[MAX_SEG][CHUNK / 32];

@@ -48,6 +48,8 @@ constexpr int TC_THREADS = 64 + EPI_WARPS * 32;
 constexpr int RF_SUBS = 4;
 constexpr int RF_THREADS = 64 + 4 * RF_SUBS * 32;
 constexpr int RF_XCH_FLOATS = RF_SUBS * 128 + 128 + 4 * RF_SUBS * 128;   // max, sum relay, top-k candidates
+constexpr int RF_SPREAD_ROWS = 64;        // row tiles up to this size share their tokens among all epilogue warps
+
 constexpr int MAX_E = 256;
 // Epilogue staging: each FFN epilogue warp packs a 32-row x 32-column bf16 piece of the output into
 // 2 KB of shared memory (64-byte rows, 64-byte swizzle) and one lane hands it to TMA to store.
@@ -56,6 +58,7 @@ constexpr int STG_BYTES = EPI_WARPS * STG_WARP_BYTES;      // 16 KB, right behin
 constexpr int TAIL_OFF = STAGES * STAGE_BYTES + STG_BYTES; // barriers and tables start here
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STG_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/ +
                            2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/ + RF_XCH_FLOATS * 4;
+static_assert(RF_SPREAD_ROWS * 64 * 4 <= STG_BYTES, "the fused router's shared logits tile lives in the staging area");
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -358,7 +361,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
   constexpr bool ROUTER = MODE == MODE_ROUTER || MODE == MODE_ROUTER_FUSED;
   constexpr bool FUSED = MODE == MODE_ROUTER_FUSED;
-  wait_for_previous_kernel();
+  allow_next_kernel();
   constexpr int N_TILE = SWIGLU ? 128 : 256;
   __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(out_ptr);
   const uint32_t idesc = make_idesc(n_mma);
@@ -390,6 +393,13 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   auto tempty_bar = [&](int b) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 + b); };
   // tile queue: barriers 40..47 and four ints behind them, inside the 512-byte barrier block
   const TileQueue<false> tq{bar0 + 8u * 40u, bar0 + 8u * 44u, bar0 + 8u * 48u, 0u, abort_flag};
+  // Set-up that touches no global memory (barriers, tensor memory) runs before the wait for the
+  // previous kernel, so that it overlaps that kernel's tail.
+  if (tid == 32) {                                       // the descriptors the first loads will need
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b0) : "memory");
+    if (SWIGLU) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b1) : "memory");
+  }
   if (tid == 0) {
     for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), nthreads - 64); }
@@ -397,9 +407,17 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  wait_for_previous_kernel();
   if (ROUTER) {
+    // (the bias is fetched by the epilogue warps, which are the only ones to use it: the first
+    // loads do not wait for that round trip to global memory)
     if (tid == 0) { offs[0] = 0; offs[1] = single_rows; }
-    for (int i = tid; i < 256; i += nthreads) bias_s[i] = (bias && i < Nout) ? bias[i] : 0.f;
     if (FUSED)
       for (int i = tid; i < EPAD; i += nthreads) hist[i] = 0;
   } else {
@@ -414,12 +432,6 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       acc += ((offs[e + 1] - offs[e] + tile_rows - 1) / tile_rows) * n_blocks;
     }
     tile_start[E] = acc;
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(512u)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -537,6 +549,10 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..9)
+    if (ROUTER) {
+      for (int i = tid - 64; i < 256; i += nthreads - 64) bias_s[i] = (bias && i < Nout) ? bias[i] : 0.f;
+      group_sync(6, nthreads - 64);
+    }
     const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
     const int row_in_tile = quarter * 32 + lane;
     const int half = (warp - 2) >> 2;                    // which half of the columns this warp converts
@@ -556,6 +572,126 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)BNB;
       const bool row_ok = row_in_tile < t.rows;
       if constexpr (FUSED) {
+        if (tile_rows <= RF_SPREAD_ROWS) {
+          // Small row tiles (few tokens per SM): with one thread per (token, column quarter) only the
+          // warps of the first one or two TMEM lane quarters would have tokens, i.e. one or two of the
+          // SM's four warp schedulers.  Instead those warps only move the logits out (global memory and
+          // a shared-memory tile), and then all sixteen warps share the tokens, eight threads per token
+          // (eight consecutive lanes, an eighth of the columns each, exchange by shuffles).
+          constexpr int COLS = EPAD / RF_SUBS;                 // columns a dumping thread reads from TMEM
+          constexpr int CS = EPAD / 8;                         // columns per thread afterwards
+          float* lt = reinterpret_cast<float*>(gen + STAGES * STAGE_BYTES);   // [RF_SPREAD_ROWS][EPAD] logits + bias
+          const int sub = (warp - 2) >> 2;
+          const int cbase = sub * COLS;
+          if (quarter * 32 < t.rows) {
+            uint32_t g[COLS];
+            if constexpr (COLS == 16) tmem_ld16(taddr + (uint32_t)cbase, g);
+            else tmem_ld8(taddr + (uint32_t)cbase, g);
+            tmem_ld_wait();
+            float v[COLS];
+#pragma unroll
+            for (int i = 0; i < COLS; ++i)
+              v[i] = cbase + i < Nout ? __fadd_rn(__uint_as_float(g[i]), bias_s[cbase + i]) : -INFINITY;
+            if (row_ok) {
+              float* lrow = reinterpret_cast<float*>(out_ptr) + ((int64_t)t.row0 + row_in_tile) * Nout + cbase;
+              if ((Nout & 3) == 0) {
+#pragma unroll
+                for (int i = 0; i < COLS; i += 4)
+                  if (cbase + i < Nout) *reinterpret_cast<float4*>(lrow + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+              } else {
+#pragma unroll
+                for (int i = 0; i < COLS; ++i)
+                  if (cbase + i < Nout) lrow[i] = v[i];
+              }
+            }
+            if (row_in_tile < RF_SPREAD_ROWS) {
+#pragma unroll
+              for (int i = 0; i < COLS; i += 4)
+                *reinterpret_cast<float4*>(lt + row_in_tile * EPAD + cbase + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(tempty_bar(b));
+          group_sync(5, 4 * RF_SUBS * 32);                     // the tile of logits is complete
+          const int et = tid - 64;                             // 0 .. 511
+          const int r = et >> 3, j = et & 7;
+          const bool tok_ok = r < t.rows;
+          const int64_t tok = (int64_t)t.row0 + r;
+          const int c0 = j * CS;
+          float v[CS];
+#pragma unroll
+          for (int i = 0; i < CS; i += 4) {
+            const float4 q4 = *reinterpret_cast<const float4*>(lt + (r & (RF_SPREAD_ROWS - 1)) * EPAD + c0 + i);
+            v[i] = q4.x; v[i + 1] = q4.y; v[i + 2] = q4.z; v[i + 3] = q4.w;
+          }
+          if (!tok_ok) {
+#pragma unroll
+            for (int i = 0; i < CS; ++i) v[i] = 0.f;          // rows past the tile: defined values, results unused
+          }
+          float mx = v[0];
+#pragma unroll
+          for (int i = 1; i < CS; ++i) mx = v[i] > mx ? v[i] : mx;
+#pragma unroll
+          for (int o = 4; o > 0; o >>= 1) { const float ov = __shfl_xor_sync(0xffffffffu, mx, o); mx = ov > mx ? ov : mx; }
+#pragma unroll
+          for (int i = 0; i < CS; ++i) v[i] = exp_fixed(__fsub_rn(v[i], mx));      // padding: exp(-inf) = 0
+          // the E terms are added left to right: the partial sum walks through the token's eight threads
+          float acc = 0.f;
+#pragma unroll
+          for (int s2 = 0; s2 < 8; ++s2) {
+            const float incoming = __shfl_up_sync(0xffffffffu, acc, 1, 8);
+            if (j == s2) {
+              acc = s2 ? incoming : 0.f;
+#pragma unroll
+              for (int i = 0; i < CS; ++i) acc = __fadd_rn(acc, v[i]);             // + 0 (padding) is exact
+            }
+          }
+          const float sum = __shfl_sync(0xffffffffu, acc, 7, 8);                   // in [1, E]
+          const float rsum = __frcp_rn(sum);
+#pragma unroll
+          for (int i = 0; i < CS; ++i) v[i] = c0 + i < Nout ? div_by(v[i], sum, rsum) : -1.f;   // padding never selected
+          if (tok_ok) {
+            float* srow = rf.scores + tok * Nout + c0;
+            if ((Nout & 3) == 0) {
+#pragma unroll
+              for (int i = 0; i < CS; i += 4)
+                if (c0 + i < Nout) *reinterpret_cast<float4*>(srow + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < CS; ++i)
+                if (c0 + i < Nout) srow[i] = v[i];
+            }
+          }
+          // top-k: k rounds; each thread offers the best of its columns (lower id on ties), the eight
+          // offers meet in a butterfly on (score, lower id), the owner marks its column taken
+#pragma unroll 1
+          for (int kk = 0; kk < rf.k; ++kk) {
+            float best = -1.f;
+            int bi = 0;
+#pragma unroll
+            for (int i = 0; i < CS; ++i) { const bool gt = v[i] > best; best = gt ? v[i] : best; bi = gt ? i : bi; }
+            int be = c0 + bi;
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {
+              const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+              const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+              const bool take = ob > best || (ob == best && oe < be);
+              best = take ? ob : best;
+              be = take ? oe : be;
+            }
+            if (be >= c0 && be < c0 + CS) {                                        // this thread's offer won
+#pragma unroll
+              for (int i = 0; i < CS; ++i) v[i] = (c0 + i == be) ? -2.f : v[i];    // taken
+              if (tok_ok) {
+                rf.topk_idx[tok * rf.k + kk] = be;
+                rf.topk_score[tok * rf.k + kk] = best;
+                atomicAdd(&hist[be], 1);
+              }
+            }
+          }
+          group_sync(5, 4 * RF_SUBS * 32);                     // the next tile may overwrite the shared tile
+          continue;
+        }
         // RF_SUBS threads per token (same lane of the quarter's four warps), each with COLS of the
         // token's columns in registers.  The accumulator goes back to the MMA issuer as soon as it
         // has been read; what is not local to a thread passes through shared memory between the
@@ -808,7 +944,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
   constexpr int N_TILE = SWIGLU ? 128 : 256;
   constexpr int BM2 = 2 * BM;                                   // rows of a pair's tile
-  wait_for_previous_kernel();
+  allow_next_kernel();
   const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BNB >> 3) << 17) |
                          ((uint32_t)(BM2 >> 4) << 24);          // M = 256, N = 256
   extern __shared__ uint8_t smem_raw[];
@@ -831,6 +967,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   // tile queue: barriers 40..47 and four ints behind them, inside the 512-byte barrier block
   const TileQueue<true> tq{bar0 + 8u * 40u, bar0 + 8u * 44u, bar0 + 8u * 48u, rank, abort_flag};
 
+  // set-up that touches no global memory comes before the wait for the previous kernel (see k_ffn_tc)
   if (tid == 0) {
     for (int s = 0; s < STAGES2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 2 * EPI_WARPS * 32); }
@@ -838,6 +975,13 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  wait_for_previous_kernel();
   for (int i = tid; i <= E; i += TC_THREADS) offs[i] = expert_offsets[i];
   __syncthreads();
   if (tid == 0) {
@@ -848,12 +992,6 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       acc += ((offs[e + 1] - offs[e] + BM2 - 1) / BM2) * n_blocks;
     }
     tile_start[E] = acc;
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(512u)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -1226,10 +1364,14 @@ int router_tc(const void* x, const void* w_router, const float* bias, int64_t N,
   // multiple of 8 rows, the swizzle atom; at most 128, the MMA's M).  The MMA always spans 128
   // rows; the rows past tile_rows cost nothing that is on the critical path.
   const int sms = sm_count();
-  const int64_t rounds = ceil_div(N, (int64_t)128 * sms);
+  // (Every tile re-reads W_r through L2, and an SM's L2 port, not HBM, bounds the k-loop of small
+  // tiles: capping tiles at 64 rows so that their epilogue hides under the next tile's loads measured
+  // no faster at 16384 tokens and 5 % slower at 65536.)
+  const int max_rows = 128;
+  const int64_t rounds = ceil_div(N, (int64_t)max_rows * sms);
   int tile_rows = (int)((ceil_div(N, (int64_t)sms * rounds) + 7) / 8 * 8);
   if (tile_rows < 32) tile_rows = 32;
-  if (tile_rows > 128) tile_rows = 128;
+  if (tile_rows > max_rows) tile_rows = max_rows;
   // A stage holds tile_rows rows of A followed by n_mma rows of B (both multiples of 1 KB).  The
   // MMA reads 128 A rows whatever tile_rows is, so the last stage must leave room for that.
   const int b_bytes = n_mma * BK * 2;

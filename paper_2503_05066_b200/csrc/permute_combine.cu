@@ -19,6 +19,7 @@ k_permute(const uint4* __restrict__ x, int64_t N, int row_vecs /* 16-byte vector
           const int32_t* __restrict__ token_group, const int32_t* __restrict__ slot_row,
           uint4* __restrict__ x_perm, int32_t* __restrict__ perm_token, float* __restrict__ perm_weight,
           unsigned long long* __restrict__ keep_mask /* NULL, or [N, ceil(E/64)] to be derived from slot_row here */) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   const int lane = threadIdx.x & 31;
   const int64_t unit = (int64_t)blockIdx.x * PC_WARPS + (threadIdx.x >> 5);
@@ -126,6 +127,7 @@ __global__ void __launch_bounds__(PC_WARPS * 32, 4)
 k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row,
           const float* __restrict__ perm_weight, int64_t N, int row_vecs, int chunks, int slots,
           const uint4* __restrict__ y_shared, uint4* __restrict__ y) {
+  allow_next_kernel();
   wait_for_previous_kernel();
   constexpr int NV = Vec16<T>::n;
   const int lane = threadIdx.x & 31;

@@ -1,4 +1,6 @@
 // Stage 1: router GEMM, softmax, per-token top-k, expert load histogram (Eq. 1, Eq. 3).
+#include <cstdlib>
+
 #include "common.cuh"
 #include "softmax.cuh"
 
@@ -15,6 +17,7 @@ template <typename T, int EPT>
 __global__ void __launch_bounds__(RT_TOK* RT_EG)
 k_router_gemm(const T* __restrict__ x, const T* __restrict__ w, const float* __restrict__ bias,
               int64_t N, int d, int E, float* __restrict__ logits) {
+  allow_next_kernel();
   extern __shared__ float smem[];
   float* xs = smem;                              // [RT_TOK][RT_BK+1]
   float* wsm = smem + RT_TOK * (RT_BK + 1);      // [E][RT_BK+1]
@@ -131,6 +134,7 @@ template <int EPL>
 __global__ void __launch_bounds__(SW_WARPS * 32)
 k_softmax_topk_warp(const float* __restrict__ logits, int64_t N, int E, int k, float* __restrict__ scores,
                     int32_t* __restrict__ topk_idx, float* __restrict__ topk_score, int32_t* __restrict__ load) {
+  allow_next_kernel();
   extern __shared__ float smem[];
   float* prow = smem + (threadIdx.x >> 5) * (EPL * 32);       // this warp's E exponentials
   int* hist = reinterpret_cast<int*>(smem + SW_WARPS * EPL * 32);
@@ -216,6 +220,7 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
              const float* __restrict__ bias, int64_t N, int d, int E, float* __restrict__ logits, int k,
              float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
              int32_t* __restrict__ load) {
+  allow_next_kernel();
   extern __shared__ float red[];                       // [RM_WARPS][16*MT][NT*8 + 1] (+ fused scratch)
   constexpr int ROWS = 16 * MT, EP = NT * 8, LD = EP + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -315,6 +320,8 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
 
 bool router_mma_ok(int d, int E) { return d % (RM_WARPS * 64) == 0 && E <= 128; }
 
+inline int dbg_tc_min_e() { static int v = getenv("CAPMOE_DEBUG_TC_MIN_E") ? atoi(getenv("CAPMOE_DEBUG_TC_MIN_E")) : 17; return v; }
+
 struct RouteOut { int k; float* scores; int32_t* topk_idx; float* topk_score; int32_t* load; };
 
 template <int MT, int NT, bool FUSED>
@@ -373,7 +380,7 @@ int capmoe::route_impl(const void* x, const void* w_router, const float* bias, c
     const RouteOut ro{k, scores, topk_idx, topk_score, load};
     if (dtype == CAPMOE_F32)
       rc = launch_gemm<float>((const float*)x, (const float*)w_router, bias, N, d, E, logits, st);
-    else if (E > 16 && router_tc_supported(N, d, E) && aligned16(x) && aligned16(w_router)) {
+    else if (E >= dbg_tc_min_e() && router_tc_supported(N, d, E) && aligned16(x) && aligned16(w_router)) {
       fused = router_tc_fusable(E, k);
       rc = router_tc(x, w_router, bias, N, d, E, logits, scores, topk_idx, topk_score, load, k, fused, st);
     }

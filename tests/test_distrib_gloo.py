@@ -50,3 +50,23 @@ def test_single_process_is_a_no_op():
     assert distrib.max_over_ranks(3.5, info) == 3.5
     assert distrib.job_throughput(10, 5.0, info) == 2000.0
     assert distrib.shard_seed(7, distrib.RankInfo(3, 4, 3)) == 10
+
+
+def test_bench_starts_its_own_ranks_when_called_with_gpus(tmp_path):
+    """`python bench.py --gpus 2` without a launcher around it re-runs itself as two ranks
+    (torch.distributed.run on 127.0.0.1).  Checked on CPU with the reference arm, which needs no
+    GPU: rank 0 prints the one JSON line for n_gpus = 2, the other rank exits 0 without output."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference",
+                        "--config", "tiny_f32", "--steps", "1", "--warmup", "0", "--ref-tokens", "4"],
+                       capture_output=True, text=True, timeout=600, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["extrapolated"] is True
+    assert line["value"] > 0 and line["e2e"]["h2d_bytes_per_step"] == 0
