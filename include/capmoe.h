@@ -257,6 +257,60 @@ int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offsets, int E,
                        void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
                        int32_t* dev_status, void* stream);
 
+/* The same stage over explicit row segments: segment s holds the rows [seg_begin[s], seg_end[s]) of
+ * x_rows (seg_begin, seg_end: device int32 [S], non-overlapping, ascending) and is multiplied with
+ * weight block s % w_mod of w_gate / w_up [w_mod,F,d] and w_down [w_mod,d,F] (w_mod = 0: block s of
+ * S).  This is the form the owner of a few experts runs under expert parallelism, where every
+ * (source rank, local expert) pair is a segment of at most C_local rows at a fixed place (see
+ * capmoe_ep_segments).  rows = allocated rows of x_rows / h_ws / y_rows; rows outside every segment
+ * are neither read into a result nor written.  dev_status as above (no straggler emulation here). */
+int capmoe_grouped_ffn_segments(const void* x_rows, const int32_t* seg_begin, const int32_t* seg_end, int S,
+                                int w_mod, int d, int F, int dtype, const void* w_gate, const void* w_up,
+                                const void* w_down, void* h_ws, void* y_rows, int64_t rows,
+                                int32_t* dev_status, void* stream);
+
+/* ---------------------------------------------------------------- expert parallelism
+ * The paper's deployment (experimental set-up: data parallel over the tokens, expert parallel over
+ * the experts) with the capacity applied "within each local device" (Capacity-Aware Token Drop
+ * paragraph), so that tokens are "discarded prior to All-to-All" (Figure 3) and no rank needs to
+ * know another rank's load: rank r of R routes and drops its own N_local tokens with
+ * C_local = capmoe_capacity(N_local, E, k, gamma) - stages 1 to 3 unchanged, Expanded Drop with
+ * D = R and every token's home device = r - and owns the m = E/R experts r*m .. r*m+m-1.
+ * Because a rank keeps at most C_local rows per expert, every message has a fixed place and a
+ * fixed bound: the row space of a rank is [E][C_local] (row e*C_local + i = the i-th kept row of
+ * expert e, token-ascending), its block [r'*m*C_local, (r'+1)*m*C_local) goes to rank r', and the
+ * owner receives [R][m][C_local] rows (source-major).  No counts cross the host.
+ *
+ * capmoe_ep_plan      slot_row (rows of the packed matrix, stages 2/3) -> slot_row_ep (rows of the
+ *                     [E][C_local] space, or -1); *bad (device int32) is set to 1 if an expert holds
+ *                     more than C_local rows.  The send counts are the stage's kept[E].
+ * capmoe_permute / capmoe_combine with slot_row_ep and [E*C_local, d] buffers then fill the send
+ *                     buffer and read the returned rows when the exchange is a collective (two
+ *                     equal-split all-to-alls each way: rows and counts).
+ * capmoe_ep_dispatch  the permute stage writing each kept row straight into its owner's receive
+ *                     buffer: peer_rows[r'] (device array of R addresses) = base of rank r''s
+ *                     [R*m*C_local, d] buffer, mapped into this process (peer access within a node);
+ *                     this rank's rows land in block `rank` of it.  perm_token / perm_weight
+ *                     [E*C_local] stay local.  Plain stores, no multicast.
+ * capmoe_ep_segments  counts [R*m] (received: kept of (source, local expert)) -> seg_begin / seg_end
+ *                     of the R*m segments for capmoe_grouped_ffn_segments (w_mod = m).
+ * capmoe_ep_combine   the combine stage reading each kept row's result straight from its owner's
+ *                     [R*m*C_local, d] output buffer (peer_rows as above).
+ * The caller orders the ranks (all rows and counts have arrived before the owner's FFN starts, all
+ * results are written before a combine reads them); no kernel of this library waits for another rank. */
+int capmoe_ep_plan(const int32_t* slot_row, const int32_t* topk_idx, const int32_t* expert_offsets, int64_t N,
+                   int E, int k, int slots, int D, const int32_t* token_group, int64_t C_local,
+                   int32_t* slot_row_ep, int32_t* bad, void* stream);
+int capmoe_ep_segments(const int32_t* counts, int S, int64_t C_local, int32_t* seg_begin, int32_t* seg_end,
+                       void* stream);
+int capmoe_ep_dispatch(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
+                       const float* scores, const int32_t* topk_idx, const int32_t* token_group,
+                       const int32_t* slot_row_ep, const uint64_t* peer_rows, int R, int rank,
+                       int64_t C_local, int32_t* perm_token, float* perm_weight, void* stream);
+int capmoe_ep_combine(const uint64_t* peer_rows, int R, int rank, int E, int64_t C_local,
+                      const int32_t* slot_row_ep, const float* perm_weight, int64_t N, int d, int slots,
+                      int dtype, const void* y_shared, void* y, void* stream);
+
 /* Self-test of the bounded device-side wait used inside the tensor-core kernels (no counterpart
  * in the paper).  Launches one warp that waits on a barrier nothing will ever signal, with the
  * same wait routine and a limit of limit_cycles SM clock cycles (1 .. 4e9); the wait must run

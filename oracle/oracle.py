@@ -22,7 +22,7 @@ _lib = None
 __all__ = ["build", "capacity", "device_capacity", "device_drop", "drop_keys", "drop_keyed", "METRICS",
            "priority_keys", "limit_experts", "rows_from_mask", "router_logits", "softmax", "topk", "token_drop",
            "expanded_drop",
-           "permute", "expert_ffn", "combine", "layer_tokens", "stats", "layer_forward", "num_threads"]
+           "permute", "expert_ffn", "combine", "layer_tokens", "stats", "layer_forward", "ep_layer", "num_threads"]
 
 
 def build(force: bool = False) -> str:
@@ -323,10 +323,12 @@ def stats(load: np.ndarray, N: int, k: int, C: int):
 
 
 def layer_forward(x, w_router, bias, w_gate, w_up, w_down, k: int, gamma: float, D: int, mode: str,
-                  dtype: str, logits: Optional[np.ndarray] = None, shared=None, round_mode: str = "ceil"):
+                  dtype: str, logits: Optional[np.ndarray] = None, shared=None, round_mode: str = "ceil",
+                  token_group: Optional[np.ndarray] = None):
     """Whole layer on the CPU.  mode in {"nodrop", "token_drop", "expanded_drop"}.
     If `logits` is given it replaces the router GEMM (parity checks downstream of the router
-    start from identical fp32 logits)."""
+    start from identical fp32 logits).  token_group: explicit home device per token for Expanded
+    Drop (default: contiguous blocks)."""
     N, d = x.shape
     E = w_router.shape[0]
     if logits is None:
@@ -335,17 +337,77 @@ def layer_forward(x, w_router, bias, w_gate, w_up, w_down, k: int, gamma: float,
     idx, val, load = topk(scores, k)
     C = N if mode == "nodrop" else capacity(N, E, k, gamma, round_mode)
     if mode == "expanded_drop":
-        r = expanded_drop(scores, idx, C, D)
+        r = expanded_drop(scores, idx, C, D, token_group=token_group)
         Dp = D
     else:
         r = token_drop(scores, idx, C)
         Dp = 0
     A = int(r["offsets"][-1])
-    p = permute(x, scores, idx, r["slot_row"], A, Dp, dtype)
+    p = permute(x, scores, idx, r["slot_row"], A, Dp, dtype, token_group)
     y_perm = expert_ffn(p["x_perm"], p["perm_expert"], w_gate, w_up, w_down, dtype)
     y_sh = None
     if shared is not None:
         y_sh = expert_ffn(x, None, shared[0], shared[1], shared[2], dtype)
-    y = combine(y_perm, r["slot_row"], scores, idx, Dp, y_sh)
+    y = combine(y_perm, r["slot_row"], scores, idx, Dp, y_sh, token_group)
     return dict(logits=logits, scores=scores, topk_idx=idx, topk_score=val, load=load, C=C, A=A, y=y,
                 y_perm=y_perm, **r, **p)
+
+
+def ep_layer(x_ranks, w_router, bias, w_gate, w_up, w_down, k: int, gamma: float, mode: str, dtype: str,
+             logits_ranks=None, round_mode: str = "ceil"):
+    """The layer under expert parallelism with per-rank capacity, rank by rank and message by message.
+
+    The paper's deployment is data parallel over the tokens and expert parallel over the experts
+    (experimental set-up), and the capacity is applied "within each local device" so that no rank
+    needs another rank's load and tokens are dropped before the all-to-all (Capacity-Aware Token
+    Drop paragraph, Figure 3).  With R = len(x_ranks) ranks and m = E/R experts per rank:
+      1. rank r routes its own N_r tokens (Eq. 1) and applies C_r = capacity(N_r, E, k, gamma) to
+         them alone: Token Drop, or Expanded Drop with D = R devices and every one of its tokens at
+         home on device r (its candidates are its top-k experts plus the m experts rank r owns);
+      2. its kept rows, expert-major and token-ascending, are cut by owner: the rows of experts
+         r'*m .. r'*m+m-1 form the message r -> r' (at most m * C_r rows);
+      3. owner r' runs E_i(x) (Eq. 2) on what it received, with its own m experts only;
+      4. the results travel back in the same order and rank r combines them (Eq. 2).
+    x_ranks / logits_ranks: one array per rank.  Returns per-rank outputs and the message sizes."""
+    R = len(x_ranks)
+    E = w_router.shape[0]
+    assert E % R == 0
+    m = E // R
+    ranks = []
+    for r in range(R):
+        x = x_ranks[r]
+        N = x.shape[0]
+        logits = router_logits(x, w_router, bias, dtype) if logits_ranks is None else logits_ranks[r]
+        scores = softmax(logits)
+        idx, val, load = topk(scores, k)
+        C = N if mode == "nodrop" else capacity(N, E, k, gamma, round_mode)
+        tg = None
+        if mode == "expanded_drop":
+            tg = np.full((N,), r, np.int32)
+            dr = expanded_drop(scores, idx, C, R, token_group=tg)
+            Dp = R
+        else:
+            dr = token_drop(scores, idx, C)
+            Dp = 0
+        A = int(dr["offsets"][-1])
+        p = permute(x, scores, idx, dr["slot_row"], A, Dp, dtype, tg)
+        ranks.append(dict(N=N, C=C, scores=scores, topk_idx=idx, load=load, Dp=Dp, tg=tg, A=A, **dr, **p))
+    # messages r -> r': rows of the experts r' owns, and how many of each
+    off = [rk["offsets"] for rk in ranks]
+    send = [[ranks[r]["x_perm"][off[r][o * m]:off[r][(o + 1) * m]] for o in range(R)] for r in range(R)]
+    send_counts = np.array([[ranks[r]["kept"][o * m:(o + 1) * m] for o in range(R)] for r in range(R)], np.int64)
+    # owners: E_i(x) on the received rows with the owner's m experts (weights [o*m, (o+1)*m) only)
+    back = [[None] * R for _ in range(R)]
+    for o in range(R):
+        wg, wu, wd = (np.ascontiguousarray(w[o * m:(o + 1) * m]) for w in (w_gate, w_up, w_down))
+        for r in range(R):
+            rows = np.ascontiguousarray(send[r][o])
+            local = np.repeat(np.arange(m, dtype=np.int32), send_counts[r, o])
+            back[r][o] = (expert_ffn(rows, local, wg, wu, wd, dtype) if len(rows)
+                          else np.zeros((0, rows.shape[1]), np.float64))
+    ys = []
+    for r in range(R):
+        rk = ranks[r]
+        y_perm = np.concatenate([back[r][o] for o in range(R)], axis=0) if rk["A"] else np.zeros((0, x_ranks[r].shape[1]))
+        ys.append(combine(y_perm, rk["slot_row"], rk["scores"], rk["topk_idx"], rk["Dp"], None, rk["tg"]))
+    return dict(y=ys, ranks=ranks, send_counts=send_counts, m=m)

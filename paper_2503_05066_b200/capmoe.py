@@ -28,7 +28,9 @@ EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_device_max_rows", "capm
            "capmoe_token_drop", "capmoe_token_drop_static", "capmoe_expanded_drop", "capmoe_device_capacity",
            "capmoe_device_drop", "capmoe_drop_keys", "capmoe_priority_keys", "capmoe_limit_experts",
            "capmoe_rows_from_mask", "capmoe_permute", "capmoe_grouped_ffn",
-           "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe"]
+           "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe",
+           "capmoe_grouped_ffn_segments", "capmoe_ep_plan", "capmoe_ep_segments", "capmoe_ep_dispatch",
+           "capmoe_ep_combine"]
 
 
 class CapmoeError(RuntimeError):
@@ -361,6 +363,76 @@ def grouped_ffn(x_perm, offsets, w_gate, w_up, w_down, D_straggler: int = 0, h_w
                                     _i64(A_max), int(D_straggler), _ptr(dev_status), _stream(stream)),
            "capmoe_grouped_ffn")
     return y_perm
+
+
+def grouped_ffn_segments(x_rows, seg_begin, seg_end, w_gate, w_up, w_down, w_mod: int, h_ws=None, y_rows=None,
+                         dev_status=None, stream=None):
+    """SwiGLU FFN over explicit row segments; segment s uses weight block s % w_mod.  -> y_rows"""
+    rows, d = x_rows.shape
+    F = w_gate.shape[-2]
+    dev = x_rows.device
+    if dev_status is None:
+        dev_status = torch.zeros((FFN_STATUS_WORDS,), device=dev, dtype=torch.int32)
+    if h_ws is None:
+        h_ws = torch.empty((rows, F), device=dev, dtype=x_rows.dtype)
+    if y_rows is None:
+        y_rows = torch.zeros((rows, d), device=dev, dtype=x_rows.dtype)
+    _check(lib().capmoe_grouped_ffn_segments(_ptr(x_rows), _ptr(seg_begin), _ptr(seg_end), int(seg_begin.numel()),
+                                             int(w_mod), int(d), int(F), _dt(x_rows), _ptr(w_gate), _ptr(w_up),
+                                             _ptr(w_down), _ptr(h_ws), _ptr(y_rows), _i64(rows), _ptr(dev_status),
+                                             _stream(stream)), "capmoe_grouped_ffn_segments")
+    return y_rows
+
+
+def ep_plan(slot_row, topk_idx, offsets, E: int, C_local: int, D: int = 1, token_group=None, stream=None):
+    """-> (slot_row_ep [N,slots], bad [1]): rows of the [E][C_local] space of an expert-parallel rank."""
+    N, slots = slot_row.shape
+    k = topk_idx.shape[1]
+    out = torch.empty_like(slot_row)
+    bad = torch.zeros((1,), device=slot_row.device, dtype=torch.int32)
+    _check(lib().capmoe_ep_plan(_ptr(slot_row), _ptr(topk_idx), _ptr(offsets), _i64(N), int(E), int(k), int(slots),
+                                int(D), _ptr(token_group), _i64(C_local), _ptr(out), _ptr(bad), _stream(stream)),
+           "capmoe_ep_plan")
+    return out, bad
+
+
+def ep_segments(counts, C_local: int, stream=None):
+    """counts [S] int32 -> (seg_begin, seg_end) of the S fixed-place segments of C_local rows each."""
+    S = counts.numel()
+    b, e = torch.empty_like(counts), torch.empty_like(counts)
+    _check(lib().capmoe_ep_segments(_ptr(counts), int(S), _i64(C_local), _ptr(b), _ptr(e), _stream(stream)),
+           "capmoe_ep_segments")
+    return b, e
+
+
+def ep_dispatch(x, scores, topk_idx, slot_row_ep, peer_rows, R: int, rank: int, C_local: int, D: int = 0,
+                token_group=None, out=None, stream=None):
+    """Permute with every kept row stored into its owner's buffer (peer_rows: int64 tensor of R base
+    addresses on the device).  -> dict(perm_token, perm_weight) of the local [E*C_local] row space."""
+    N, d = x.shape
+    E = scores.shape[1]
+    k = topk_idx.shape[1]
+    slots = slot_row_ep.shape[1]
+    if out is None:
+        out = dict(perm_token=torch.full((max(E * C_local, 1),), -1, device=x.device, dtype=torch.int32),
+                   perm_weight=torch.zeros((max(E * C_local, 1),), device=x.device, dtype=torch.float32))
+    _check(lib().capmoe_ep_dispatch(_ptr(x), _i64(N), int(d), int(E), int(k), int(slots), int(D), _dt(x), _ptr(scores),
+                                    _ptr(topk_idx), _ptr(token_group), _ptr(slot_row_ep), _ptr(peer_rows), int(R),
+                                    int(rank), _i64(C_local), _ptr(out["perm_token"]), _ptr(out["perm_weight"]),
+                                    _stream(stream)), "capmoe_ep_dispatch")
+    return out
+
+
+def ep_combine(peer_rows, R: int, rank: int, E: int, C_local: int, slot_row_ep, perm_weight, d: int, dtype,
+               y_shared=None, y=None, stream=None):
+    """Combine with every kept row's result read from its owner's buffer (peer_rows as in ep_dispatch)."""
+    N, slots = slot_row_ep.shape
+    if y is None:
+        y = torch.empty((N, d), device=slot_row_ep.device, dtype=dtype)
+    _check(lib().capmoe_ep_combine(_ptr(peer_rows), int(R), int(rank), int(E), _i64(C_local), _ptr(slot_row_ep),
+                                   _ptr(perm_weight), _i64(N), int(d), int(slots), _dt(dtype), _ptr(y_shared), _ptr(y),
+                                   _stream(stream)), "capmoe_ep_combine")
+    return y
 
 
 def combine(y_perm, slot_row, perm_weight, y_shared=None, y=None, stream=None):

@@ -38,34 +38,36 @@ int sm_count() {
 }
 
 // defined in ffn_simt.cu / ffn_tc.cu
-int ffn_simt(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
-             const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
+int ffn_simt(const void* x_perm, const int32_t* seg_begin, const int32_t* seg_end, int E, int w_mod, int d, int F,
+             int dtype, const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
              int64_t A_max, cudaEvent_t mid, cudaStream_t st);
-bool ffn_tc_supported(int d, int F, int dtype);
-int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
-           const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
-           int32_t* dev_status, int sched_slot, bool counters_cleared, cudaEvent_t mid, cudaStream_t st);
+int ffn_tc(const void* x_perm, const int32_t* seg_begin, const int32_t* seg_end, int E, int w_mod, int n_w, int d, int F,
+           const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max,
+           int D_straggler, int32_t* dev_status, int sched_slot, bool counters_cleared, cudaEvent_t mid, cudaStream_t st);
 int wait_probe(long long limit_cycles, int32_t* dev_status, cudaStream_t st);
 
-static int grouped_ffn_impl(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
-                            const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
-                            int64_t A_max, int D_straggler, int32_t* dev_status, cudaEvent_t mid, void* stream,
-                            int sched_slot = 0, bool counters_cleared = false) {
-  if (E < 1 || d < 1 || F < 1 || A_max < 0 || D_straggler < 0) return CAPMOE_EINVAL;
+// Row segments [seg_begin[e], seg_end[e]), e < E; segment e uses weight block e % w_mod (w_mod = 0:
+// block e).  The packed form of the stage is seg_begin = expert_offsets, seg_end = expert_offsets + 1.
+static int grouped_ffn_impl(const void* x_perm, const int32_t* seg_begin, const int32_t* seg_end, int E, int w_mod, int d,
+                            int F, int dtype, const void* w_gate, const void* w_up, const void* w_down, void* h_ws,
+                            void* y_perm, int64_t A_max, int D_straggler, int32_t* dev_status, cudaEvent_t mid,
+                            void* stream, int sched_slot = 0, bool counters_cleared = false) {
+  if (E < 1 || d < 1 || F < 1 || A_max < 0 || D_straggler < 0 || w_mod < 0 || w_mod > E) return CAPMOE_EINVAL;
   if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
   if (D_straggler > 0 && E % D_straggler != 0) return CAPMOE_EINVAL;
   if (E > 256) return CAPMOE_EUNSUPPORTED;
-  if (!expert_offsets) return CAPMOE_EINVAL;
+  if (!seg_begin || !seg_end) return CAPMOE_EINVAL;
   if (A_max == 0) return CAPMOE_OK;
   if (!x_perm || !w_gate || !w_up || !w_down || !h_ws || !y_perm) return CAPMOE_EINVAL;
   if (!aligned16(x_perm) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) || !aligned16(h_ws) ||
       !aligned16(y_perm))
     return CAPMOE_EINVAL;
+  const int n_w = w_mod > 0 ? w_mod : E;
   if (ffn_tc_supported(d, F, dtype))
-    return ffn_tc(x_perm, expert_offsets, E, d, F, w_gate, w_up, w_down, h_ws, y_perm, A_max, D_straggler,
-                  dev_status, sched_slot, counters_cleared, mid, as_stream(stream));
+    return ffn_tc(x_perm, seg_begin, seg_end, E, w_mod, n_w, d, F, w_gate, w_up, w_down, h_ws, y_perm, A_max,
+                  D_straggler, dev_status, sched_slot, counters_cleared, mid, as_stream(stream));
   if (D_straggler > 0) return CAPMOE_EUNSUPPORTED;   // SM partitioning exists only in the tensor-core kernel
-  return ffn_simt(x_perm, expert_offsets, E, d, F, dtype, w_gate, w_up, w_down, h_ws, y_perm, A_max, mid,
+  return ffn_simt(x_perm, seg_begin, seg_end, E, w_mod, d, F, dtype, w_gate, w_up, w_down, h_ws, y_perm, A_max, mid,
                   as_stream(stream));
 }
 
@@ -149,8 +151,17 @@ extern "C" int capmoe_grouped_ffn(const void* x_perm, const int32_t* expert_offs
                                   int dtype, const void* w_gate, const void* w_up, const void* w_down,
                                   void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
                                   int32_t* dev_status, void* stream) {
-  return grouped_ffn_impl(x_perm, expert_offsets, E, d, F, dtype, w_gate, w_up, w_down, h_ws, y_perm, A_max,
-                          D_straggler, dev_status, nullptr, stream);
+  if (!expert_offsets) return CAPMOE_EINVAL;
+  return grouped_ffn_impl(x_perm, expert_offsets, expert_offsets + 1, E, 0, d, F, dtype, w_gate, w_up, w_down, h_ws,
+                          y_perm, A_max, D_straggler, dev_status, nullptr, stream);
+}
+
+extern "C" int capmoe_grouped_ffn_segments(const void* x_rows, const int32_t* seg_begin, const int32_t* seg_end, int S,
+                                           int w_mod, int d, int F, int dtype, const void* w_gate, const void* w_up,
+                                           const void* w_down, void* h_ws, void* y_rows, int64_t rows,
+                                           int32_t* dev_status, void* stream) {
+  return grouped_ffn_impl(x_rows, seg_begin, seg_end, S, w_mod, d, F, dtype, w_gate, w_up, w_down, h_ws, y_rows, rows,
+                          0, dev_status, nullptr, stream);
 }
 
 namespace capmoe {
@@ -313,7 +324,8 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
                     L->x_perm, L->perm_token, L->perm_weight, defer_mask ? L->keep_mask : nullptr, stream);
   if (rc != CAPMOE_OK) return rc;
   if ((rc = mark(3)) != CAPMOE_OK) return rc;
-  rc = grouped_ffn_impl(L->x_perm, L->expert_offsets, L->E, L->d, L->F, L->dtype, L->w_gate, L->w_up, L->w_down,
+  rc = grouped_ffn_impl(L->x_perm, L->expert_offsets, L->expert_offsets + 1, L->E, 0, L->d, L->F, L->dtype, L->w_gate,
+                        L->w_up, L->w_down,
                         L->h_ws, L->y_perm, L->A_max, L->straggler ? L->D : 0, L->dev_status,
                         L->stage_events ? (cudaEvent_t)L->stage_events[4] : nullptr, stream, 0, true);
   if (rc != CAPMOE_OK) return rc;
@@ -321,7 +333,8 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if ((rc = mark(5)) != CAPMOE_OK) return rc;
   const void* y_shared = nullptr;
   if (L->F_shared > 0) {
-    rc = grouped_ffn_impl(L->x, L->one_segment, 1, L->d, L->F_shared, L->dtype, L->ws_gate, L->ws_up, L->ws_down,
+    rc = grouped_ffn_impl(L->x, L->one_segment, L->one_segment + 1, 1, 0, L->d, L->F_shared, L->dtype, L->ws_gate,
+                          L->ws_up, L->ws_down,
                           L->hs_ws, L->y_shared, L->N, 0, L->dev_status, nullptr, stream, 1, true);
     if (rc != CAPMOE_OK) return rc;
     y_shared = L->y_shared;

@@ -16,8 +16,8 @@ constexpr int NT = 256;      // threads: 16 x 16, each a 4 x 4 micro-tile
 // SWIGLU: two B operands (gate, up) and out = silu(g) * u.
 template <typename T, bool SWIGLU>
 __global__ void __launch_bounds__(NT)
-k_grouped_gemm(const T* __restrict__ A, const int32_t* __restrict__ expert_offsets, int E, int K, int Nout,
-               const T* __restrict__ B0, const T* __restrict__ B1, T* __restrict__ C) {
+k_grouped_gemm(const T* __restrict__ A, const int32_t* __restrict__ seg_begin, const int32_t* __restrict__ seg_end,
+               int w_mod, int E, int K, int Nout, const T* __restrict__ B0, const T* __restrict__ B1, T* __restrict__ C) {
   __shared__ float As[BK][TS + 4];
   __shared__ float Bs0[BK][TS + 4];
   __shared__ float Bs1[SWIGLU ? BK : 1][TS + 4];
@@ -27,7 +27,7 @@ k_grouped_gemm(const T* __restrict__ A, const int32_t* __restrict__ expert_offse
     int slot = blockIdx.y, found = -1, row0 = 0, rows = 0;
     int acc = 0;
     for (int e = 0; e < E; ++e) {
-      const int b = expert_offsets[e], n = expert_offsets[e + 1] - b;
+      const int b = seg_begin[e], n = seg_end[e] - b;
       const int nt = (n + TS - 1) / TS;
       if (slot < acc + nt) {
         found = e;
@@ -45,8 +45,9 @@ k_grouped_gemm(const T* __restrict__ A, const int32_t* __restrict__ expert_offse
   const int row0 = seg[1], rows = seg[2];
   const int col0 = blockIdx.x * TS;
   const int tx = tid & 15, ty = tid >> 4;
-  const T* Be0 = B0 + (int64_t)e * Nout * K;
-  const T* Be1 = SWIGLU ? B1 + (int64_t)e * Nout * K : nullptr;
+  const int we = w_mod > 0 ? e % w_mod : e;             // weight block of this segment
+  const T* Be0 = B0 + (int64_t)we * Nout * K;
+  const T* Be1 = SWIGLU ? B1 + (int64_t)we * Nout * K : nullptr;
 
   float acc0[4][4], acc1[4][4];
 #pragma unroll
@@ -100,29 +101,29 @@ k_grouped_gemm(const T* __restrict__ A, const int32_t* __restrict__ expert_offse
 }
 
 template <typename T>
-int run(const T* x_perm, const int32_t* expert_offsets, int E, int d, int F, const T* wg, const T* wu,
-        const T* wd, T* h, T* y, int64_t A_max, cudaEvent_t mid, cudaStream_t st) {
+int run(const T* x_perm, const int32_t* seg_begin, const int32_t* seg_end, int E, int w_mod, int d, int F, const T* wg,
+        const T* wu, const T* wd, T* h, T* y, int64_t A_max, cudaEvent_t mid, cudaStream_t st) {
   const unsigned slots = (unsigned)(ceil_div(A_max, TS) + E);
   if (slots > 65535u) return CAPMOE_EUNSUPPORTED;
-  k_grouped_gemm<T, true><<<dim3((unsigned)ceil_div(F, TS), slots), NT, 0, st>>>(x_perm, expert_offsets, E, d, F,
-                                                                                wg, wu, h);
+  k_grouped_gemm<T, true><<<dim3((unsigned)ceil_div(F, TS), slots), NT, 0, st>>>(x_perm, seg_begin, seg_end, w_mod, E,
+                                                                                d, F, wg, wu, h);
   int rc = check_launch();
   if (rc != CAPMOE_OK) return rc;
   if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
-  k_grouped_gemm<T, false><<<dim3((unsigned)ceil_div(d, TS), slots), NT, 0, st>>>(h, expert_offsets, E, F, d, wd,
-                                                                                 nullptr, y);
+  k_grouped_gemm<T, false><<<dim3((unsigned)ceil_div(d, TS), slots), NT, 0, st>>>(h, seg_begin, seg_end, w_mod, E, F,
+                                                                                 d, wd, nullptr, y);
   return check_launch();
 }
 
 }  // namespace
 
-int ffn_simt(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, int dtype,
-             const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
+int ffn_simt(const void* x_perm, const int32_t* seg_begin, const int32_t* seg_end, int E, int w_mod, int d, int F,
+             int dtype, const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm,
              int64_t A_max, cudaEvent_t mid, cudaStream_t st) {
   if (dtype == CAPMOE_F32)
-    return run<float>((const float*)x_perm, expert_offsets, E, d, F, (const float*)w_gate, (const float*)w_up,
-                      (const float*)w_down, (float*)h_ws, (float*)y_perm, A_max, mid, st);
-  return run<__nv_bfloat16>((const __nv_bfloat16*)x_perm, expert_offsets, E, d, F, (const __nv_bfloat16*)w_gate,
+    return run<float>((const float*)x_perm, seg_begin, seg_end, E, w_mod, d, F, (const float*)w_gate,
+                      (const float*)w_up, (const float*)w_down, (float*)h_ws, (float*)y_perm, A_max, mid, st);
+  return run<__nv_bfloat16>((const __nv_bfloat16*)x_perm, seg_begin, seg_end, E, w_mod, d, F, (const __nv_bfloat16*)w_gate,
                             (const __nv_bfloat16*)w_up, (const __nv_bfloat16*)w_down, (__nv_bfloat16*)h_ws,
                             (__nv_bfloat16*)y_perm, A_max, mid, st);
 }

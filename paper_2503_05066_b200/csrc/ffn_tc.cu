@@ -16,7 +16,7 @@
 // GEMM1 puts 128 gate rows and 128 up rows of the same output columns into one 256-row B tile,
 // so one MMA yields both halves of the SwiGLU pair.  k_ffn_tc2 is the same pipeline on CTA pairs
 // (cta_group::2, 256 x 256 tiles, each CTA loads half of B) and serves long expert segments.
-// Tiles are enumerated on the device from expert_offsets (no host synchronisation); within an
+// Tiles are enumerated on the device from the segment bounds (no host synchronisation); within an
 // expert the row-block index runs fastest so that concurrently running CTAs share weight tiles
 // through L2.  With a status block from the caller the CTAs take their tiles from a device counter
 // (TileQueue below), else each walks a fixed list.  In straggler-emulation mode the CTAs are split
@@ -57,7 +57,8 @@ constexpr int STG_WARP_BYTES = 32 * 64;
 constexpr int STG_BYTES = EPI_WARPS * STG_WARP_BYTES;      // 16 KB, right behind the operand ring
 constexpr int TAIL_OFF = STAGES * STAGE_BYTES + STG_BYTES; // barriers and tables start here
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STG_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/ +
-                           2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/ + RF_XCH_FLOATS * 4;
+                           2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/ + RF_XCH_FLOATS * 4 + MAX_E * 4 /*segment ends*/;
+static_assert(SMEM_BYTES <= 227 * 1024, "dynamic shared memory limit of a thread block");
 static_assert(RF_SPREAD_ROWS * 64 * 4 <= STG_BYTES, "the fused router's shared logits tile lives in the staging area");
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
 
@@ -321,12 +322,13 @@ struct TileQueue {
 struct Tile { int e, row0, rows, n0; };
 
 // tile_start[e] = first tile of expert e; tiles of an expert: row block fastest, then column block.
-__device__ __forceinline__ bool locate_tile(int tile, int& cursor, const int* tile_start, const int* offs, int E,
-                                            int n_tile, int bm, Tile& t) {
+// offs[e] / ends[e]: first row of segment e and the row after its last.
+__device__ __forceinline__ bool locate_tile(int tile, int& cursor, const int* tile_start, const int* offs,
+                                            const int* ends, int E, int n_tile, int bm, Tile& t) {
   while (cursor < E && tile >= tile_start[cursor + 1]) ++cursor;
   if (cursor >= E) return false;
   const int local = tile - tile_start[cursor];
-  const int cnt = offs[cursor + 1] - offs[cursor];
+  const int cnt = ends[cursor] - offs[cursor];
   const int nmb = (cnt + bm - 1) / bm;
   const int nb = local / nmb, mb = local - nb * nmb;
   t.e = cursor;
@@ -352,7 +354,9 @@ template <int MODE, int EPAD = 32>
 __global__ void __launch_bounds__(MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, 1)
 k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
          const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_out /* FFN modes: the
-         output as 32 x 32 boxes */, const int32_t* __restrict__ expert_offsets, int E,
+         output as 32 x 32 boxes */, const int32_t* __restrict__ seg_begin, const int32_t* __restrict__ seg_end /* [E]:
+         rows [seg_begin[e], seg_end[e]) form segment e; for packed segments seg_end = seg_begin + 1 */,
+         int w_mod /* > 0: segment e uses weight block e % w_mod */, int E,
          int K /* reduction length */, int Nout /* output columns */, void* __restrict__ out_ptr,
          int D_straggler, int32_t* __restrict__ dev_status, int n_mma, int single_rows,
          const float* __restrict__ bias, int tile_rows /* rows per tile actually loaded (<= 128) */,
@@ -383,6 +387,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   float* bias_s = reinterpret_cast<float*>(tile_start + (MAX_E + 1) + 2);   // [256], router mode only
   int* hist = tile_start + 8;                          // [<= 128] load histogram, fused router only
   float* xch = bias_s + 256;                           // [RF_XCH_FLOATS] exchange between a token's threads
+  int* ends = reinterpret_cast<int*>(xch + RF_XCH_FLOATS);   // [MAX_E] row after the last of each segment
   const int nthreads = (int)blockDim.x;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -417,11 +422,11 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
   if (ROUTER) {
     // (the bias is fetched by the epilogue warps, which are the only ones to use it: the first
     // loads do not wait for that round trip to global memory)
-    if (tid == 0) { offs[0] = 0; offs[1] = single_rows; }
+    if (tid == 0) { offs[0] = 0; ends[0] = single_rows; }
     if (FUSED)
       for (int i = tid; i < EPAD; i += nthreads) hist[i] = 0;
   } else {
-    for (int i = tid; i <= E; i += nthreads) offs[i] = expert_offsets[i];
+    for (int i = tid; i < E; i += nthreads) { offs[i] = seg_begin[i]; ends[i] = seg_end[i]; }
   }
   __syncthreads();
   if (tid == 0) {
@@ -429,7 +434,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     int acc = 0;
     for (int e = 0; e < E; ++e) {
       tile_start[e] = acc;
-      acc += ((offs[e + 1] - offs[e] + tile_rows - 1) / tile_rows) * n_blocks;
+      acc += ((ends[e] - offs[e] + tile_rows - 1) / tile_rows) * n_blocks;
     }
     tile_start[E] = acc;
   }
@@ -485,7 +490,8 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       for (int j = 0; ok; ++j) {
         const int tile = dyn ? cur : next_tile(j, false);
         if (tile < 0) break;
-        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
+        if (!locate_tile(tile, cursor, tile_start, offs, ends, E, N_TILE, tile_rows, t)) break;
+        const int we = w_mod > 0 ? t.e % w_mod : t.e;     // weight block of this segment
         for (int kb = 0; kb < num_kb; ++kb) {
           if (dyn && kb == pub_kb) {
             cur = tile_lo + claim;
@@ -499,10 +505,10 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
           const uint32_t b_dst = a_dst + a_bytes;
           tma_load_2d(a_dst, &map_a, kb * BK, t.row0, full_bar(s));
           if (SWIGLU) {
-            tma_load_3d(b_dst, &map_b0, kb * BK, t.n0, t.e, full_bar(s));
-            tma_load_3d(b_dst + B_BYTES / 2, &map_b1, kb * BK, t.n0, t.e, full_bar(s));
+            tma_load_3d(b_dst, &map_b0, kb * BK, t.n0, we, full_bar(s));
+            tma_load_3d(b_dst + B_BYTES / 2, &map_b1, kb * BK, t.n0, we, full_bar(s));
           } else {
-            tma_load_3d(b_dst, &map_b0, kb * BK, ROUTER ? 0 : t.n0, t.e, full_bar(s));
+            tma_load_3d(b_dst, &map_b0, kb * BK, ROUTER ? 0 : t.n0, we, full_bar(s));
           }
           if (++s == n_stages) { s = 0; ph ^= 1u; }
         }
@@ -525,7 +531,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
       for (int j = 0; ok; ++j, ++it) {
         const int tile = next_tile(j, false);
         if (tile < 0) break;
-        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
+        if (!locate_tile(tile, cursor, tile_start, offs, ends, E, N_TILE, tile_rows, t)) break;
         const uint32_t b = it & 1u, use = it >> 1;
         if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -562,7 +568,7 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
     for (int j = 0;; ++j, ++it) {
       const int tile = next_tile(j, true);
       if (tile < 0) break;
-      if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, tile_rows, t)) break;
+      if (!locate_tile(tile, cursor, tile_start, offs, ends, E, N_TILE, tile_rows, t)) break;
       const uint32_t b = it & 1u, use = it >> 1;
       bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
       ready = __all_sync(0xffffffffu, ready);            // warp-uniform: tcgen05.ld below is .sync.aligned
@@ -938,7 +944,7 @@ template <int MODE>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
           const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_out /* the output as
-          32 x 32 boxes */, const int32_t* __restrict__ expert_offsets, int E,
+          32 x 32 boxes */, const int32_t* __restrict__ seg_begin, const int32_t* __restrict__ seg_end, int w_mod, int E,
           int K, int Nout, __nv_bfloat16* __restrict__ out, int D_straggler, int32_t* __restrict__ dev_status,
           int32_t* __restrict__ sched /* tile counters, one per straggler group, zeroed; NULL = fixed lists */) {
   constexpr bool SWIGLU = MODE == MODE_GATE_UP;
@@ -956,6 +962,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* offs = reinterpret_cast<int*>(gen + TAIL_OFF + 512);
   int* tile_start = offs + (MAX_E + 1);
+  int* ends = reinterpret_cast<int*>(reinterpret_cast<float*>(tile_start + (MAX_E + 1) + 2) + 256 + RF_XCH_FLOATS);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();                      // 0 = leader (issues the MMAs)
@@ -982,14 +989,14 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   wait_for_previous_kernel();
-  for (int i = tid; i <= E; i += TC_THREADS) offs[i] = expert_offsets[i];
+  for (int i = tid; i < E; i += TC_THREADS) { offs[i] = seg_begin[i]; ends[i] = seg_end[i]; }
   __syncthreads();
   if (tid == 0) {
     const int n_blocks = (Nout + N_TILE - 1) / N_TILE;
     int acc = 0;
     for (int e = 0; e < E; ++e) {
       tile_start[e] = acc;
-      acc += ((offs[e + 1] - offs[e] + BM2 - 1) / BM2) * n_blocks;
+      acc += ((ends[e] - offs[e] + BM2 - 1) / BM2) * n_blocks;
     }
     tile_start[E] = acc;
   }
@@ -1051,8 +1058,9 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       for (int j = 0; ok; ++j) {
         const int tile = scheduler ? cur : next_tile(j, false);
         if (tile < 0) break;
-        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
+        if (!locate_tile(tile, cursor, tile_start, offs, ends, E, N_TILE, BM2, t)) break;
         const int my_row0 = t.row0 + (int)rank * BM;
+        const int we = w_mod > 0 ? t.e % w_mod : t.e;     // weight block of this segment
         for (int kb = 0; kb < num_kb; ++kb) {
           if (scheduler && kb == pub_kb) {
             cur = tile_lo + claim;
@@ -1066,8 +1074,8 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           const uint32_t a_dst = tiles + (uint32_t)s * STAGE2_BYTES;
           const uint32_t b_dst = a_dst + A_BYTES;
           tma2_load_2d(a_dst, &map_a, kb * BK, my_row0, lead_full);
-          if (SWIGLU) tma2_load_3d(b_dst, rank == 0 ? &map_b0 : &map_b1, kb * BK, t.n0, t.e, lead_full);
-          else tma2_load_3d(b_dst, &map_b0, kb * BK, t.n0 + (int)rank * 128, t.e, lead_full);
+          if (SWIGLU) tma2_load_3d(b_dst, rank == 0 ? &map_b0 : &map_b1, kb * BK, t.n0, we, lead_full);
+          else tma2_load_3d(b_dst, &map_b0, kb * BK, t.n0 + (int)rank * 128, we, lead_full);
           if (++s == STAGES2) { s = 0; ph ^= 1u; }
         }
       }
@@ -1086,7 +1094,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       for (int j = 0; ok; ++j, ++it) {
         const int tile = next_tile(j, false);
         if (tile < 0) break;
-        if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
+        if (!locate_tile(tile, cursor, tile_start, offs, ends, E, N_TILE, BM2, t)) break;
         const uint32_t b = it & 1u, use = it >> 1;
         if (!mbar_wait(tempty_bar(b), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -1116,7 +1124,7 @@ k_ffn_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     for (int j = 0;; ++j, ++it) {
       const int tile = next_tile(j, true);
       if (tile < 0) break;
-      if (!locate_tile(tile, cursor, tile_start, offs, E, N_TILE, BM2, t)) break;
+      if (!locate_tile(tile, cursor, tile_start, offs, ends, E, N_TILE, BM2, t)) break;
       const uint32_t b = it & 1u, use = it >> 1;
       bool ready = mbar_wait(tfull_bar(b), use & 1u, abort_flag);
       ready = __all_sync(0xffffffffu, ready);
@@ -1248,18 +1256,20 @@ bool ffn_tc_supported(int d, int F, int dtype) {
   return dtype == CAPMOE_BF16 && d % 64 == 0 && F % 64 == 0 && d >= 64 && F >= 64;
 }
 
-int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int F, const void* w_gate,
-           const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max, int D_straggler,
-           int32_t* dev_status, int sched_slot, bool counters_cleared, cudaEvent_t mid, cudaStream_t st) {
+// E row segments [seg_begin[e], seg_end[e]); segment e multiplies with weight block e % w_mod
+// (w_mod = 0: block e) out of n_w blocks.
+int ffn_tc(const void* x_perm, const int32_t* seg_begin, const int32_t* seg_end, int E, int w_mod, int n_w, int d, int F,
+           const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max,
+           int D_straggler, int32_t* dev_status, int sched_slot, bool counters_cleared, cudaEvent_t mid, cudaStream_t st) {
   if (E > MAX_E) return CAPMOE_EUNSUPPORTED;
   alignas(64) CUtensorMap a1, bg, bu, a2, bd, o1, o2;
   if (!make_store_map(&o1, h_ws, (uint64_t)F, (uint64_t)A_max) ||
       !make_store_map(&o2, y_perm, (uint64_t)d, (uint64_t)A_max) ||
       !make_map(&a1, x_perm, (uint64_t)d, (uint64_t)A_max, 0, BM) ||
-      !make_map(&bg, w_gate, (uint64_t)d, (uint64_t)F, (uint64_t)E, 128) ||
-      !make_map(&bu, w_up, (uint64_t)d, (uint64_t)F, (uint64_t)E, 128) ||
+      !make_map(&bg, w_gate, (uint64_t)d, (uint64_t)F, (uint64_t)n_w, 128) ||
+      !make_map(&bu, w_up, (uint64_t)d, (uint64_t)F, (uint64_t)n_w, 128) ||
       !make_map(&a2, h_ws, (uint64_t)F, (uint64_t)A_max, 0, BM) ||
-      !make_map(&bd, w_down, (uint64_t)F, (uint64_t)d, (uint64_t)E, 256))
+      !make_map(&bd, w_down, (uint64_t)F, (uint64_t)d, (uint64_t)n_w, 256))
     return note_cuda(cudaErrorInvalidValue);
   cudaError_t err = cudaFuncSetAttribute(k_ffn_tc<MODE_GATE_UP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          SMEM_BYTES);
@@ -1289,7 +1299,7 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
   if (grid >= 2 && (avg_rows >= 1024 || (avg_rows >= 256 && avg_rows % 256 == 0)) &&
       (D_straggler == 0 || grid / 2 >= D_straggler)) {
     alignas(64) CUtensorMap bd128;
-    if (!make_map(&bd128, w_down, (uint64_t)F, (uint64_t)d, (uint64_t)E, 128)) return note_cuda(cudaErrorInvalidValue);
+    if (!make_map(&bd128, w_down, (uint64_t)F, (uint64_t)d, (uint64_t)n_w, 128)) return note_cuda(cudaErrorInvalidValue);
     int pairs = grid / 2;
     if (D_straggler > 0) pairs = (pairs / D_straggler) * D_straggler;
     err = cudaFuncSetAttribute(k_ffn_tc2<MODE_GATE_UP>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
@@ -1308,13 +1318,13 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_GATE_UP>, a1, bg, bu, o1, expert_offsets, E, d, F,
+    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_GATE_UP>, a1, bg, bu, o1, seg_begin, seg_end, w_mod, E, d, F,
                              (__nv_bfloat16*)h_ws, D_straggler, dev_status, sched1);
     count_launch(1);
     if (err != cudaSuccess) return note_cuda(err);
     int rc2;
     if (mid && (rc2 = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc2;
-    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_DOWN>, a2, bd128, bd128, o2, expert_offsets, E, F, d,
+    err = cudaLaunchKernelEx(&cfg, k_ffn_tc2<MODE_DOWN>, a2, bd128, bd128, o2, seg_begin, seg_end, w_mod, E, F, d,
                              (__nv_bfloat16*)y_perm, D_straggler, dev_status, sched2);
     count_launch(1);
     return note_cuda(err);
@@ -1324,13 +1334,13 @@ int ffn_tc(const void* x_perm, const int32_t* expert_offsets, int E, int d, int 
     grid = (grid / D_straggler) * D_straggler;          // equal share of SMs per virtual device
   }
   int rc = note_cuda(launch_chained(k_ffn_tc<MODE_GATE_UP, 32>, (unsigned)grid, TC_THREADS, SMEM_BYTES, st, a1, bg, bu, o1,
-                                    expert_offsets, E, d, F, h_ws, D_straggler, dev_status, BNB, 0,
+                                    seg_begin, seg_end, w_mod, E, d, F, h_ws, D_straggler, dev_status, BNB, 0,
                                     (const float*)nullptr, BM, STAGES, STAGE_BYTES, RouterFused{}, sched1));
   count_launch(1);
   if (rc != CAPMOE_OK) return rc;
   if (mid && (rc = note_cuda(cudaEventRecord(mid, st))) != CAPMOE_OK) return rc;
   rc = note_cuda(launch_chained(k_ffn_tc<MODE_DOWN, 32>, (unsigned)grid, TC_THREADS, SMEM_BYTES, st, a2, bd, bd, o2,
-                                expert_offsets, E, F, d, y_perm, D_straggler, dev_status, BNB, 0,
+                                seg_begin, seg_end, w_mod, E, F, d, y_perm, D_straggler, dev_status, BNB, 0,
                                 (const float*)nullptr, BM, STAGES, STAGE_BYTES, RouterFused{}, sched2));
   count_launch(1);
   return rc;
@@ -1350,8 +1360,8 @@ static int launch_router_tc(const CUtensorMap& ax, const CUtensorMap& bw, int gr
   if (err != cudaSuccess) return note_cuda(err);
   // (the fourth tensor map is the FFN modes' output map: unused here)
   k_ffn_tc<MODE, EPAD><<<grid, MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, SMEM_BYTES, st>>>(
-      ax, bw, bw, bw, nullptr, 1, d, E, logits, 0, nullptr, n_mma, (int)N, bias, tile_rows, n_stages, stage_stride, rf,
-      nullptr);
+      ax, bw, bw, bw, nullptr, nullptr, 0, 1, d, E, logits, 0, nullptr, n_mma, (int)N, bias, tile_rows, n_stages,
+      stage_stride, rf, nullptr);
   return check_launch();
 }
 

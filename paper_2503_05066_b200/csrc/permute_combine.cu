@@ -13,12 +13,27 @@ constexpr int VPL = 4;               // 16-byte vectors per lane per unit
 constexpr int CHUNK_VECS = 32 * VPL; // vectors per unit (2 KB)
 constexpr int MAX_SLOTS = 288;       // k + m <= 32 + 256
 
+// Where a row of the permuted matrix lives when the matrix is spread over the ranks of an
+// expert-parallel group: rows [p*rows_per_peer, (p+1)*rows_per_peer) belong to rank p and sit in
+// that rank's buffer (base address table[p]) from row `row0` on, the block this rank owns there.
+// table == NULL: one local matrix.
+struct PeerRows {
+  const unsigned long long* table;
+  int rows_per_peer, row0;
+};
+__device__ __forceinline__ uint4* peer_row(const PeerRows& pr, uint4* local_base, int32_t r, int row_vecs) {
+  if (!pr.table) return local_base + (int64_t)r * row_vecs;
+  const int p = r / pr.rows_per_peer, i = r - p * pr.rows_per_peer;
+  return reinterpret_cast<uint4*>(pr.table[p]) + (int64_t)(pr.row0 + i) * row_vecs;
+}
+
 __global__ void __launch_bounds__(PC_WARPS * 32)
 k_permute(const uint4* __restrict__ x, int64_t N, int row_vecs /* 16-byte vectors per row */, int chunks, int E,
           int k, int slots, int D, const float* __restrict__ scores, const int32_t* __restrict__ topk_idx,
           const int32_t* __restrict__ token_group, const int32_t* __restrict__ slot_row,
           uint4* __restrict__ x_perm, int32_t* __restrict__ perm_token, float* __restrict__ perm_weight,
-          unsigned long long* __restrict__ keep_mask /* NULL, or [N, ceil(E/64)] to be derived from slot_row here */) {
+          unsigned long long* __restrict__ keep_mask /* NULL, or [N, ceil(E/64)] to be derived from slot_row here */,
+          const PeerRows peers) {
   allow_next_kernel();
   wait_for_previous_kernel();
   const int lane = threadIdx.x & 31;
@@ -71,7 +86,7 @@ k_permute(const uint4* __restrict__ x, int64_t N, int row_vecs /* 16-byte vector
       const int b = __ffs(rem) - 1;
       rem &= rem - 1;
       const int32_t r = __shfl_sync(0xffffffffu, mine, b);
-      uint4* dst = x_perm + (int64_t)r * row_vecs + v0;
+      uint4* dst = peer_row(peers, x_perm, r, row_vecs) + v0;
 #pragma unroll
       for (int u = 0; u < VPL; ++u)
         if (v0 + u * 32 < row_vecs) dst[u * 32] = val[u];
@@ -126,7 +141,7 @@ template <typename T>
 __global__ void __launch_bounds__(PC_WARPS * 32, 4)
 k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row,
           const float* __restrict__ perm_weight, int64_t N, int row_vecs, int chunks, int slots,
-          const uint4* __restrict__ y_shared, uint4* __restrict__ y) {
+          const uint4* __restrict__ y_shared, uint4* __restrict__ y, const PeerRows peers) {
   allow_next_kernel();
   wait_for_previous_kernel();
   constexpr int NV = Vec16<T>::n;
@@ -157,8 +172,8 @@ k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row
       rem &= rem - 1;                                  // no-op when rem is already 0
       const int32_t r0 = __shfl_sync(0xffffffffu, mine, b0), r1 = __shfl_sync(0xffffffffu, mine, b1);
       const float w0 = __shfl_sync(0xffffffffu, wmine, b0), w1 = __shfl_sync(0xffffffffu, wmine, b1);
-      const uint4* p0 = y_perm + (int64_t)r0 * row_vecs + v0;
-      const uint4* p1 = y_perm + (int64_t)r1 * row_vecs + v0;
+      const uint4* p0 = peer_row(peers, const_cast<uint4*>(y_perm), r0, row_vecs) + v0;
+      const uint4* p1 = peer_row(peers, const_cast<uint4*>(y_perm), r1, row_vecs) + v0;
       uint4 raw0[VPL], raw1[VPL];
 #pragma unroll
       for (int u = 0; u < VPL; ++u) {                  // all loads first, arithmetic after
@@ -180,10 +195,11 @@ k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_row
 
 using namespace capmoe;
 
-int capmoe::permute_impl(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
-                         const float* scores, const int32_t* topk_idx, const int32_t* token_group,
-                         const int32_t* slot_row, void* x_perm, int32_t* perm_token, float* perm_weight,
-                         uint64_t* keep_mask_out, void* stream) {
+namespace capmoe {
+namespace {
+int permute_rows(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype, const float* scores,
+                 const int32_t* topk_idx, const int32_t* token_group, const int32_t* slot_row, void* x_perm,
+                 int32_t* perm_token, float* perm_weight, uint64_t* keep_mask_out, const PeerRows& peers, void* stream) {
   if (N < 0 || d < 1 || E < 1 || k < 1 || k > E || slots < k || D < 0) return CAPMOE_EINVAL;
   if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
   if (D > 0 && (E % D != 0 || slots != k + E / D)) return CAPMOE_EINVAL;
@@ -191,7 +207,8 @@ int capmoe::permute_impl(const void* x, int64_t N, int d, int E, int k, int slot
   if (slots > MAX_SLOTS) return CAPMOE_EUNSUPPORTED;
   if (((size_t)d * elt_size(dtype)) % 16 != 0) return CAPMOE_EUNSUPPORTED;
   if (N == 0) return CAPMOE_OK;
-  if (!x || !scores || !topk_idx || !slot_row || !x_perm || !perm_token || !perm_weight) return CAPMOE_EINVAL;
+  if (!x || !scores || !topk_idx || !slot_row || (!x_perm && !peers.table) || !perm_token || !perm_weight)
+    return CAPMOE_EINVAL;
   if (!aligned16(x) || !aligned16(x_perm)) return CAPMOE_EINVAL;
   const int row_vecs = (int)((size_t)d * elt_size(dtype) / 16);
   const int chunks = (row_vecs + CHUNK_VECS - 1) / CHUNK_VECS;
@@ -200,21 +217,13 @@ int capmoe::permute_impl(const void* x, int64_t N, int d, int E, int k, int slot
   const int rc = note_cuda(launch_chained(k_permute, (unsigned)blocks, PC_WARPS * 32, 0, as_stream(stream),
                                           (const uint4*)x, N, row_vecs, chunks, E, k, slots, D, scores, topk_idx,
                                           token_group, slot_row, (uint4*)x_perm, perm_token, perm_weight,
-                                          reinterpret_cast<unsigned long long*>(keep_mask_out)));
+                                          reinterpret_cast<unsigned long long*>(keep_mask_out), peers));
   count_launch(1);
   return rc;
 }
 
-extern "C" int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
-                              const float* scores, const int32_t* topk_idx, const int32_t* token_group,
-                              const int32_t* slot_row, void* x_perm, int32_t* perm_token, float* perm_weight,
-                              void* stream) {
-  return permute_impl(x, N, d, E, k, slots, D, dtype, scores, topk_idx, token_group, slot_row, x_perm, perm_token,
-                      perm_weight, nullptr, stream);
-}
-
-extern "C" int capmoe_combine(const void* y_perm, const int32_t* slot_row, const float* perm_weight, int64_t N,
-                              int d, int slots, int dtype, const void* y_shared, void* y, void* stream) {
+int combine_rows(const void* y_perm, const int32_t* slot_row, const float* perm_weight, int64_t N, int d, int slots,
+                 int dtype, const void* y_shared, void* y, const PeerRows& peers, void* stream) {
   if (N < 0 || d < 1 || slots < 1) return CAPMOE_EINVAL;
   if (dtype != CAPMOE_F32 && dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
   if (slots > MAX_SLOTS) return CAPMOE_EUNSUPPORTED;
@@ -230,10 +239,131 @@ extern "C" int capmoe_combine(const void* y_perm, const int32_t* slot_row, const
   cudaError_t err;
   if (dtype == CAPMOE_F32)
     err = launch_chained(k_combine<float>, (unsigned)blocks, PC_WARPS * 32, 0, st, (const uint4*)y_perm, slot_row,
-                         perm_weight, N, row_vecs, chunks, slots, (const uint4*)y_shared, (uint4*)y);
+                         perm_weight, N, row_vecs, chunks, slots, (const uint4*)y_shared, (uint4*)y, peers);
   else
     err = launch_chained(k_combine<__nv_bfloat16>, (unsigned)blocks, PC_WARPS * 32, 0, st, (const uint4*)y_perm,
-                         slot_row, perm_weight, N, row_vecs, chunks, slots, (const uint4*)y_shared, (uint4*)y);
+                         slot_row, perm_weight, N, row_vecs, chunks, slots, (const uint4*)y_shared, (uint4*)y, peers);
   count_launch(1);
   return note_cuda(err);
+}
+
+// Expert parallelism, bookkeeping kernels (see capmoe_ep_plan / capmoe_ep_segments in the header).
+__global__ void __launch_bounds__(256)
+k_ep_plan(const int32_t* __restrict__ slot_row, const int32_t* __restrict__ topk_idx,
+          const int32_t* __restrict__ expert_offsets, int64_t N, int E, int k, int slots, int D,
+          const int32_t* __restrict__ token_group, int C_local, int32_t* __restrict__ slot_row_ep,
+          int32_t* __restrict__ bad) {
+  allow_next_kernel();
+  wait_for_previous_kernel();
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= N * slots) return;
+  const int64_t t = i / slots;
+  const int s = (int)(i - t * slots);
+  const int32_t r = slot_row[i];
+  int32_t out = -1;
+  if (r >= 0) {
+    const int m = slots > k ? E / D : 0;
+    const int e = s < k ? topk_idx[t * k + s] : home_group(t, N, D, token_group) * m + (s - k);
+    const int32_t within = r - expert_offsets[e];
+    if (within < 0 || within >= C_local) *bad = 1;           // more rows on an expert than its capacity allows
+    else out = e * C_local + within;
+  }
+  slot_row_ep[i] = out;
+}
+
+__global__ void __launch_bounds__(256)
+k_ep_segments(const int32_t* __restrict__ counts, int S, int C_local, int32_t* __restrict__ seg_begin,
+              int32_t* __restrict__ seg_end) {
+  allow_next_kernel();
+  wait_for_previous_kernel();
+  const int s = blockIdx.x * 256 + threadIdx.x;
+  if (s >= S) return;
+  const int c = counts[s];
+  seg_begin[s] = s * C_local;
+  seg_end[s] = s * C_local + (c < 0 ? 0 : (c > C_local ? C_local : c));
+}
+
+}  // namespace
+}  // namespace capmoe
+
+int capmoe::permute_impl(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
+                         const float* scores, const int32_t* topk_idx, const int32_t* token_group,
+                         const int32_t* slot_row, void* x_perm, int32_t* perm_token, float* perm_weight,
+                         uint64_t* keep_mask_out, void* stream) {
+  return permute_rows(x, N, d, E, k, slots, D, dtype, scores, topk_idx, token_group, slot_row, x_perm, perm_token,
+                      perm_weight, keep_mask_out, PeerRows{nullptr, 0, 0}, stream);
+}
+
+extern "C" int capmoe_permute(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
+                              const float* scores, const int32_t* topk_idx, const int32_t* token_group,
+                              const int32_t* slot_row, void* x_perm, int32_t* perm_token, float* perm_weight,
+                              void* stream) {
+  return permute_impl(x, N, d, E, k, slots, D, dtype, scores, topk_idx, token_group, slot_row, x_perm, perm_token,
+                      perm_weight, nullptr, stream);
+}
+
+extern "C" int capmoe_combine(const void* y_perm, const int32_t* slot_row, const float* perm_weight, int64_t N,
+                              int d, int slots, int dtype, const void* y_shared, void* y, void* stream) {
+  return combine_rows(y_perm, slot_row, perm_weight, N, d, slots, dtype, y_shared, y, PeerRows{nullptr, 0, 0}, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Expert parallelism with per-rank capacity (entry points documented in capmoe.h).
+namespace {
+int check_ep(int R, int rank, int E, int64_t C_local) {
+  if (R < 1 || rank < 0 || rank >= R || E < 1 || E % R != 0 || C_local < 0) return CAPMOE_EINVAL;
+  if ((int64_t)E * C_local >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  return CAPMOE_OK;
+}
+}  // namespace
+
+extern "C" int capmoe_ep_plan(const int32_t* slot_row, const int32_t* topk_idx, const int32_t* expert_offsets, int64_t N,
+                              int E, int k, int slots, int D, const int32_t* token_group, int64_t C_local,
+                              int32_t* slot_row_ep, int32_t* bad, void* stream) {
+  if (N < 0 || E < 1 || k < 1 || k > E || slots < k || C_local < 0) return CAPMOE_EINVAL;
+  if (slots > k && (D < 1 || E % D != 0 || slots != k + E / D)) return CAPMOE_EINVAL;
+  if ((int64_t)E * C_local >= ((int64_t)1 << 31) || N * (int64_t)slots >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  if (N == 0) return CAPMOE_OK;
+  if (!slot_row || !topk_idx || !expert_offsets || !slot_row_ep || !bad) return CAPMOE_EINVAL;
+  const int rc = note_cuda(launch_chained(k_ep_plan, (unsigned)ceil_div(N * slots, 256), 256, 0, as_stream(stream),
+                                          slot_row, topk_idx, expert_offsets, N, E, k, slots, D < 1 ? 1 : D, token_group,
+                                          (int)C_local, slot_row_ep, bad));
+  count_launch(1);
+  return rc;
+}
+
+extern "C" int capmoe_ep_segments(const int32_t* counts, int S, int64_t C_local, int32_t* seg_begin, int32_t* seg_end,
+                                  void* stream) {
+  if (S < 1 || C_local < 0 || (int64_t)S * C_local >= ((int64_t)1 << 31)) return CAPMOE_EINVAL;
+  if (!counts || !seg_begin || !seg_end) return CAPMOE_EINVAL;
+  const int rc = note_cuda(launch_chained(k_ep_segments, (unsigned)ceil_div(S, 256), 256, 0, as_stream(stream), counts, S,
+                                          (int)C_local, seg_begin, seg_end));
+  count_launch(1);
+  return rc;
+}
+
+extern "C" int capmoe_ep_dispatch(const void* x, int64_t N, int d, int E, int k, int slots, int D, int dtype,
+                                  const float* scores, const int32_t* topk_idx, const int32_t* token_group,
+                                  const int32_t* slot_row_ep, const uint64_t* peer_rows, int R, int rank,
+                                  int64_t C_local, int32_t* perm_token, float* perm_weight, void* stream) {
+  const int rc = check_ep(R, rank, E, C_local);
+  if (rc != CAPMOE_OK) return rc;
+  if (!peer_rows) return CAPMOE_EINVAL;
+  const int per = (int)((E / R) * C_local);
+  return permute_rows(x, N, d, E, k, slots, D, dtype, scores, topk_idx, token_group, slot_row_ep, nullptr, perm_token,
+                      perm_weight, nullptr,
+                      PeerRows{reinterpret_cast<const unsigned long long*>(peer_rows), per > 0 ? per : 1, rank * per},
+                      stream);
+}
+
+extern "C" int capmoe_ep_combine(const uint64_t* peer_rows, int R, int rank, int E, int64_t C_local,
+                                 const int32_t* slot_row_ep, const float* perm_weight, int64_t N, int d, int slots,
+                                 int dtype, const void* y_shared, void* y, void* stream) {
+  const int rc = check_ep(R, rank, E, C_local);
+  if (rc != CAPMOE_OK) return rc;
+  if (!peer_rows) return CAPMOE_EINVAL;
+  const int per = (int)((E / R) * C_local);
+  return combine_rows(nullptr, slot_row_ep, perm_weight, N, d, slots, dtype, y_shared, y,
+                      PeerRows{reinterpret_cast<const unsigned long long*>(peer_rows), per > 0 ? per : 1, rank * per},
+                      stream);
 }
