@@ -25,6 +25,24 @@ int check_launch() {
   return note_cuda(cudaPeekAtLastError());
 }
 
+namespace {
+__global__ void __launch_bounds__(256) k_clear_words(int32_t* __restrict__ a, int na, int32_t* __restrict__ b, int nb) {
+  allow_next_kernel();
+  wait_for_previous_kernel();
+  for (int i = threadIdx.x; i < na; i += 256) a[i] = 0;
+  for (int i = threadIdx.x; i < nb; i += 256) b[i] = 0;
+}
+}  // namespace
+
+int clear_words(int32_t* a, int na, int32_t* b, int nb, cudaStream_t st) {
+  if (!a) na = 0;
+  if (!b) nb = 0;
+  if (na <= 0 && nb <= 0) return CAPMOE_OK;
+  const int rc = note_cuda(launch_chained(k_clear_words, 1u, 256u, 0, st, a, na, b, nb));
+  count_launch(1);
+  return rc;
+}
+
 int sm_count() {
   static int cached[64];
   int dev = 0;
@@ -254,12 +272,11 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
   if (rc != CAPMOE_OK) return rc;
   // The tile counters of all FFN launches of this forward are cleared here, away from the kernels
   // that use them, so that no memset sits between the permute and the first GEMM.
-  if (L->dev_status) {
-    rc = note_cuda(cudaMemsetAsync(L->dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st));
-    if (rc != CAPMOE_OK) return rc;
-  }
-  // Likewise the load histogram and the drop stage's counters; the stages are told so below.
-  if ((rc = note_cuda(cudaMemsetAsync(L->load, 0, sizeof(int32_t) * L->E, st))) != CAPMOE_OK) return rc;
+  // Likewise the load histogram (one small kernel for both) and the drop stage's counters; the
+  // stages are told so below.
+  if ((rc = clear_words(L->dev_status ? L->dev_status + 1 : nullptr, CAPMOE_FFN_STATUS_WORDS - 1, L->load, L->E, st)) !=
+      CAPMOE_OK)
+    return rc;
   if ((rc = drop_clear_counters(L->mode, L->N, L->E, L->k, L->D < 1 ? 1 : L->D, L->cand, L->drop_ws, L->drop_ws_bytes,
                                 st)) != CAPMOE_OK)
     return rc;

@@ -89,6 +89,10 @@ inline cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsig
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Zeroes up to two small int32 arrays with one chained kernel launch (a memset node between two
+// kernels costs more stream time than this and breaks the chain of overlapped launches).
+int clear_words(int32_t* a, int na, int32_t* b, int nb, cudaStream_t st);
+
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <typename T> __device__ __forceinline__ T from_float(float v);

@@ -28,6 +28,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "mbarrier.cuh"
 #include "softmax.cuh"
 
 namespace capmoe {
@@ -60,47 +61,8 @@ constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STG_BYTES + 1024 /*alignment s
                            2 * (MAX_E + 1) * 4 + 8 + 256 * 4 /*router bias*/ + RF_XCH_FLOATS * 4 + MAX_E * 4 /*segment ends*/;
 static_assert(SMEM_BYTES <= 227 * 1024, "dynamic shared memory limit of a thread block");
 static_assert(RF_SPREAD_ROWS * 64 * 4 <= STG_BYTES, "the fused router's shared logits tile lives in the staging area");
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the wait ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          long long limit_cycles = WAIT_LIMIT_CYCLES) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t it = 1; it < 0x40000000u; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 127u) == 0u) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > limit_cycles) break;
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
-
+// ---------------------------------------------------------------- PTX wrappers (mbarriers: mbarrier.cuh)
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -1290,8 +1252,8 @@ int ffn_tc(const void* x_perm, const int32_t* seg_begin, const int32_t* seg_end,
     sched2 = sched1 + 1;
   }
   if (sched1 && !counters_cleared) {
-    err = cudaMemsetAsync(dev_status + 1, 0, sizeof(int32_t) * (CAPMOE_FFN_STATUS_WORDS - 1), st);
-    if (err != cudaSuccess) return note_cuda(err);
+    const int rc0 = clear_words(dev_status + 1, CAPMOE_FFN_STATUS_WORDS - 1, nullptr, 0, st);
+    if (rc0 != CAPMOE_OK) return rc0;
   }
   // CTA pairs (256-row tiles) when the expert segments are long enough that the extra tail
   // padding does not matter, or are known multiples of 256 rows
@@ -1359,10 +1321,13 @@ static int launch_router_tc(const CUtensorMap& ax, const CUtensorMap& bw, int gr
                                          SMEM_BYTES);
   if (err != cudaSuccess) return note_cuda(err);
   // (the fourth tensor map is the FFN modes' output map: unused here)
-  k_ffn_tc<MODE, EPAD><<<grid, MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, SMEM_BYTES, st>>>(
-      ax, bw, bw, bw, nullptr, nullptr, 0, 1, d, E, logits, 0, nullptr, n_mma, (int)N, bias, tile_rows, n_stages,
-      stage_stride, rf, nullptr);
-  return check_launch();
+  const int rc = note_cuda(launch_chained(k_ffn_tc<MODE, EPAD>, (unsigned)grid,
+                                          MODE == MODE_ROUTER_FUSED ? RF_THREADS : TC_THREADS, SMEM_BYTES, st, ax, bw, bw, bw,
+                                          (const int32_t*)nullptr, (const int32_t*)nullptr, 0, 1, d, E, (void*)logits, 0,
+                                          (int32_t*)nullptr, n_mma, (int)N, bias, tile_rows, n_stages, stage_stride, rf,
+                                          (int32_t*)nullptr));
+  count_launch(1);
+  return rc;
 }
 
 int router_tc(const void* x, const void* w_router, const float* bias, int64_t N, int d, int E, float* logits,

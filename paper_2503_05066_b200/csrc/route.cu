@@ -1,6 +1,4 @@
 // Stage 1: router GEMM, softmax, per-token top-k, expert load histogram (Eq. 1, Eq. 3).
-#include <cstdlib>
-
 #include "common.cuh"
 #include "softmax.cuh"
 
@@ -18,6 +16,7 @@ __global__ void __launch_bounds__(RT_TOK* RT_EG)
 k_router_gemm(const T* __restrict__ x, const T* __restrict__ w, const float* __restrict__ bias,
               int64_t N, int d, int E, float* __restrict__ logits) {
   allow_next_kernel();
+  wait_for_previous_kernel();
   extern __shared__ float smem[];
   float* xs = smem;                              // [RT_TOK][RT_BK+1]
   float* wsm = smem + RT_TOK * (RT_BK + 1);      // [E][RT_BK+1]
@@ -135,6 +134,7 @@ __global__ void __launch_bounds__(SW_WARPS * 32)
 k_softmax_topk_warp(const float* __restrict__ logits, int64_t N, int E, int k, float* __restrict__ scores,
                     int32_t* __restrict__ topk_idx, float* __restrict__ topk_score, int32_t* __restrict__ load) {
   allow_next_kernel();
+  wait_for_previous_kernel();
   extern __shared__ float smem[];
   float* prow = smem + (threadIdx.x >> 5) * (EPL * 32);       // this warp's E exponentials
   int* hist = reinterpret_cast<int*>(smem + SW_WARPS * EPL * 32);
@@ -155,9 +155,10 @@ int launch_softmax_warp(const float* lg, int64_t N, int E, int k, float* scores,
   int64_t blocks = ceil_div(N, SW_WARPS);
   const int64_t cap = (int64_t)sm_count() * 8;                 // resident CTAs; more tokens loop inside
   if (blocks > cap) blocks = cap;
-  k_softmax_topk_warp<EPL><<<(unsigned)blocks, SW_WARPS * 32, smem, st>>>(lg, N, E, k, scores, topk_idx,
-                                                                          topk_score, load);
-  return check_launch();
+  const int rc = note_cuda(launch_chained(k_softmax_topk_warp<EPL>, (unsigned)blocks, SW_WARPS * 32, smem, st, lg, N, E, k,
+                                          scores, topk_idx, topk_score, load));
+  count_launch(1);
+  return rc;
 }
 
 template <typename T>
@@ -166,6 +167,7 @@ int launch_gemm(const T* x, const T* w, const float* bias, int64_t N, int d, int
   const int ept = (E + RT_EG - 1) / RT_EG;
   const size_t smem = (size_t)(RT_TOK + E) * (RT_BK + 1) * sizeof(float);
   const dim3 grid((unsigned)ceil_div(N, RT_TOK)), block(RT_TOK * RT_EG);
+  cudaError_t launch_err = cudaSuccess;
 #define CAPMOE_RT_CASE(EPT)                                                                      \
   {                                                                                              \
     if (smem > 48 * 1024) {                                                                      \
@@ -173,7 +175,7 @@ int launch_gemm(const T* x, const T* w, const float* bias, int64_t N, int d, int
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
       if (e_ != cudaSuccess) return note_cuda(e_);                                               \
     }                                                                                            \
-    k_router_gemm<T, EPT><<<grid, block, smem, st>>>(x, w, bias, N, d, E, logits);               \
+    launch_err = launch_chained(k_router_gemm<T, EPT>, grid.x, block.x, smem, st, x, w, bias, N, d, E, logits); \
   }
   if (ept <= 1) CAPMOE_RT_CASE(1)
   else if (ept <= 2) CAPMOE_RT_CASE(2)
@@ -182,7 +184,8 @@ int launch_gemm(const T* x, const T* w, const float* bias, int64_t N, int d, int
   else if (ept <= 16) CAPMOE_RT_CASE(16)
   else CAPMOE_RT_CASE(32)
 #undef CAPMOE_RT_CASE
-  return check_launch();
+  count_launch(1);
+  return note_cuda(launch_err);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -221,6 +224,7 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
              float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
              int32_t* __restrict__ load) {
   allow_next_kernel();
+  wait_for_previous_kernel();
   extern __shared__ float red[];                       // [RM_WARPS][16*MT][NT*8 + 1] (+ fused scratch)
   constexpr int ROWS = 16 * MT, EP = NT * 8, LD = EP + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -318,11 +322,10 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
   }
 }
 
+struct RouteOut { int k; float* scores; int32_t* topk_idx; float* topk_score; int32_t* load; };
+
 bool router_mma_ok(int d, int E) { return d % (RM_WARPS * 64) == 0 && E <= 128; }
 
-inline int dbg_tc_min_e() { static int v = getenv("CAPMOE_DEBUG_TC_MIN_E") ? atoi(getenv("CAPMOE_DEBUG_TC_MIN_E")) : 17; return v; }
-
-struct RouteOut { int k; float* scores; int32_t* topk_idx; float* topk_score; int32_t* load; };
 
 template <int MT, int NT, bool FUSED>
 int launch_router_mma_inst(const __nv_bfloat16* x, const __nv_bfloat16* w, const float* bias, int64_t N, int d,
@@ -334,9 +337,11 @@ int launch_router_mma_inst(const __nv_bfloat16* x, const __nv_bfloat16* w, const
                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e_ != cudaSuccess) return note_cuda(e_);
   }
-  k_router_mma<MT, NT, FUSED><<<(unsigned)ceil_div(N, 16 * MT), RM_WARPS * 32, smem, st>>>(
-      x, w, bias, N, d, E, logits, o.k, o.scores, o.topk_idx, o.topk_score, o.load);
-  return check_launch();
+  const int rc = note_cuda(launch_chained(k_router_mma<MT, NT, FUSED>, (unsigned)ceil_div(N, 16 * MT), RM_WARPS * 32, smem,
+                                          st, x, w, bias, N, d, E, logits, o.k, o.scores, o.topk_idx, o.topk_score,
+                                          o.load));
+  count_launch(1);
+  return rc;
 }
 
 // fused = true: the kernel also produced scores, top-k and the load histogram.
@@ -370,8 +375,10 @@ int capmoe::route_impl(const void* x, const void* w_router, const float* bias, c
   if (N * (int64_t)E >= (int64_t)1 << 40) return CAPMOE_EUNSUPPORTED;
   cudaStream_t st = as_stream(stream);
   cudaError_t err = cudaSuccess;
-  if (!load_cleared) err = cudaMemsetAsync(load, 0, sizeof(int32_t) * E, st);
-  if (err != cudaSuccess) return note_cuda(err);
+  if (!load_cleared) {
+    const int rc0 = clear_words(load, E, nullptr, 0, st);
+    if (rc0 != CAPMOE_OK) return rc0;
+  }
   if (N == 0) return CAPMOE_OK;
   const float* lg = logits_in;
   if (!logits_in) {
@@ -380,7 +387,7 @@ int capmoe::route_impl(const void* x, const void* w_router, const float* bias, c
     const RouteOut ro{k, scores, topk_idx, topk_score, load};
     if (dtype == CAPMOE_F32)
       rc = launch_gemm<float>((const float*)x, (const float*)w_router, bias, N, d, E, logits, st);
-    else if (E >= dbg_tc_min_e() && router_tc_supported(N, d, E) && aligned16(x) && aligned16(w_router)) {
+    else if (E > 16 && router_tc_supported(N, d, E) && aligned16(x) && aligned16(w_router)) {
       fused = router_tc_fusable(E, k);
       rc = router_tc(x, w_router, bias, N, d, E, logits, scores, topk_idx, topk_score, load, k, fused, st);
     }
