@@ -548,15 +548,26 @@ def main():
         reps = 24
 
         def timed(fn):
-            for i in range(4):
+            """ms per call of fn(i), i = 0..reps-1, replayed from one CUDA graph: device time of the
+            stage's launches back to back, without the host's per-call cost (which exceeds the
+            duration of the shortest of these kernels)."""
+            for i in range(2):
                 fn(i)
+            torch.cuda.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.graph(gr, stream=side):
+                for i in range(reps):
+                    fn(i)
+            gr.replay()
             torch.cuda.synchronize()
             e0.record()
-            for i in range(reps):
-                fn(i)
+            for _ in range(3):
+                gr.replay()
             e1.record()
             torch.cuda.synchronize()
-            return e0.elapsed_time(e1) / reps
+            return e0.elapsed_time(e1) / (3 * reps)
 
         t = layer.t
         ncopy = max(2, int(200e6 // (cfg.N * cfg.d * elt)) + 1)
@@ -564,6 +575,8 @@ def main():
         r_out = capmoe.route(g["x"], g["w_router"], g["bias"], cfg.k)
         ms = timed(lambda i: capmoe.route(xs[i % ncopy], g["w_router"], g["bias"], cfg.k, out=r_out))
         hbm_kernels["route"] = ms
+        # what a kernel that only reads the same activations once would take (launch included)
+        route_floor_ms = timed(lambda i: capmoe.debug_read_probe(xs[i % ncopy]))
         A_rows = t["x_perm"].shape[0]
         pcopy = max(2, int(200e6 // (A_rows * cfg.d * elt)) + 1)
         p_outs = [dict(x_perm=torch.empty_like(t["x_perm"]), perm_token=torch.empty_like(t["perm_token"]),
@@ -579,6 +592,10 @@ def main():
         hbm_kernels = {k: {"ms": v, "bytes": hbm[k], "GB/s": hbm[k] / (v * 1e-3) / 1e9,
                            "frac_of_measured_copy": hbm[k] / (v * 1e-3) / 1e9 / peaks["hbm_gbs"]}
                        for k, v in hbm_kernels.items()}
+        hbm_kernels["route"]["one_shot_read_floor_ms"] = route_floor_ms
+        hbm_kernels["route"]["frac_of_read_floor"] = route_floor_ms / hbm_kernels["route"]["ms"]
+        hbm_kernels["route"]["read_floor_frac_of_measured_copy"] = (cfg.N * cfg.d * elt / (route_floor_ms * 1e-3) / 1e9 /
+                                                                    peaks["hbm_gbs"])
         del xs, p_outs, ys, y_outs
 
     # The drop stage moves a few MB: it is bound by launch and dependency latency, not by bandwidth.

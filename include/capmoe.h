@@ -318,6 +318,13 @@ int capmoe_ep_combine(const uint64_t* peer_rows, int R, int rank, int E, int64_t
  * (the caller zeroes it first).  The context stays usable. */
 int capmoe_debug_wait_probe(int64_t limit_cycles, int32_t* dev_status, void* stream);
 
+/* Measurement aid (no counterpart in the paper): one launch that reads `bytes` bytes from p once,
+ * as fast as plain loads go, and does nothing else.  Its device time is the floor for any kernel
+ * that has to read that much from HBM once, launch included - for the few ten megabytes of a small
+ * batch that floor is well below the bandwidth of a long copy, which is what the bandwidth-bound
+ * stages are otherwise compared with.  p: device, 16-byte aligned; sink: device int32 or NULL. */
+int capmoe_debug_read_probe(const void* p, size_t bytes, int32_t* sink, void* stream);
+
 /* ---------------------------------------------------------------- stage 6: combine
  * y[t] = sum over slots s with slot_row[t,s] >= 0 of perm_weight[row] * y_perm[row], added in
  * ascending slot order in fp32, plus y_shared[t] (weight 1) when y_shared is not NULL; a token

@@ -30,7 +30,7 @@ EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_device_max_rows", "capm
            "capmoe_rows_from_mask", "capmoe_permute", "capmoe_grouped_ffn",
            "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe",
            "capmoe_grouped_ffn_segments", "capmoe_ep_plan", "capmoe_ep_segments", "capmoe_ep_dispatch",
-           "capmoe_ep_combine"]
+           "capmoe_ep_combine", "capmoe_debug_read_probe"]
 
 
 class CapmoeError(RuntimeError):
@@ -444,6 +444,12 @@ def combine(y_perm, slot_row, perm_weight, y_shared=None, y=None, stream=None):
     _check(lib().capmoe_combine(_ptr(y_perm), _ptr(slot_row), _ptr(perm_weight), _i64(N), int(d), int(slots),
                                 _dt(y_perm), _ptr(y_shared), _ptr(y), _stream(stream)), "capmoe_combine")
     return y
+
+
+def debug_read_probe(t: torch.Tensor, stream=None):
+    """One plain pass of loads over the tensor's bytes (the one-shot read floor of that size)."""
+    _check(lib().capmoe_debug_read_probe(_ptr(t), ctypes.c_size_t(t.numel() * t.element_size()), ctypes.c_void_p(0),
+                                         _stream(stream)), "capmoe_debug_read_probe")
 
 
 def debug_wait_probe(limit_cycles: int = 50_000_000, stream=None) -> int:

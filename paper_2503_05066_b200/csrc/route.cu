@@ -129,6 +129,46 @@ __device__ __forceinline__ void softmax_topk_token(const float* lrow, int E, int
   }
 }
 
+// The same for few experts (E <= G <= 16): G lanes per token, 32 / G tokens per warp side by side,
+// so that a short list of tokens is one step deep.  Lane e of a group holds expert e; the sum is
+// still taken left to right (every lane walks the group's exponentials in order), the arg-max
+// rounds are butterflies on (score, lower expert id) inside the group.
+template <int G>
+__device__ __forceinline__ void softmax_topk_group(const float* lrow, bool active, int E, int k, int64_t t,
+                                                   float* __restrict__ scores, int32_t* __restrict__ topk_idx,
+                                                   float* __restrict__ topk_score, int* hist) {
+  const int lane = threadIdx.x & 31, e = lane & (G - 1), first = lane & ~(G - 1);
+  const bool mine = active && e < E;
+  const float v = mine ? lrow[e] : -INFINITY;
+  float mx = v;
+#pragma unroll
+  for (int o = G / 2; o > 0; o >>= 1) {
+    const float other = __shfl_xor_sync(0xffffffffu, mx, o);
+    mx = other > mx ? other : mx;
+  }
+  const float p = mine ? exp_fixed(__fsub_rn(v, mx)) : 0.f;
+  float sum = 0.f;
+  for (int j = 0; j < E; ++j) sum = __fadd_rn(sum, __shfl_sync(0xffffffffu, p, first + j));
+  float cur = mine ? __fdiv_rn(p, sum) : -1.f;                   // never selected (scores are >= 0)
+  if (mine) scores[t * E + e] = cur;
+  for (int j = 0; j < k; ++j) {
+    float best = cur;
+    int be = e;
+#pragma unroll
+    for (int o = G / 2; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+      if (ob > best || (ob == best && oe < be)) { best = ob; be = oe; }
+    }
+    if (be == e) cur = -2.f;                                     // taken
+    if (active && e == j) {
+      topk_idx[t * k + j] = be;
+      topk_score[t * k + j] = best;
+      atomicAdd(&hist[be], 1);
+    }
+  }
+}
+
 template <int EPL>
 __global__ void __launch_bounds__(SW_WARPS * 32)
 k_softmax_topk_warp(const float* __restrict__ logits, int64_t N, int E, int k, float* __restrict__ scores,
@@ -313,9 +353,23 @@ k_router_mma(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restric
     int* hist = reinterpret_cast<int*>(fin + ROWS * 32 + RM_WARPS * 32);   // [32]
     if (threadIdx.x < 32) hist[threadIdx.x] = 0;
     __syncthreads();
-    for (int r = warp; r < ROWS; r += RM_WARPS) {
-      const int64_t t = t0 + r;
-      if (t < N) softmax_topk_token<1>(fin + r * 32, E, k, t, prow, scores, topk_idx, topk_score, hist);
+    if (E <= 8) {
+      for (int r0 = warp * 4; r0 < ROWS; r0 += RM_WARPS * 4) {      // four tokens per warp at a time
+        const int r = r0 + (lane >> 3);
+        const int64_t t = t0 + r;
+        softmax_topk_group<8>(fin + (r < ROWS ? r : 0) * 32, r < ROWS && t < N, E, k, t, scores, topk_idx, topk_score, hist);
+      }
+    } else if (E <= 16) {
+      for (int r0 = warp * 2; r0 < ROWS; r0 += RM_WARPS * 2) {
+        const int r = r0 + (lane >> 4);
+        const int64_t t = t0 + r;
+        softmax_topk_group<16>(fin + (r < ROWS ? r : 0) * 32, r < ROWS && t < N, E, k, t, scores, topk_idx, topk_score, hist);
+      }
+    } else {
+      for (int r = warp; r < ROWS; r += RM_WARPS) {
+        const int64_t t = t0 + r;
+        if (t < N) softmax_topk_token<1>(fin + r * 32, E, k, t, prow, scores, topk_idx, topk_score, hist);
+      }
     }
     __syncthreads();
     if (threadIdx.x < E && hist[threadIdx.x]) atomicAdd(&load[threadIdx.x], hist[threadIdx.x]);
