@@ -42,7 +42,8 @@ typedef enum {
   CAPMOE_EUNSUPPORTED = 2, /* well-formed request with no kernel (dtype, row size not 16-byte) */
   CAPMOE_EWORKSPACE = 3,   /* workspace smaller than capmoe_*_workspace_bytes reports        */
   CAPMOE_ECUDA = 4,        /* a CUDA call failed; see capmoe_last_cuda_error                   */
-  CAPMOE_ETIMEOUT = 5      /* a bounded device-side wait ran out (read from dev_status)       */
+  CAPMOE_ETIMEOUT = 5,     /* a bounded device-side wait ran out (read from dev_status)       */
+  CAPMOE_EINDEX = 6        /* debug check: a row index lies outside its buffer or segment (dev_status) */
 } capmoe_status;
 
 typedef enum { CAPMOE_F32 = 0, CAPMOE_BF16 = 1 } capmoe_dtype;
@@ -318,6 +319,17 @@ int capmoe_ep_combine(const uint64_t* peer_rows, int R, int rank, int E, int64_t
  * (the caller zeroes it first).  The context stays usable. */
 int capmoe_debug_wait_probe(int64_t limit_cycles, int32_t* dev_status, void* stream);
 
+/* Debug check of the indices the later stages will use as addresses (no counterpart in the paper;
+ * the stand-in for a memory checker on machines where none can run).  Reads only: expert_offsets must
+ * be non-decreasing with expert_offsets[E] <= A_max, and every slot_row[t,s] must be -1 or lie inside
+ * the segment of the expert the slot stands for (slots = k, or k + E/D with the home-device slots).
+ * On a violation *dev_status is set to CAPMOE_EINDEX (never a trap); the caller zeroes it first and
+ * reads it after synchronising.  capmoe_layer_forward runs it after the drop stage when the struct's
+ * debug_checks field is non-zero. */
+int capmoe_debug_check_indices(const int32_t* slot_row, const int32_t* topk_idx, const int32_t* expert_offsets,
+                               int64_t N, int E, int k, int slots, int D, const int32_t* token_group,
+                               int64_t A_max, int32_t* dev_status, void* stream);
+
 /* Measurement aid (no counterpart in the paper): one launch that reads `bytes` bytes from p once,
  * as fast as plain loads go, and does nothing else.  Its device time is the floor for any kernel
  * that has to read that much from HBM once, launch included - for the few ten megabytes of a small
@@ -374,6 +386,7 @@ typedef struct {
   float* drop_keys;            /* scratch for the keys, [N,k] (mode 1) or [N,E] (mode 2) 32-bit words; needed
                                   unless metric is Score, token_class is NULL and topk_first is 0 */
   int32_t* bad;                /* device int32, needed when max_experts > 0 (see capmoe_rows_from_mask) */
+  int debug_checks;            /* non-zero: run capmoe_debug_check_indices after the drop (needs dev_status) */
 } capmoe_layer;
 #define CAPMOE_N_STAGE_EVENTS 8
 

@@ -18,7 +18,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libcapmoe.so")
 _lib = None
 
-OK, EINVAL, EUNSUPPORTED, EWORKSPACE, ECUDA, ETIMEOUT = range(6)
+OK, EINVAL, EUNSUPPORTED, EWORKSPACE, ECUDA, ETIMEOUT, EINDEX = range(7)
 F32, BF16 = 0, 1
 MODE_NODROP, MODE_TOKEN_DROP, MODE_EXPANDED_DROP = 0, 1, 2
 MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2, "device_token_drop": 3, "device_expanded_drop": 4}
@@ -30,7 +30,7 @@ EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_device_max_rows", "capm
            "capmoe_rows_from_mask", "capmoe_permute", "capmoe_grouped_ffn",
            "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe",
            "capmoe_grouped_ffn_segments", "capmoe_ep_plan", "capmoe_ep_segments", "capmoe_ep_dispatch",
-           "capmoe_ep_combine", "capmoe_debug_read_probe"]
+           "capmoe_ep_combine", "capmoe_debug_read_probe", "capmoe_debug_check_indices"]
 
 
 class CapmoeError(RuntimeError):
@@ -64,7 +64,7 @@ class _Layer(ctypes.Structure):
         ("stage_events", ctypes.POINTER(ctypes.c_void_p)),
         ("metric", ctypes.c_int), ("metric_seed", ctypes.c_uint64), ("token_class", ctypes.c_void_p),
         ("topk_first", ctypes.c_int), ("max_experts", ctypes.c_int), ("drop_keys", ctypes.c_void_p),
-        ("bad", ctypes.c_void_p),
+        ("bad", ctypes.c_void_p), ("debug_checks", ctypes.c_int),
     ]
 
 N_STAGE_EVENTS = 8
@@ -446,6 +446,17 @@ def combine(y_perm, slot_row, perm_weight, y_shared=None, y=None, stream=None):
     return y
 
 
+def debug_check_indices(slot_row, topk_idx, offsets, E: int, A_max: int, D: int = 1, token_group=None, stream=None):
+    """Runs the index check; returns the device status it produced (OK or EINDEX)."""
+    N, slots = slot_row.shape
+    k = topk_idx.shape[1]
+    st = torch.zeros((1,), device=slot_row.device, dtype=torch.int32)
+    _check(lib().capmoe_debug_check_indices(_ptr(slot_row), _ptr(topk_idx), _ptr(offsets), _i64(N), int(E), int(k),
+                                            int(slots), int(D), _ptr(token_group), _i64(A_max), _ptr(st), _stream(stream)),
+           "capmoe_debug_check_indices")
+    return int(st.item())
+
+
 def debug_read_probe(t: torch.Tensor, stream=None):
     """One plain pass of loads over the tensor's bytes (the one-shot read floor of that size)."""
     _check(lib().capmoe_debug_read_probe(_ptr(t), ctypes.c_size_t(t.numel() * t.element_size()), ctypes.c_void_p(0),
@@ -468,7 +479,7 @@ class MoELayer:
     def __init__(self, x, w_router, bias, w_gate, w_up, w_down, k: int, D: int, mode: str, gamma: float = 1.0,
                  straggler: bool = False, shared=None, round_mode: str = "ceil", C: Optional[int] = None,
                  metric: str = "score", seed: int = 0, token_class=None, topk_first: bool = False,
-                 max_experts: int = 0):
+                 max_experts: int = 0, debug_checks: bool = False):
         """Variants of the drop (token_drop / expanded_drop modes): `metric` ranks candidates by Score, Order,
         Reverse Order or Random; `token_class` (uint8 [N], 1 = protected modality) drops the other modality
         first; `topk_first` lets the expansion only fill spare capacity; `max_experts` > 0 is 'w/ max'."""
@@ -536,6 +547,7 @@ class MoELayer:
             t["bad"] = torch.zeros((1,), **i32)
         L = self.c = _Layer()
         L.metric, L.metric_seed, L.topk_first, L.max_experts = METRICS[metric], seed, int(bool(topk_first)), max_experts
+        L.debug_checks = int(bool(debug_checks))
         L.N, L.d, L.E, L.k, L.F, L.D, L.dtype = N, d, E, k, F, D, _dt(x)
         L.mode, L.C, L.straggler = MODES[mode], C, int(bool(straggler))
         L.F_shared, L.A_max = F_shared, A_max

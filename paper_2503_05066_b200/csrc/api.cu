@@ -180,6 +180,7 @@ extern "C" const char* capmoe_status_str(int status) {
     case CAPMOE_EWORKSPACE: return "workspace too small";
     case CAPMOE_ECUDA: return "CUDA error";
     case CAPMOE_ETIMEOUT: return "device-side wait timed out";
+    case CAPMOE_EINDEX: return "row index outside its buffer (debug check)";
     default: return "unknown status";
   }
 }
@@ -256,6 +257,7 @@ int validate_layer(const capmoe_layer* L) {
                      (L->metric != CAPMOE_METRIC_SCORE || L->token_class || (L->mode == 2 && L->topk_first));
   if (keyed && !L->drop_keys) return CAPMOE_EINVAL;
   if (L->mode != 0 && L->max_experts > 0 && !L->bad) return CAPMOE_EINVAL;
+  if (L->debug_checks && !L->dev_status) return CAPMOE_EINVAL;
   // buffers
   if (!L->logits || !L->scores || !L->topk_idx || !L->topk_score || !L->load || !L->kept || !L->expert_offsets)
     return CAPMOE_EINVAL;
@@ -369,6 +371,10 @@ extern "C" int capmoe_layer_forward(const capmoe_layer* L, void* stream) {
     }
   }
   if (rc != CAPMOE_OK) return rc;
+  if (L->debug_checks && L->N > 0 &&
+      (rc = capmoe_debug_check_indices(L->slot_row, L->topk_idx, L->expert_offsets, L->N, L->E, L->k, slots,
+                                       Dp > 0 ? Dp : 1, nullptr, L->A_max, L->dev_status, stream)) != CAPMOE_OK)
+    return rc;
   if ((rc = mark(2)) != CAPMOE_OK) return rc;
   rc = permute_impl(L->x, L->N, L->d, L->E, L->k, slots, Dp, L->dtype, L->scores, L->topk_idx, nullptr, L->slot_row,
                     L->x_perm, L->perm_token, L->perm_weight, defer_mask ? L->keep_mask : nullptr, stream);

@@ -271,6 +271,33 @@ k_ep_plan(const int32_t* __restrict__ slot_row, const int32_t* __restrict__ topk
   slot_row_ep[i] = out;
 }
 
+// Debug check: every index a later stage uses as an address lies where it should.  Reads only.
+__global__ void __launch_bounds__(256)
+k_check_indices(const int32_t* __restrict__ slot_row, const int32_t* __restrict__ topk_idx,
+                const int32_t* __restrict__ expert_offsets, int64_t N, int E, int k, int slots, int D,
+                const int32_t* __restrict__ token_group, int64_t A_max, int32_t* __restrict__ dev_status) {
+  allow_next_kernel();
+  wait_for_previous_kernel();
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  bool bad = false;
+  if (i <= E) {                                          // offsets: non-decreasing, inside the buffers
+    const int64_t o = expert_offsets[i];
+    bad = o < 0 || o > A_max || (i > 0 && o < expert_offsets[i - 1]);
+  }
+  if (i < N * slots) {
+    const int64_t t = i / slots;
+    const int s = (int)(i - t * slots);
+    const int32_t r = slot_row[i];
+    if (r != -1) {
+      const int m = slots > k ? E / D : 0;
+      const int e = s < k ? topk_idx[t * k + s] : home_group(t, N, D, token_group) * m + (s - k);
+      bad = bad || e < 0 || e >= E || r < expert_offsets[e < 0 || e >= E ? 0 : e] ||
+            r >= expert_offsets[e < 0 || e >= E ? 0 : e + 1];
+    }
+  }
+  if (bad) atomicExch(dev_status, (int)CAPMOE_EINDEX);
+}
+
 __global__ void __launch_bounds__(256)
 k_ep_segments(const int32_t* __restrict__ counts, int S, int C_local, int32_t* __restrict__ seg_begin,
               int32_t* __restrict__ seg_end) {
@@ -328,6 +355,21 @@ extern "C" int capmoe_ep_plan(const int32_t* slot_row, const int32_t* topk_idx, 
   const int rc = note_cuda(launch_chained(k_ep_plan, (unsigned)ceil_div(N * slots, 256), 256, 0, as_stream(stream),
                                           slot_row, topk_idx, expert_offsets, N, E, k, slots, D < 1 ? 1 : D, token_group,
                                           (int)C_local, slot_row_ep, bad));
+  count_launch(1);
+  return rc;
+}
+
+extern "C" int capmoe_debug_check_indices(const int32_t* slot_row, const int32_t* topk_idx, const int32_t* expert_offsets,
+                                          int64_t N, int E, int k, int slots, int D, const int32_t* token_group,
+                                          int64_t A_max, int32_t* dev_status, void* stream) {
+  if (N < 0 || E < 1 || k < 1 || k > E || slots < k || A_max < 0) return CAPMOE_EINVAL;
+  if (slots > k && (D < 1 || E % D != 0 || slots != k + E / D)) return CAPMOE_EINVAL;
+  if (!expert_offsets || !dev_status || (N > 0 && (!slot_row || !topk_idx))) return CAPMOE_EINVAL;
+  const int64_t items = N * slots > E + 1 ? N * slots : E + 1;
+  if (items >= ((int64_t)1 << 38)) return CAPMOE_EUNSUPPORTED;
+  const int rc = note_cuda(launch_chained(k_check_indices, (unsigned)ceil_div(items, 256), 256, 0, as_stream(stream),
+                                          slot_row, topk_idx, expert_offsets, N, E, k, slots, D < 1 ? 1 : D, token_group,
+                                          A_max, dev_status));
   count_launch(1);
   return rc;
 }

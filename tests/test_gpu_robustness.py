@@ -227,3 +227,48 @@ def test_two_layers_on_two_streams_do_not_disturb_each_other(cm, name, mode, ove
     torch.cuda.synchronize()
     a.check_device_status()
     b.check_device_status()
+
+
+def test_debug_index_check_passes_on_real_drops_and_flags_bad_indices(cm):
+    """The index check (the stand-in for a memory checker) accepts what the drop stages produce and
+    flags, through the status word and without touching anything, a row outside its expert's segment,
+    a row count beyond the buffers, and offsets that go backwards."""
+    import numpy as np
+    from paper_2503_05066_b200 import synth
+    N, E, k, D = 3000, 16, 4, 4
+    lg = synth.synthetic_logits(N, E, 8, bias=(-np.log(np.arange(E) + 1.0)).astype(np.float32))
+    r = cm.route(None, None, None, k, logits_in=torch.from_numpy(lg).cuda())
+    C = cm.capacity(N, E, k, 1.0)
+    td = cm.token_drop(r["topk_score"], r["topk_idx"], E, C)
+    ed = cm.expanded_drop(r["scores"], r["topk_idx"], C, D)
+    A_td, A_ed = int(td["offsets"][-1]), int(ed["offsets"][-1])
+    assert cm.debug_check_indices(td["slot_row"], r["topk_idx"], td["offsets"], E, A_td) == cm.OK
+    assert cm.debug_check_indices(ed["slot_row"], r["topk_idx"], ed["offsets"], E, A_ed, D=D) == cm.OK
+    # buffers one row too short
+    assert cm.debug_check_indices(td["slot_row"], r["topk_idx"], td["offsets"], E, A_td - 1) == cm.EINDEX
+    # one kept pair pointed at another expert's segment
+    bad = td["slot_row"].clone()
+    t, s = [int(v[0]) for v in torch.nonzero(bad >= 0, as_tuple=True)]
+    e = int(r["topk_idx"][t, s])
+    bad[t, s] = int(td["offsets"][(e + 1) % E + 1]) - 1 if int(td["kept"][(e + 1) % E]) > 0 else A_td + 5
+    assert cm.debug_check_indices(bad, r["topk_idx"], td["offsets"], E, A_td) == cm.EINDEX
+    # offsets that go backwards
+    off = td["offsets"].clone()
+    off[3] = off[4] + 1
+    assert cm.debug_check_indices(td["slot_row"], r["topk_idx"], off, E, A_td) == cm.EINDEX
+
+
+def test_layer_forward_with_debug_checks(cm):
+    from paper_2503_05066_b200 import synth
+    cfg = synth.CONFIGS["olmoe"].with_(N=1500, d=256, F=256, E=16, k=4, D=4)
+    inp = synth.make_layer_inputs(cfg)
+    for mode in ("nodrop", "token_drop", "expanded_drop", "device_expanded_drop"):
+        lay = cm.MoELayer(inp.x.cuda(), inp.w_router.cuda(), inp.bias.cuda(), inp.w_gate.cuda(), inp.w_up.cuda(),
+                          inp.w_down.cuda(), cfg.k, cfg.D, mode, gamma=1.0, debug_checks=True)
+        plain = cm.MoELayer(inp.x.cuda(), inp.w_router.cuda(), inp.bias.cuda(), inp.w_gate.cuda(), inp.w_up.cuda(),
+                            inp.w_down.cuda(), cfg.k, cfg.D, mode, gamma=1.0)
+        y = lay.forward()
+        y0 = plain.forward()
+        torch.cuda.synchronize()
+        lay.check_device_status()                       # raises on CAPMOE_EINDEX / CAPMOE_ETIMEOUT
+        assert torch.equal(y, y0)
