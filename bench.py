@@ -271,6 +271,66 @@ def run_table(args):
         del g, inp
 
 
+def run_ep(args):
+    """--ep R: the layer under expert parallelism with per-rank capacity, R ranks with N/R tokens and
+    E/R experts each, every rank's stages timed ALONE on this one GPU (as if it had a B200 to itself).
+    What a rank's owner FFN takes depends on the rows the other ranks send it, so the slowest owner is
+    the straggler of the paper's latency model (Eq. 4); the layer time under expert parallelism is
+    estimated as the sum over the stages of the slowest rank's time.  The exchange itself is not timed
+    (one GPU): this is a measurement of the per-rank work, not a multi-GPU number.  One JSON line per mode."""
+    import torch
+    from paper_2503_05066_b200 import capmoe, ep, synth
+    cfg = _pick_config(args)
+    R = args.ep
+    assert cfg.E % R == 0 and cfg.N % R == 0
+    n_local, m = cfg.N // R, cfg.E // R
+    inp = synth.make_layer_inputs(cfg)
+    wr, b = inp.w_router.cuda(), inp.bias.cuda()
+    wg, wu, wd = inp.w_gate.cuda(), inp.w_up.cuda(), inp.w_down.cuda()
+    xs = [inp.x[r * n_local:(r + 1) * n_local].cuda().contiguous() for r in range(R)]
+    steps = max(3, min(args.steps, 20))
+
+    def med(fn):
+        ts = []
+        for i in range(steps + 2):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    base = None
+    for mode, gam in [("nodrop", None)] + [(mo, g_) for g_ in cfg.gammas for mo in ("token_drop", "expanded_drop")]:
+        ranks = [ep.EPRank(r, R, xs[r], wr, b, wg[r * m:(r + 1) * m], wu[r * m:(r + 1) * m], wd[r * m:(r + 1) * m],
+                           cfg.k, mode, 1.0 if gam is None else gam) for r in range(R)]
+        group = ep.EPGroupOnOneDevice(ranks, "peer")
+        group.forward()
+        torch.cuda.synchronize()
+        for rk in ranks:
+            rk.check()
+        t_route = [med(rk.route_and_drop) for rk in ranks]
+        t_disp = [med(lambda rk=rk: rk.dispatch_to_peers(group.peer_x)) for rk in ranks]
+        t_ffn = [med(rk.expert_ffn) for rk in ranks]
+        t_comb = [med(lambda rk=rk: rk.combine_from_peers(group.peer_y)) for rk in ranks]
+        rows = [int(rk.cnt_recv.sum().item()) for rk in ranks]
+        layer_ms = max(t_route) + max(t_disp) + max(t_ffn) + max(t_comb)
+        if mode == "nodrop":
+            base = layer_ms
+        print(json.dumps({
+            "workload": f"{cfg.name}: N={cfg.N} d={cfg.d} E={cfg.E} k={cfg.k} F={cfg.F} {cfg.dtype}, {R} ranks x {n_local} tokens, "
+                        f"{m} expert(s) per rank", "mode": mode, "gamma": gam, "C_local": ranks[0].C_local,
+            "rows_received_per_owner": rows, "max_over_mean_rows": max(rows) / (sum(rows) / R) if sum(rows) else None,
+            "owner_ffn_ms": t_ffn, "route_drop_ms_max": max(t_route), "dispatch_ms_max": max(t_disp),
+            "combine_ms_max": max(t_comb), "ep_layer_ms_slowest_rank_per_stage": layer_ms,
+            "tokens_per_s_all_ranks": cfg.N / (layer_ms * 1e-3), "speedup_vs_nodrop": base / layer_ms,
+            "note": "each rank timed alone on one GPU; exchange not timed; not a multi-GPU measurement"}), flush=True)
+        del group, ranks
+        torch.cuda.empty_cache()
+
+
 def _pick_config(args):
     from paper_2503_05066_b200 import synth
     cfg = synth.CONFIGS[args.config]
@@ -385,6 +445,9 @@ def main():
                          "chosen config (for the Qwen-shape sweep: N in 128..65536, gamma in 0.5..2.0)")
     ap.add_argument("--markdown", action="store_true", help="with --table: print a markdown table instead of JSON lines")
     ap.add_argument("--no-cpu", dest="cpu", action="store_false", help="skip the CPU baseline")
+    ap.add_argument("--ep", type=int, default=0,
+                    help="R > 0: instead of the benchmark line, time the ranks of an R-way expert-parallel group with "
+                         "per-rank capacity one after another on this GPU (one JSON line per mode)")
     ap.add_argument("--impl", default="capmoe", choices=["capmoe", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=None,
                     help="tokens in the CPU checker's FFN sample (default 1024 for cpu_baseline, 64 per step "
@@ -405,6 +468,9 @@ def main():
         return
     if args.table:
         run_table(args)
+        return
+    if args.ep > 0:
+        run_ep(args)
         return
 
     import torch
