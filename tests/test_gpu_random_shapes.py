@@ -111,7 +111,13 @@ def _ffn_cases(n, seed):
     return out
 
 
-@pytest.mark.parametrize("E,d,F,rows,D_straggler", _ffn_cases(16, 99))
+# CTA-pair kernel with an expert width that is an odd multiple of 64 (the last 128-column block of
+# the gate/up GEMM is half filled), with and without straggler emulation
+_FFN_ODD_WIDTH = [(4, 128, 192, (1100, 1200, 1300, 1025), 0), (3, 64, 320, (256, 512, 768), 3),
+                  (2, 192, 64, (1500, 30), 0), (2, 128, 448, (1024, 1024), 2)]
+
+
+@pytest.mark.parametrize("E,d,F,rows,D_straggler", _ffn_cases(16, 99) + _FFN_ODD_WIDTH)
 def test_grouped_ffn_on_random_segments(cm, E, d, F, rows, D_straggler):
     """bf16 tensor-core FFN over random expert segments against the double-precision SwiGLU of the
     CPU checker on sampled rows; rows past the last segment stay untouched."""
