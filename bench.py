@@ -311,19 +311,18 @@ def run_ep(args):
         torch.cuda.synchronize()
         for rk in ranks:
             rk.check()
-        t_route = [med(rk.route_and_drop) for rk in ranks]
-        t_disp = [med(lambda rk=rk: rk.dispatch_to_peers(group.peer_x)) for rk in ranks]
+        t_disp = [med(rk.dispatch) for rk in ranks]
         t_ffn = [med(rk.expert_ffn) for rk in ranks]
-        t_comb = [med(lambda rk=rk: rk.combine_from_peers(group.peer_y)) for rk in ranks]
+        t_comb = [med(rk.combine) for rk in ranks]
         rows = [int(rk.cnt_recv.sum().item()) for rk in ranks]
-        layer_ms = max(t_route) + max(t_disp) + max(t_ffn) + max(t_comb)
+        layer_ms = max(t_disp) + max(t_ffn) + max(t_comb)
         if mode == "nodrop":
             base = layer_ms
         print(json.dumps({
             "workload": f"{cfg.name}: N={cfg.N} d={cfg.d} E={cfg.E} k={cfg.k} F={cfg.F} {cfg.dtype}, {R} ranks x {n_local} tokens, "
                         f"{m} expert(s) per rank", "mode": mode, "gamma": gam, "C_local": ranks[0].C_local,
             "rows_received_per_owner": rows, "max_over_mean_rows": max(rows) / (sum(rows) / R) if sum(rows) else None,
-            "owner_ffn_ms": t_ffn, "route_drop_ms_max": max(t_route), "dispatch_ms_max": max(t_disp),
+            "owner_ffn_ms": t_ffn, "route_drop_dispatch_ms_max": max(t_disp),
             "combine_ms_max": max(t_comb), "ep_layer_ms_slowest_rank_per_stage": layer_ms,
             "tokens_per_s_all_ranks": cfg.N / (layer_ms * 1e-3), "speedup_vs_nodrop": base / layer_ms,
             "note": "each rank timed alone on one GPU; exchange not timed; not a multi-GPU measurement"}), flush=True)

@@ -312,6 +312,46 @@ int capmoe_ep_combine(const uint64_t* peer_rows, int R, int rank, int E, int64_t
                       const int32_t* slot_row_ep, const float* perm_weight, int64_t N, int d, int slots,
                       int dtype, const void* y_shared, void* y, void* stream);
 
+/* One rank's forward under expert parallelism, in the three phases between which the caller orders
+ * the ranks.  Every pointer is a device pointer; sizes in brackets.
+ *   capmoe_ep_forward_dispatch  stages 1-3 on the rank's own N tokens with C_local (mode 1 = Token Drop,
+ *                               2 = Expanded Drop with D = R and every token at home on `rank`, 0 = no
+ *                               drop, C_local = N), capmoe_ep_plan with row stride C (>= C_local, the same
+ *                               on all ranks), then the rows go out: into the owners' x_recv buffers
+ *                               through peer_x (a table of R addresses), or, with peer_x == NULL, into
+ *                               this rank's send buffer x_send for an all-to-all.  kept [E] = [R][m] are
+ *                               the counts the owners need (cnt_recv block `rank` of owner r').
+ *   capmoe_ep_forward_experts   the owner's part, once rows (x_recv) and counts (cnt_recv [R*m]) of all
+ *                               ranks have arrived: segments, SwiGLU FFN with the rank's own m experts,
+ *                               results in y_recv.
+ *   capmoe_ep_forward_combine   once all owners are done: Eq. 2 for the rank's tokens, reading the
+ *                               results through peer_y, or, with peer_y == NULL, from y_ret (the
+ *                               all-to-all's output).  Writes y [N,d].
+ * All fields are checked before anything is enqueued.  dev_status [CAPMOE_FFN_STATUS_WORDS] and
+ * bad [1] report as in capmoe_grouped_ffn / capmoe_ep_plan. */
+typedef struct {
+  int64_t N; int d, E, k, F, dtype;
+  int R, rank, mode;           /* mode: 0 no drop, 1 Token Drop, 2 Expanded Drop */
+  int64_t C_local, C;          /* the rank's capacity; the row stride all ranks agreed on */
+  const void* x; const void* w_router; const float* bias;
+  const void* w_gate; const void* w_up; const void* w_down;            /* this rank's m = E/R experts */
+  float* logits; float* scores; int32_t* topk_idx; float* topk_score; int32_t* load;   /* [N,E] .. [E] */
+  uint64_t* keep_mask; int32_t* cand; int32_t* kept; int32_t* expert_offsets; int32_t* slot_row;
+  int32_t* slot_row_ep;        /* [N, slots] rows of the [E][C] space */
+  const int32_t* token_group;  /* [N] filled with `rank` (mode 2), else NULL */
+  int32_t* perm_token; float* perm_weight;                              /* [E*C] */
+  void* x_send; void* y_ret;                                            /* [E*C, d]: collective transport */
+  const uint64_t* peer_x; const uint64_t* peer_y;                       /* [R] addresses: peer transport */
+  void* x_recv; void* h_ws; void* y_recv;                               /* [R*m*C, d], [.., F], [.., d] */
+  int32_t* cnt_recv; int32_t* seg_begin; int32_t* seg_end;              /* [R*m] */
+  void* y;                                                              /* [N, d] */
+  void* drop_ws; size_t drop_ws_bytes;
+  int32_t* dev_status; int32_t* bad;
+} capmoe_ep_rank;
+int capmoe_ep_forward_dispatch(const capmoe_ep_rank* P, void* stream);
+int capmoe_ep_forward_experts(const capmoe_ep_rank* P, void* stream);
+int capmoe_ep_forward_combine(const capmoe_ep_rank* P, void* stream);
+
 /* Self-test of the bounded device-side wait used inside the tensor-core kernels (no counterpart
  * in the paper).  Launches one warp that waits on a barrier nothing will ever signal, with the
  * same wait routine and a limit of limit_cycles SM clock cycles (1 .. 4e9); the wait must run

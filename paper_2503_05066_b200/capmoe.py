@@ -29,7 +29,7 @@ EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_device_max_rows", "capm
            "capmoe_device_drop", "capmoe_drop_keys", "capmoe_priority_keys", "capmoe_limit_experts",
            "capmoe_rows_from_mask", "capmoe_permute", "capmoe_grouped_ffn",
            "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe",
-           "capmoe_grouped_ffn_segments", "capmoe_ep_plan", "capmoe_ep_segments", "capmoe_ep_dispatch",
+           "capmoe_grouped_ffn_segments", "capmoe_ep_plan", "capmoe_ep_forward_dispatch", "capmoe_ep_forward_experts", "capmoe_ep_forward_combine", "capmoe_ep_segments", "capmoe_ep_dispatch",
            "capmoe_ep_combine", "capmoe_debug_read_probe", "capmoe_debug_check_indices"]
 
 
@@ -65,6 +65,29 @@ class _Layer(ctypes.Structure):
         ("metric", ctypes.c_int), ("metric_seed", ctypes.c_uint64), ("token_class", ctypes.c_void_p),
         ("topk_first", ctypes.c_int), ("max_experts", ctypes.c_int), ("drop_keys", ctypes.c_void_p),
         ("bad", ctypes.c_void_p), ("debug_checks", ctypes.c_int),
+    ]
+
+class _EPRank(ctypes.Structure):
+    _fields_ = [
+        ("N", ctypes.c_int64), ("d", ctypes.c_int), ("E", ctypes.c_int), ("k", ctypes.c_int),
+        ("F", ctypes.c_int), ("dtype", ctypes.c_int),
+        ("R", ctypes.c_int), ("rank", ctypes.c_int), ("mode", ctypes.c_int),
+        ("C_local", ctypes.c_int64), ("C", ctypes.c_int64),
+        ("x", ctypes.c_void_p), ("w_router", ctypes.c_void_p), ("bias", ctypes.c_void_p),
+        ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p), ("w_down", ctypes.c_void_p),
+        ("logits", ctypes.c_void_p), ("scores", ctypes.c_void_p), ("topk_idx", ctypes.c_void_p),
+        ("topk_score", ctypes.c_void_p), ("load", ctypes.c_void_p),
+        ("keep_mask", ctypes.c_void_p), ("cand", ctypes.c_void_p), ("kept", ctypes.c_void_p),
+        ("expert_offsets", ctypes.c_void_p), ("slot_row", ctypes.c_void_p),
+        ("slot_row_ep", ctypes.c_void_p), ("token_group", ctypes.c_void_p),
+        ("perm_token", ctypes.c_void_p), ("perm_weight", ctypes.c_void_p),
+        ("x_send", ctypes.c_void_p), ("y_ret", ctypes.c_void_p),
+        ("peer_x", ctypes.c_void_p), ("peer_y", ctypes.c_void_p),
+        ("x_recv", ctypes.c_void_p), ("h_ws", ctypes.c_void_p), ("y_recv", ctypes.c_void_p),
+        ("cnt_recv", ctypes.c_void_p), ("seg_begin", ctypes.c_void_p), ("seg_end", ctypes.c_void_p),
+        ("y", ctypes.c_void_p),
+        ("drop_ws", ctypes.c_void_p), ("drop_ws_bytes", ctypes.c_size_t),
+        ("dev_status", ctypes.c_void_p), ("bad", ctypes.c_void_p),
     ]
 
 N_STAGE_EVENTS = 8
@@ -433,6 +456,34 @@ def ep_combine(peer_rows, R: int, rank: int, E: int, C_local: int, slot_row_ep, 
                                    _ptr(perm_weight), _i64(N), int(d), int(slots), _dt(dtype), _ptr(y_shared), _ptr(y),
                                    _stream(stream)), "capmoe_ep_combine")
     return y
+
+
+EP_MODES = {"nodrop": 0, "token_drop": 1, "expanded_drop": 2}
+
+
+def ep_rank_struct(**fields) -> _EPRank:
+    """capmoe_ep_rank from tensors (device pointers taken), ints and None."""
+    P = _EPRank()
+    for name, v in fields.items():
+        if isinstance(v, torch.Tensor):
+            assert v.is_contiguous()
+            v = v.data_ptr()
+        elif v is None:
+            v = 0
+        setattr(P, name, v)
+    return P
+
+
+def ep_forward_dispatch(P: _EPRank, stream=None):
+    _check(lib().capmoe_ep_forward_dispatch(ctypes.byref(P), _stream(stream)), "ep_forward_dispatch")
+
+
+def ep_forward_experts(P: _EPRank, stream=None):
+    _check(lib().capmoe_ep_forward_experts(ctypes.byref(P), _stream(stream)), "ep_forward_experts")
+
+
+def ep_forward_combine(P: _EPRank, stream=None):
+    _check(lib().capmoe_ep_forward_combine(ctypes.byref(P), _stream(stream)), "ep_forward_combine")
 
 
 def combine(y_perm, slot_row, perm_weight, y_shared=None, y=None, stream=None):

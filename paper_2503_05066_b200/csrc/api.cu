@@ -413,3 +413,83 @@ extern "C" int capmoe_layer_forward_host(const capmoe_layer* L, const void* x_ho
   err = cudaMemcpyAsync(y_host, L->y, bytes, cudaMemcpyDeviceToHost, st);
   return note_cuda(err);
 }
+
+// ---------------------------------------------------------------------------------------------
+// One rank of an expert-parallel group (see capmoe_ep_rank in the header).
+namespace {
+int validate_ep_rank(const capmoe_ep_rank* P) {
+  if (!P) return CAPMOE_EINVAL;
+  if (P->N < 0 || P->d < 1 || P->E < 1 || P->k < 1 || P->k > P->E || P->F < 1) return CAPMOE_EINVAL;
+  if (P->dtype != CAPMOE_F32 && P->dtype != CAPMOE_BF16) return CAPMOE_EUNSUPPORTED;
+  if (P->E > 256 || P->k > 32) return CAPMOE_EUNSUPPORTED;
+  if (P->R < 1 || P->rank < 0 || P->rank >= P->R || P->E % P->R != 0) return CAPMOE_EINVAL;
+  if (P->mode < 0 || P->mode > 2) return CAPMOE_EINVAL;
+  if (P->C_local < 0 || P->C_local > P->N || P->C < P->C_local) return CAPMOE_EINVAL;
+  if (P->mode == 0 && P->C_local != P->N) return CAPMOE_EINVAL;
+  if ((int64_t)P->E * P->C >= ((int64_t)1 << 31)) return CAPMOE_EUNSUPPORTED;
+  if (((size_t)P->d * elt_size(P->dtype)) % 16 != 0) return CAPMOE_EUNSUPPORTED;
+  if (!P->logits || !P->scores || !P->topk_idx || !P->topk_score || !P->load || !P->kept || !P->expert_offsets ||
+      !P->bad || !P->cnt_recv || !P->seg_begin || !P->seg_end)
+    return CAPMOE_EINVAL;
+  if (P->mode == 2 && (!P->cand || (P->N > 0 && !P->token_group))) return CAPMOE_EINVAL;
+  if (P->N > 0 && (!P->x || !P->w_router || !P->keep_mask || !P->slot_row || !P->slot_row_ep || !P->y || !P->drop_ws))
+    return CAPMOE_EINVAL;
+  if (P->N > 0 && P->drop_ws_bytes < drop_ws_required(P->mode, P->N, P->E, P->k, P->mode == 2 ? P->R : 1))
+    return CAPMOE_EWORKSPACE;
+  if ((int64_t)P->E * P->C > 0) {
+    if (!P->perm_token || !P->perm_weight || !P->x_recv || !P->h_ws || !P->y_recv || !P->w_gate || !P->w_up || !P->w_down)
+      return CAPMOE_EINVAL;
+    if (!P->peer_x && !P->x_send) return CAPMOE_EINVAL;
+    if (!P->peer_y && !P->y_ret) return CAPMOE_EINVAL;
+  }
+  return CAPMOE_OK;
+}
+}  // namespace
+
+extern "C" int capmoe_ep_forward_dispatch(const capmoe_ep_rank* P, void* stream) {
+  int rc = validate_ep_rank(P);
+  if (rc != CAPMOE_OK) return rc;
+  cudaStream_t st = as_stream(stream);
+  if ((rc = clear_words(P->load, P->E, P->bad, 1, st)) != CAPMOE_OK) return rc;
+  rc = route_impl(P->x, P->w_router, P->bias, nullptr, P->N, P->d, P->E, P->k, P->dtype, P->logits, P->scores, P->topk_idx,
+                  P->topk_score, P->load, stream, true);
+  if (rc != CAPMOE_OK) return rc;
+  const bool expanded = P->mode == 2;
+  const int slots = expanded ? P->k + P->E / P->R : P->k;
+  if (expanded)
+    rc = expanded_drop_impl(P->scores, P->topk_idx, P->N, P->E, P->k, P->C_local, P->R, P->token_group, P->keep_mask, P->cand,
+                            P->kept, P->expert_offsets, P->slot_row, P->drop_ws, P->drop_ws_bytes, stream, false, nullptr,
+                            P->load);
+  else
+    rc = token_drop_impl(P->topk_score, P->topk_idx, P->N, P->E, P->k, P->C_local, P->keep_mask, P->kept, P->expert_offsets,
+                         P->slot_row, P->drop_ws, P->drop_ws_bytes, stream, false, nullptr, P->load);
+  if (rc != CAPMOE_OK) return rc;
+  rc = capmoe_ep_plan(P->slot_row, P->topk_idx, P->expert_offsets, P->N, P->E, P->k, slots, expanded ? P->R : 1,
+                      P->token_group, P->C, P->slot_row_ep, P->bad, stream);
+  if (rc != CAPMOE_OK || P->N == 0 || (int64_t)P->E * P->C == 0) return rc;
+  if (P->peer_x)
+    return capmoe_ep_dispatch(P->x, P->N, P->d, P->E, P->k, slots, expanded ? P->R : 0, P->dtype, P->scores, P->topk_idx,
+                              P->token_group, P->slot_row_ep, P->peer_x, P->R, P->rank, P->C, P->perm_token, P->perm_weight,
+                              stream);
+  return capmoe_permute(P->x, P->N, P->d, P->E, P->k, slots, expanded ? P->R : 0, P->dtype, P->scores, P->topk_idx,
+                        P->token_group, P->slot_row_ep, P->x_send, P->perm_token, P->perm_weight, stream);
+}
+
+extern "C" int capmoe_ep_forward_experts(const capmoe_ep_rank* P, void* stream) {
+  int rc = validate_ep_rank(P);
+  if (rc != CAPMOE_OK) return rc;
+  rc = capmoe_ep_segments(P->cnt_recv, P->E, P->C, P->seg_begin, P->seg_end, stream);
+  if (rc != CAPMOE_OK || (int64_t)P->E * P->C == 0) return rc;
+  return capmoe_grouped_ffn_segments(P->x_recv, P->seg_begin, P->seg_end, P->E, P->E / P->R, P->d, P->F, P->dtype, P->w_gate,
+                                     P->w_up, P->w_down, P->h_ws, P->y_recv, (int64_t)P->E * P->C, P->dev_status, stream);
+}
+
+extern "C" int capmoe_ep_forward_combine(const capmoe_ep_rank* P, void* stream) {
+  int rc = validate_ep_rank(P);
+  if (rc != CAPMOE_OK) return rc;
+  const int slots = P->mode == 2 ? P->k + P->E / P->R : P->k;
+  if (P->peer_y && (int64_t)P->E * P->C > 0)
+    return capmoe_ep_combine(P->peer_y, P->R, P->rank, P->E, P->C, P->slot_row_ep, P->perm_weight, P->N, P->d, slots,
+                             P->dtype, nullptr, P->y, stream);
+  return capmoe_combine(P->y_ret, P->slot_row_ep, P->perm_weight, P->N, P->d, slots, P->dtype, nullptr, P->y, stream);
+}

@@ -29,11 +29,11 @@ import torch.distributed as dist
 from . import capmoe
 
 
-def exchange_rows(send: torch.Tensor, R: int, group=None) -> torch.Tensor:
+def exchange_rows(send: torch.Tensor, R: int, group=None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """send [R * B, ...]: block r' goes to rank r'.  Returns recv of the same shape: block r came
     from rank r.  Equal splits: the per-rank capacity bounds every block, so no sizes are exchanged."""
     assert send.shape[0] % R == 0
-    recv = torch.empty_like(send)
+    recv = torch.empty_like(send) if out is None else out
     if R == 1:
         recv.copy_(send)
     else:
@@ -47,11 +47,12 @@ def owner_layout(rank: int, R: int, m: int, C: int):
 
 
 class EPRank:
-    """One rank of the group: its tokens, the router, its m experts, and every buffer of a forward."""
+    """One rank of the group: its tokens, the router, its m experts, and every buffer of a forward.
+    The three phases of the forward are the library's capmoe_ep_forward_* calls on one struct."""
 
     def __init__(self, rank: int, R: int, x, w_router, bias, w_gate_local, w_up_local, w_down_local, k: int,
                  mode: str, gamma: float = 1.0, C_buf: Optional[int] = None, round_mode: str = "ceil"):
-        assert mode in ("nodrop", "token_drop", "expanded_drop")
+        assert mode in capmoe.EP_MODES
         self.rank, self.R, self.k, self.mode = rank, R, k, mode
         self.x, self.w_router, self.bias = x, w_router, bias
         self.w_gate, self.w_up, self.w_down = w_gate_local, w_up_local, w_down_local
@@ -59,6 +60,7 @@ class EPRank:
         E = w_router.shape[0]
         assert E % R == 0 and w_gate_local.shape[0] == E // R
         self.N, self.d, self.E, self.m = N, d, E, E // R
+        self.F = w_gate_local.shape[-2]
         self.C_local = N if mode == "nodrop" else capmoe.capacity(N, E, k, gamma, round_mode)
         # the row stride every rank of the group uses (>= every rank's own capacity)
         self.C = self.C_local if C_buf is None else int(C_buf)
@@ -66,66 +68,67 @@ class EPRank:
         self.expanded = mode == "expanded_drop"
         self.slots = k + self.m if self.expanded else k
         dev, dt = x.device, x.dtype
+        i32 = dict(device=dev, dtype=torch.int32)
+        f32 = dict(device=dev, dtype=torch.float32)
         rows = max(E * self.C, 1)
-        self.token_group = torch.full((N,), rank, device=dev, dtype=torch.int32) if self.expanded else None
-        self.drop_ws = torch.empty((capmoe.drop_workspace_bytes(N, E, k, R, self.expanded),), device=dev,
+        self.token_group = torch.full((N,), rank, **i32) if self.expanded else None
+        self.drop_ws = torch.empty((max(capmoe.drop_workspace_bytes(N, E, k, R, self.expanded), 1),), device=dev,
                                    dtype=torch.uint8)
+        self.r = dict(logits=torch.empty((N, E), **f32), scores=torch.empty((N, E), **f32),
+                      topk_idx=torch.empty((N, k), **i32), topk_score=torch.empty((N, k), **f32),
+                      load=torch.zeros((E,), **i32))
+        self.dr = dict(keep_mask=torch.zeros((N, (E + 63) // 64), device=dev, dtype=torch.int64),
+                       cand=torch.zeros((E,), **i32), kept=torch.zeros((E,), **i32),
+                       offsets=torch.zeros((E + 1,), **i32), slot_row=torch.full((N, self.slots), -1, **i32))
+        self.slot_row_ep = torch.full((N, self.slots), -1, **i32)
+        self.bad = torch.zeros((1,), **i32)
         self.x_send = torch.zeros((rows, d), device=dev, dtype=dt)         # [E][C] rows of this rank
         self.x_recv = torch.zeros((rows, d), device=dev, dtype=dt)         # [R][m][C] rows this rank owns
-        self.h_ws = torch.empty((rows, w_gate_local.shape[-2]), device=dev, dtype=dt)
+        self.h_ws = torch.empty((rows, self.F), device=dev, dtype=dt)
         self.y_recv = torch.zeros((rows, d), device=dev, dtype=dt)
         self.y_ret = torch.zeros((rows, d), device=dev, dtype=dt)
-        self.perm = dict(perm_token=torch.full((rows,), -1, device=dev, dtype=torch.int32),
-                         perm_weight=torch.zeros((rows,), device=dev, dtype=torch.float32))
-        self.cnt_recv = torch.zeros((E,), device=dev, dtype=torch.int32)   # [R][m] kept of (source, local expert)
-        self.dev_status = torch.zeros((capmoe.FFN_STATUS_WORDS,), device=dev, dtype=torch.int32)
+        self.perm = dict(perm_token=torch.full((rows,), -1, **i32), perm_weight=torch.zeros((rows,), **f32))
+        self.cnt_recv = torch.zeros((E,), **i32)                           # [R][m] kept of (source, local expert)
+        self.seg_begin = torch.zeros((E,), **i32)
+        self.seg_end = torch.zeros((E,), **i32)
+        self.dev_status = torch.zeros((capmoe.FFN_STATUS_WORDS,), **i32)
         self.y = torch.empty((N, d), device=dev, dtype=dt)
+        self._peer_x = self._peer_y = None
 
-    # ---- stage 1-3 on the rank's own tokens, then the fixed row places
-    def route_and_drop(self):
-        self.r = capmoe.route(self.x, self.w_router, self.bias, self.k)
-        if self.expanded:
-            self.dr = capmoe.expanded_drop(self.r["scores"], self.r["topk_idx"], self.C_local, self.R,
-                                           token_group=self.token_group, ws=self.drop_ws)
-        else:
-            self.dr = capmoe.token_drop(self.r["topk_score"], self.r["topk_idx"], self.E, self.C_local, ws=self.drop_ws)
-        self.slot_row_ep, self.bad = capmoe.ep_plan(self.dr["slot_row"], self.r["topk_idx"], self.dr["offsets"], self.E,
-                                                    self.C, D=self.R if self.expanded else 1,
-                                                    token_group=self.token_group)
-        return self.dr["kept"]                         # [E] = [R][m]: rows for (owner, its local expert)
+    def set_peers(self, peer_x: Optional[torch.Tensor], peer_y: Optional[torch.Tensor]):
+        """Device tables [R] (int64) of the ranks' x_recv / y_recv addresses: peer transport."""
+        self._peer_x, self._peer_y = peer_x, peer_y
 
-    @property
-    def _Dp(self):
-        return self.R if self.expanded else 0
+    def _struct(self):
+        return capmoe.ep_rank_struct(
+            N=self.N, d=self.d, E=self.E, k=self.k, F=self.F, dtype=capmoe._dt(self.x), R=self.R, rank=self.rank,
+            mode=capmoe.EP_MODES[self.mode], C_local=self.C_local, C=self.C,
+            x=self.x, w_router=self.w_router, bias=self.bias, w_gate=self.w_gate, w_up=self.w_up, w_down=self.w_down,
+            logits=self.r["logits"], scores=self.r["scores"], topk_idx=self.r["topk_idx"],
+            topk_score=self.r["topk_score"], load=self.r["load"], keep_mask=self.dr["keep_mask"], cand=self.dr["cand"],
+            kept=self.dr["kept"], expert_offsets=self.dr["offsets"], slot_row=self.dr["slot_row"],
+            slot_row_ep=self.slot_row_ep, token_group=self.token_group, perm_token=self.perm["perm_token"],
+            perm_weight=self.perm["perm_weight"], x_send=self.x_send, y_ret=self.y_ret, peer_x=self._peer_x,
+            peer_y=self._peer_y, x_recv=self.x_recv, h_ws=self.h_ws, y_recv=self.y_recv, cnt_recv=self.cnt_recv,
+            seg_begin=self.seg_begin, seg_end=self.seg_end, y=self.y, drop_ws=self.drop_ws,
+            drop_ws_bytes=self.drop_ws.numel(), dev_status=self.dev_status, bad=self.bad)
 
-    # ---- stage 4, collective transport: fill the send buffer
-    def fill_send_buffer(self):
-        capmoe.permute(self.x, self.r["scores"], self.r["topk_idx"], self.slot_row_ep, self.x_send.shape[0], self._Dp,
-                       token_group=self.token_group,
-                       out=dict(x_perm=self.x_send, perm_token=self.perm["perm_token"],
-                                perm_weight=self.perm["perm_weight"]))
-        return self.x_send
+    def dispatch(self):
+        """Stages 1-4 on the rank's own tokens: router, drop with C_local, fixed row places, and the
+        rows on their way (into the owners' buffers, or into x_send).  Returns kept [E] = [R][m]:
+        rows for (owner, its local expert)."""
+        capmoe.ep_forward_dispatch(self._struct())
+        return self.dr["kept"]
 
-    # ---- stage 4, peer transport: store rows straight into the owners' buffers
-    def dispatch_to_peers(self, peer_x_recv: torch.Tensor):
-        capmoe.ep_dispatch(self.x, self.r["scores"], self.r["topk_idx"], self.slot_row_ep, peer_x_recv, self.R,
-                           self.rank, self.C, D=self._Dp, token_group=self.token_group, out=self.perm)
-
-    # ---- stage 5 on the owner: every (source, local expert) pair is a segment at a fixed place
     def expert_ffn(self):
-        self.seg_begin, self.seg_end = capmoe.ep_segments(self.cnt_recv, self.C)
-        if self.E * self.C > 0:
-            capmoe.grouped_ffn_segments(self.x_recv, self.seg_begin, self.seg_end, self.w_gate, self.w_up, self.w_down,
-                                        self.m, h_ws=self.h_ws, y_rows=self.y_recv, dev_status=self.dev_status)
+        """Stage 5 on the owner: every (source, local expert) pair is a segment at a fixed place."""
+        capmoe.ep_forward_experts(self._struct())
         return self.y_recv
 
-    # ---- stage 6
-    def combine_returned(self):
-        return capmoe.combine(self.y_ret, self.slot_row_ep, self.perm["perm_weight"], y=self.y)
-
-    def combine_from_peers(self, peer_y_recv: torch.Tensor):
-        return capmoe.ep_combine(peer_y_recv, self.R, self.rank, self.E, self.C, self.slot_row_ep,
-                                 self.perm["perm_weight"], self.d, self.x.dtype, y=self.y)
+    def combine(self):
+        """Stage 6: from the owners' buffers (peer transport) or from y_ret."""
+        capmoe.ep_forward_combine(self._struct())
+        return self.y
 
     def check(self):
         if int(self.bad.item()) != 0:
@@ -152,13 +155,12 @@ class EPLayer(EPRank):
                          C_buf=c_local, round_mode=round_mode)
 
     def forward(self):
-        kept = self.route_and_drop()
-        self.fill_send_buffer()
-        self.x_recv = exchange_rows(self.x_send, self.R, self.group)
-        self.cnt_recv = exchange_rows(kept, self.R, self.group)
+        kept = self.dispatch()
+        exchange_rows(self.x_send, self.R, self.group, out=self.x_recv)
+        exchange_rows(kept, self.R, self.group, out=self.cnt_recv)
         self.expert_ffn()
-        self.y_ret = exchange_rows(self.y_recv, self.R, self.group)
-        return self.combine_returned()
+        exchange_rows(self.y_recv, self.R, self.group, out=self.y_ret)
+        return self.combine()
 
 
 class EPGroupOnOneDevice:
@@ -175,6 +177,8 @@ class EPGroupOnOneDevice:
         dev = ranks[0].x.device
         self.peer_x = torch.tensor([rk.x_recv.data_ptr() for rk in ranks], device=dev, dtype=torch.int64)
         self.peer_y = torch.tensor([rk.y_recv.data_ptr() for rk in ranks], device=dev, dtype=torch.int64)
+        for rk in ranks:
+            rk.set_peers(*((self.peer_x, self.peer_y) if transport == "peer" else (None, None)))
 
     def _all_to_all(self, bufs_send, bufs_recv):
         R = self.R
@@ -184,18 +188,12 @@ class EPGroupOnOneDevice:
                 bufs_recv[o][r * B:(r + 1) * B].copy_(bufs_send[r][o * B:(o + 1) * B])
 
     def forward(self):
-        kept = [rk.route_and_drop() for rk in self.ranks]
+        kept = [rk.dispatch() for rk in self.ranks]
         if self.transport == "collective":
-            for rk in self.ranks:
-                rk.fill_send_buffer()
             self._all_to_all([rk.x_send for rk in self.ranks], [rk.x_recv for rk in self.ranks])
-        else:
-            for rk in self.ranks:
-                rk.dispatch_to_peers(self.peer_x)
         self._all_to_all(kept, [rk.cnt_recv for rk in self.ranks])
         for rk in self.ranks:
             rk.expert_ffn()
         if self.transport == "collective":
             self._all_to_all([rk.y_recv for rk in self.ranks], [rk.y_ret for rk in self.ranks])
-            return [rk.combine_returned() for rk in self.ranks]
-        return [rk.combine_from_peers(self.peer_y) for rk in self.ranks]
+        return [rk.combine() for rk in self.ranks]

@@ -167,3 +167,41 @@ def test_device_max_rows(cm):
     assert cm.device_max_rows(4096, 64, 8, 8, 10 ** 9, True) == 4096 * 16
     with pytest.raises(cm.CapmoeError):
         cm.device_max_rows(4096, 64, 8, 7, 10, False)
+
+
+def _fake_ep_rank(cm, **over):
+    """A capmoe_ep_rank whose every field passes validation (dummy pointers, never dereferenced)."""
+    P = cm._EPRank()
+    P.N, P.d, P.E, P.k, P.F, P.dtype = 64, 64, 8, 2, 64, cm.BF16
+    P.R, P.rank, P.mode, P.C_local, P.C = 4, 1, 2, 16, 20
+    P.drop_ws_bytes = cm.drop_workspace_bytes(64, 8, 2, 4, True)
+    for name, typ in cm._EPRank._fields_:
+        if typ is ctypes.c_void_p:
+            setattr(P, name, 4096)
+    for key, v in over.items():
+        setattr(P, key, v)
+    return P
+
+
+def test_ep_rank_phases_check_every_field_before_they_enqueue_anything(cm):
+    lib = cm.lib()
+    cases = [
+        (dict(mode=3), cm.EINVAL), (dict(R=3), cm.EINVAL), (dict(rank=4), cm.EINVAL), (dict(rank=-1), cm.EINVAL),
+        (dict(C=15), cm.EINVAL),                                  # row stride below the rank's own capacity
+        (dict(C_local=65, C=65), cm.EINVAL), (dict(mode=0), cm.EINVAL),          # no drop needs C_local = N
+        (dict(k=9), cm.EINVAL), (dict(dtype=3), cm.EUNSUPPORTED), (dict(E=512, R=4), cm.EUNSUPPORTED),
+        (dict(d=4, dtype=cm.BF16), cm.EUNSUPPORTED),              # rows of 8 bytes: not a multiple of 16
+        (dict(token_group=0), cm.EINVAL), (dict(cand=0), cm.EINVAL), (dict(bad=0), cm.EINVAL),
+        (dict(cnt_recv=0), cm.EINVAL), (dict(seg_end=0), cm.EINVAL), (dict(slot_row_ep=0), cm.EINVAL),
+        (dict(x_recv=0), cm.EINVAL), (dict(w_up=0), cm.EINVAL), (dict(perm_weight=0), cm.EINVAL),
+        (dict(peer_x=0, x_send=0), cm.EINVAL), (dict(peer_y=0, y_ret=0), cm.EINVAL),
+        (dict(drop_ws_bytes=8), cm.EWORKSPACE),
+    ]
+    before = cm.launch_count()
+    for over, want in cases:
+        P = _fake_ep_rank(cm, **over)
+        for fn in (lib.capmoe_ep_forward_dispatch, lib.capmoe_ep_forward_experts, lib.capmoe_ep_forward_combine):
+            got = fn(ctypes.byref(P), ctypes.c_void_p(0))
+            assert got == want, (over, fn.__name__, got, want)
+    assert lib.capmoe_ep_forward_dispatch(None, ctypes.c_void_p(0)) == cm.EINVAL
+    assert cm.launch_count() == before
