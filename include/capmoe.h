@@ -352,6 +352,14 @@ int capmoe_ep_forward_dispatch(const capmoe_ep_rank* P, void* stream);
 int capmoe_ep_forward_experts(const capmoe_ep_rank* P, void* stream);
 int capmoe_ep_forward_combine(const capmoe_ep_rank* P, void* stream);
 
+/* Which tensor-core kernel capmoe_grouped_ffn* and the layer forward use for bf16 shapes, for the whole
+ * process: 0 = chosen from the shape (the default), 1 = CTA pairs with 256-token tiles, 2 = one CTA per
+ * 128-token tile, 3 = the short-segment form (256 weight rows x up to 256 tokens per pair, tokens in
+ * steps of 16), 4 = that form for the down GEMM only, behind the gate/up kernel the shape selects.  All compute the same thing (Eq. 2's experts); tests force each on the same inputs.
+ * A variant the device cannot run (fewer than two SMs per straggler group) returns
+ * CAPMOE_EUNSUPPORTED at the next FFN call.  Not stream-ordered: set it while no FFN call is being issued. */
+int capmoe_debug_ffn_variant(int variant);
+
 /* Self-test of the bounded device-side wait used inside the tensor-core kernels (no counterpart
  * in the paper).  Launches one warp that waits on a barrier nothing will ever signal, with the
  * same wait routine and a limit of limit_cycles SM clock cycles (1 .. 4e9); the wait must run

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcapmoe.so")
-SOURCES = ["api.cu", "route.cu", "drop.cu", "drop_cluster.cu", "drop_parallel.cu", "variants.cu", "permute_combine.cu", "ffn_simt.cu", "ffn_tc.cu"]
+SOURCES = ["api.cu", "route.cu", "drop.cu", "drop_cluster.cu", "drop_parallel.cu", "variants.cu", "permute_combine.cu", "ffn_simt.cu", "ffn_tc.cu", "ffn_tc_t.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

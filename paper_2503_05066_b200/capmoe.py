@@ -29,7 +29,7 @@ EXPORTS = ["capmoe_capacity", "capmoe_max_rows", "capmoe_device_max_rows", "capm
            "capmoe_device_drop", "capmoe_drop_keys", "capmoe_priority_keys", "capmoe_limit_experts",
            "capmoe_rows_from_mask", "capmoe_permute", "capmoe_grouped_ffn",
            "capmoe_combine", "capmoe_layer_forward", "capmoe_layer_forward_host", "capmoe_debug_wait_probe",
-           "capmoe_grouped_ffn_segments", "capmoe_ep_plan", "capmoe_ep_forward_dispatch", "capmoe_ep_forward_experts", "capmoe_ep_forward_combine", "capmoe_ep_segments", "capmoe_ep_dispatch",
+           "capmoe_grouped_ffn_segments", "capmoe_debug_ffn_variant", "capmoe_ep_plan", "capmoe_ep_forward_dispatch", "capmoe_ep_forward_experts", "capmoe_ep_forward_combine", "capmoe_ep_segments", "capmoe_ep_dispatch",
            "capmoe_ep_combine", "capmoe_debug_read_probe", "capmoe_debug_check_indices"]
 
 
@@ -506,6 +506,14 @@ def debug_check_indices(slot_row, topk_idx, offsets, E: int, A_max: int, D: int 
                                             int(slots), int(D), _ptr(token_group), _i64(A_max), _ptr(st), _stream(stream)),
            "capmoe_debug_check_indices")
     return int(st.item())
+
+
+FFN_VARIANTS = {"auto": 0, "pair": 1, "single": 2, "short": 3, "short_down": 4}
+
+
+def debug_ffn_variant(name: str):
+    """Forces one tensor-core FFN kernel for the whole process ("auto" restores the choice by shape)."""
+    _check(lib().capmoe_debug_ffn_variant(FFN_VARIANTS[name]), "debug_ffn_variant")
 
 
 def debug_read_probe(t: torch.Tensor, stream=None):

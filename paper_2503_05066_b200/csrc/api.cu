@@ -414,6 +414,17 @@ extern "C" int capmoe_layer_forward_host(const capmoe_layer* L, const void* x_ho
   return note_cuda(err);
 }
 
+namespace capmoe {
+static std::atomic<int> g_ffn_variant{FFN_AUTO};
+int ffn_variant() { return g_ffn_variant.load(std::memory_order_relaxed); }
+}  // namespace capmoe
+
+extern "C" int capmoe_debug_ffn_variant(int variant) {
+  if (variant < capmoe::FFN_AUTO || variant > capmoe::FFN_SHORT_DOWN) return CAPMOE_EINVAL;
+  capmoe::g_ffn_variant.store(variant, std::memory_order_relaxed);
+  return CAPMOE_OK;
+}
+
 // ---------------------------------------------------------------------------------------------
 // One rank of an expert-parallel group (see capmoe_ep_rank in the header).
 namespace {

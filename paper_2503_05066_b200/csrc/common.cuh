@@ -89,6 +89,14 @@ inline cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsig
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Which tensor-core FFN kernel serves a call: chosen from the shape (FFN_AUTO), or forced through
+// capmoe_debug_ffn_variant (process-wide; tests run every variant on the same inputs with it).
+enum { FFN_AUTO = 0, FFN_PAIR = 1, FFN_SINGLE = 2, FFN_SHORT = 3, FFN_SHORT_DOWN = 4 };
+int ffn_variant();
+int ffn_tc_short(bool gate_up, bool down, const void* x_perm, const int32_t* seg_begin, const int32_t* seg_end, int E, int w_mod, int n_w, int d, int F,
+                 const void* w_gate, const void* w_up, const void* w_down, void* h_ws, void* y_perm, int64_t A_max,
+                 int D_straggler, int32_t* dev_status, int32_t* sched1, int32_t* sched2, cudaEvent_t mid, cudaStream_t st);
+
 // Zeroes up to two small int32 arrays with one chained kernel launch (a memset node between two
 // kernels costs more stream time than this and breaks the chain of overlapped launches).
 int clear_words(int32_t* a, int na, int32_t* b, int nb, cudaStream_t st);

@@ -143,3 +143,61 @@ def test_grouped_ffn_on_random_segments(cm, E, d, F, rows, D_straggler):
     ref = oracle.expert_ffn(np.ascontiguousarray(to_np(x_perm)[sample]), row_expert, to_np(wg), to_np(wu), to_np(wd),
                             "bf16")
     assert rel_err(got[sample], ref) <= 2e-2
+
+
+# Every tensor-core FFN kernel on the same segments: short and ragged ones (token counts around the
+# short-segment kernel's steps of 16 and its 256-token tiles), long ones, empty ones, widths that are
+# odd multiples of 64, with and without the straggler partition.
+_FFN_VARIANT_CASES = [
+    (6, 128, 256, (0, 1, 15, 16, 17, 255), 0),
+    (5, 192, 192, (256, 257, 300, 512, 513), 0),
+    (4, 64, 320, (31, 33, 700, 1), 2),
+    (3, 256, 448, (1030, 129, 270), 3),
+    (8, 128, 128, (40, 0, 0, 90, 272, 16, 48, 600), 4),
+]
+
+
+@pytest.mark.parametrize("variant", ["pair", "single", "short", "short_down", "auto"])
+@pytest.mark.parametrize("E,d,F,rows,D_straggler", _FFN_VARIANT_CASES)
+def test_every_ffn_kernel_on_the_same_segments(cm, variant, E, d, F, rows, D_straggler):
+    A = int(sum(rows))
+    A_max = A + 40                                               # rows a last tile may read but never write
+    g = torch.Generator().manual_seed(E * 77 + d + F + A)
+    x_perm = torch.randn((A_max, d), generator=g).to(torch.bfloat16)
+    x_perm[A:] = float("nan")                                    # what lies past the last segment must not leak in
+    wg = (torch.randn((E, F, d), generator=g) * 0.05).to(torch.bfloat16)
+    wu = (torch.randn((E, F, d), generator=g) * 0.05).to(torch.bfloat16)
+    wd = (torch.randn((E, d, F), generator=g) * 0.05).to(torch.bfloat16)
+    offsets = np.concatenate([[0], np.cumsum(rows)]).astype(np.int32)
+    y = torch.full((A_max, d), 7.0, dtype=torch.bfloat16).cuda()
+    st = torch.zeros((cm.FFN_STATUS_WORDS,), dtype=torch.int32).cuda()
+    cm.debug_ffn_variant(variant)
+    try:
+        out = cm.grouped_ffn(dev(x_perm), dev(offsets), dev(wg), dev(wu), dev(wd), D_straggler=D_straggler, y_perm=y,
+                             dev_status=st)
+        torch.cuda.synchronize()
+    finally:
+        cm.debug_ffn_variant("auto")
+    assert int(st[0].item()) == cm.OK
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert (got[A:] == 7.0).all()                               # never written
+    assert np.isfinite(got[:A]).all()
+    rng = np.random.default_rng(A)
+    nz = np.array(rows) > 0
+    edges = np.concatenate([offsets[:-1][nz], offsets[1:][nz] - 1])
+    steps = np.concatenate([np.arange(offsets[e], offsets[e + 1], 16) for e in range(E)] + [np.zeros(0, np.int64)])
+    sample = np.unique(np.concatenate([rng.integers(0, A, size=64), edges, steps, np.minimum(steps + 15, A - 1)])).astype(np.int64)
+    row_expert = (np.searchsorted(offsets, sample, side="right") - 1).astype(np.int32)
+    ref = oracle.expert_ffn(np.ascontiguousarray(to_np(x_perm)[sample]), row_expert, to_np(wg), to_np(wu), to_np(wd),
+                            "bf16")
+    assert rel_err(got[sample], ref) <= 2e-2
+    # all kernels accumulate over K in the same order: the same bits
+    if variant != "single":
+        cm.debug_ffn_variant("single")
+        try:
+            y2 = torch.full((A_max, d), 7.0, dtype=torch.bfloat16).cuda()
+            ref_k = cm.grouped_ffn(dev(x_perm), dev(offsets), dev(wg), dev(wu), dev(wd), D_straggler=D_straggler, y_perm=y2)
+            torch.cuda.synchronize()
+        finally:
+            cm.debug_ffn_variant("auto")
+        assert torch.equal(out[:A].view(torch.int16), ref_k[:A].view(torch.int16))
