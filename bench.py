@@ -562,14 +562,12 @@ def main():
     use_tc = capmoe.ffn_uses_tensor_cores(cfg.d, cfg.F, g["x"].dtype)
     # Which measured cuBLAS figure bounds the kernel depends on the clock regime of the timed region:
     # a region of a second or more runs under the power cap like the sustained measurement, a short
-    # one at burst clocks.  Both fractions are printed; `frac` uses the regime this run was in, and a
-    # run that beats the sustained figure is compared with the burst one.
+    # one at burst clocks.  Both fractions are printed; `frac` uses the regime this run was in (the
+    # denominator is cuBLAS measured the same way, so a fraction slightly above 1 is possible).
     region_s = (ms_step + ms_with_events) * 1e-3 * K
     ach1 = gemm1_flops / t1 / 1e12 if t1 > 0 else None
     ach2 = gemm2_flops / t2 / 1e12 if t2 > 0 else None
     regime = "sustained" if (region_s >= 0.5 and "sw_power_cap" in (clocks.get("reasons") or [])) else "burst"
-    if use_tc and regime == "sustained" and max(ach1 or 0.0, ach2 or 0.0) > peaks["bf16_tflops_sustained"]:
-        regime = "burst"
     peak_tf = (peaks["bf16_tflops_sustained"] if regime == "sustained" else peaks["bf16_tflops"]) if use_tc else None
     tr1, tr2, tr_note = _recorded_traffic((cfg.name, cfg.N, cfg.F, args.mode, args.gamma, bool(args.straggler)))
     sm_mhz, sm_max = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
