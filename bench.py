@@ -36,17 +36,17 @@ UNIT = "tokens/s"
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the two FFN GEMM
 # kernels, from a one-pass ncu capture.  A capture describes one build of the kernel: it is keyed
-# by the SHA-256 of the kernel's source file at the time of the capture, and is reported only while
-# the file still has that hash (else `traffic` is null and says why).
+# by the SHA-256 of the kernel's source files (concatenated) at the time of the capture, and is
+# reported only while they still have that hash (else `traffic` is null and says why).
 # key = (config, N, F, mode, gamma, straggler) -> {"gate_up": bytes, "down": bytes}
 NCU_TRAFFIC = {
-    "kernel_source": "paper_2503_05066_b200/csrc/ffn_tc.cu",
-    "sha256": "754a04056b16863c9cd2a2a855ba55652ec9593c9b4d67b05500ad413bff5338",
+    "kernel_sources": ["paper_2503_05066_b200/csrc/ffn_tc.cu", "paper_2503_05066_b200/csrc/tc_common.cuh"],
+    "sha256": "3f26b24dce1e0deed7412bc54ae49b065b0385ed7942868599a8b7076a42af7f",
     "captures": {
         # ncu --metrics gpu__time_duration.sum,dram__bytes_read.sum,dram__bytes_write.sum (one pass),
         # means of nine launches each of the two GEMM kernels
-        ("mixtral", 8192, 14336, "expanded_drop", 1.0, True): {"gate_up": 2306900000 + 460500000,
-                                                                "down": 4978600000 + 130200000},
+        ("mixtral", 8192, 14336, "expanded_drop", 1.0, True): {"gate_up": 2567100000 + 460500000,
+                                                                "down": 3038800000 + 126500000},
     },
 }
 
@@ -55,9 +55,9 @@ def _recorded_traffic(key):
     """(gate_up_bytes, down_bytes, note) for this workload from the recorded ncu capture, or
     (None, None, reason)."""
     import hashlib
-    path = os.path.join(ROOT, NCU_TRAFFIC["kernel_source"])
     try:
-        digest = hashlib.sha256(open(path, "rb").read()).hexdigest()
+        digest = hashlib.sha256(b"".join(open(os.path.join(ROOT, f), "rb").read()
+                                         for f in NCU_TRAFFIC["kernel_sources"])).hexdigest()
     except OSError:
         return None, None, "kernel source not found"
     if NCU_TRAFFIC["sha256"] is None:
