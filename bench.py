@@ -578,6 +578,9 @@ def main():
         "frac": (ach1 / peak_tf) if (ach1 and peak_tf) else None,
         "peak_source": "%s cuBLAS bf16, %s figure (timed region %.2f s, median SM clock %s MHz of %s)"
                        % (peaks["source"], regime, region_s, sm_mhz, sm_max),
+        "frac_note": ("above 1: this launch ran faster than the cuBLAS loop behind the %s figure, which was measured in the "
+                      "same clock regime; see frac_of_burst_peak for the other denominator" % regime)
+        if (ach1 and peak_tf and ach1 > peak_tf) else None,
         "frac_of_burst_peak": (ach1 / peaks["bf16_tflops"]) if (ach1 and use_tc) else None,
         "frac_of_sustained_peak": (ach1 / peaks["bf16_tflops_sustained"]) if (ach1 and use_tc) else None,
         "peak_burst": peaks["bf16_tflops"], "peak_sustained": peaks["bf16_tflops_sustained"],
