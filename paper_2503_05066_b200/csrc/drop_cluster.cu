@@ -327,9 +327,11 @@ static int cluster_size(int64_t N, int E, bool expanded) {
 // Every cluster reads all N top-k lists, E times in total, so the cluster select wins while a CTA
 // holds few tokens per thread: measured faster up to 4 per thread (16384 tokens with 64 experts:
 // 27 us against 35 us), and up to 8 with at most 16 experts (65536 tokens, 8 experts: 27 against
-// 48 us), slower beyond (32768 tokens, 60 experts: 54 against 38 us).
+// 48 us), slower beyond (32768 tokens, 60 experts: 54 against 38 us).  Expanded Drop goes up to 8 per
+// thread whatever E: the token-parallel select then walks five radix levels of two launches each
+// (16384 tokens, 64 experts, D = 8: 49 against 57 us; 60 experts, D = 4: 52 against 61 us).
 bool drop_cluster_takes(int64_t N, int E, bool expanded) {
-  const int max_tpt = E <= 16 ? 8 : 4;
+  const int max_tpt = (E <= 16 || expanded) ? 8 : 4;
   return N > 0 && ceil_div(N, cluster_size(N, E, expanded)) <= (int64_t)SEL_THREADS * max_tpt;
 }
 

@@ -154,6 +154,8 @@ DROP_CASES = [
     (16384, 8, 2, 2, float("inf"), 0.0),
     (3500, 130, 6, 10, 1.0, 0.0),
     (4000, 200, 4, 8, 1.0, 1.0),
+    (16000, 60, 4, 4, 1.0, 1.0),     # Expanded Drop: 8 tokens per thread with many experts, heavy ties
+    (15000, 64, 8, 8, 0.5, 0.5),
     # larger batches take the token-parallel select
     (17001, 60, 4, 4, 0.5, 1.0),     # ties at the threshold resolved by position
     (16400, 130, 6, 10, 1.0, 0.0),
