@@ -910,9 +910,13 @@ int ffn_tc(const void* x_perm, const int32_t* seg_begin, const int32_t* seg_end,
                         A_max, D_straggler, dev_status, sched1, sched2, nullptr, st);
   };
   // CTA pairs (256-row tiles) when the expert segments are long enough that the extra tail
-  // padding does not matter, or are known multiples of 256 rows
+  // padding does not matter, or when a typical segment (A_max / E rows) pads to about the same number
+  // of rows with 256-row tiles as with 128-row ones (the pair kernel moves a third less through
+  // shared memory per flop: 134 against 154 us on 137-row segments, Qwen shape at 2048 tokens; the
+  // other way round on 547-row segments, 179 against 170 us)
+  const int64_t pad256 = ceil_div(avg_rows, (int64_t)256) * 256, pad128 = ceil_div(avg_rows, (int64_t)128) * 128;
   const bool want_pairs = variant == FFN_AUTO || variant == FFN_SHORT_DOWN
-                              ? avg_rows >= 1024 || (avg_rows >= 256 && avg_rows % 256 == 0)
+                              ? avg_rows >= 1024 || (avg_rows > 0 && pad256 * 10 <= pad128 * 11)
                               : variant == FFN_PAIR;
   if (want_pairs && !pairs_fit && variant == FFN_PAIR) return CAPMOE_EUNSUPPORTED;
   if (want_pairs && pairs_fit) {
