@@ -201,3 +201,36 @@ def test_every_ffn_kernel_on_the_same_segments(cm, variant, E, d, F, rows, D_str
         finally:
             cm.debug_ffn_variant("auto")
         assert torch.equal(out[:A].view(torch.int16), ref_k[:A].view(torch.int16))
+
+
+def _layer_cases(n, seed):
+    """Random whole-layer configurations: token counts that leave ragged tiles, expert counts that
+    are not powers of two, every drop mode, with and without shared experts and the straggler
+    partition; bf16 shapes on the tensor-core kernels and fp32 shapes on the FMA kernel."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        bf16 = i % 3 != 2
+        D = int(rng.choice([1, 2, 3, 4]))
+        m = int(rng.integers(1, 6))
+        E = D * m
+        k = int(rng.integers(1, min(E, 6) + 1))
+        N = int(rng.choice([1, 63, 200, 777, 1500, 2304]))
+        if bf16:
+            d, F = 64 * int(rng.integers(1, 5)), 64 * int(rng.integers(1, 6))
+        else:
+            d, F = int(rng.integers(3, 40)) * 4, int(rng.integers(5, 90))
+        mode = ["nodrop", "token_drop", "expanded_drop"][int(rng.integers(0, 3))]
+        gamma = float(rng.choice([0.5, 1.0, 1.3, 2.0]))
+        F_shared = int(rng.choice([0, 0, 64 * int(rng.integers(1, 4)) if bf16 else int(rng.integers(4, 50))]))
+        straggler = bool(bf16 and rng.integers(0, 3) == 0)
+        out.append((N, d, E, k, F, D, "bf16" if bf16 else "f32", mode, gamma, F_shared, straggler, 100 + i))
+    return out
+
+
+@pytest.mark.parametrize("N,d,E,k,F,D,dtype,mode,gamma,F_shared,straggler,seed", _layer_cases(24, 2024) + _layer_cases(24, 7))
+def test_layer_on_random_configurations(cm, N, d, E, k, F, D, dtype, mode, gamma, F_shared, straggler, seed):
+    from tests.test_gpu_parity import _layer_case
+    cfg = synth.LayerConfig("random", N=N, d=d, E=E, k=k, F=F, D=D, dtype=dtype, gammas=(gamma,), bias_kind="zipf",
+                            bias_s=0.7, F_shared=F_shared, seed=seed)
+    _layer_case(cm, cfg, mode, gamma, straggler=straggler, std=0.05)
