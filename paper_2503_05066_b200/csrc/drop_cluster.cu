@@ -4,8 +4,10 @@
 // the first.
 //
 // An expert is served by a thread-block cluster of R CTAs (R = 1, 2, 4 or 8, chosen so that the
-// E*R CTAs about fill the GPU).  CTA r of the cluster owns the r-th contiguous block of tokens and
-// every thread TPT consecutive tokens of it, so token order is (rank, thread, u) order.  A thread
+// E*R CTAs about fill the GPU).  CTA r of the cluster owns the r-th contiguous block of tokens, warp
+// w of it 32*TPT consecutive ones, and lane l of the warp tokens l, l+32, ... of those: for a fixed u
+// the lanes of a warp hold 32 consecutive tokens, so their loads and stores share cache lines, and
+// token order is (rank, warp, u, lane) order.  A thread
 // reads the top-k lists of its tokens once and keeps, for each token that is a candidate of the
 // expert, the candidate's slot and key (the score's bit pattern: non-negative floats order like
 // unsigned integers) in registers for the rest of the kernel:
@@ -64,6 +66,39 @@ __device__ __forceinline__ uint32_t block_scan1(uint32_t v, uint32_t* wt, uint32
   return warp_before + incl - v;
 }
 
+// The same for TPT values per thread whose order is (warp, u, lane): ex[u] = sum of all values that
+// come before this thread's u-th one.
+template <int TPT>
+__device__ __forceinline__ void block_scan_tokens(const uint32_t (&p)[TPT], uint32_t (&ex)[TPT], uint32_t* wt,
+                                                  uint32_t& total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  uint32_t run = 0;                                    // the warp's values of the lower u (warp-uniform)
+#pragma unroll
+  for (int u = 0; u < TPT; ++u) {
+    uint32_t incl = p[u];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    ex[u] = run + incl - p[u];
+    run += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (lane == 31) wt[wid] = run;
+  __syncthreads();
+  const uint32_t w = wt[lane];                          // SEL_WARPS == 32
+  uint32_t wi = w;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t n = __shfl_up_sync(0xffffffffu, wi, o);
+    if (lane >= o) wi += n;
+  }
+  total = __shfl_sync(0xffffffffu, wi, 31);
+  const uint32_t warp_before = __shfl_sync(0xffffffffu, wi - w, wid);
+#pragma unroll
+  for (int u = 0; u < TPT; ++u) ex[u] += warp_before;
+}
+
 template <bool EXPANDED, int TPT>
 __global__ void __launch_bounds__(SEL_THREADS)
 k_select_cluster(const float* __restrict__ score_src,   // topk_score [N,k] (Token Drop) or scores [N,E] (Expanded)
@@ -92,28 +127,64 @@ k_select_cluster(const float* __restrict__ score_src,   // topk_score [N,k] (Tok
   if (tid < MAX_E) { cnt[tid] = 0; dupc[tid] = 0; homec[tid] = 0; }
   __syncthreads();
 
-  // This thread's tokens.  Sixteen top-k entries (JJ of every token) are requested before the first
-  // is used, so that the loads of a thread overlap; each entry is counted for its expert and
-  // compared with this cluster's expert.
-  const int64_t lo = (int64_t)rank * T + (int64_t)tid * TPT;
+  // This thread's tokens (see the head of the file).  Sixteen top-k entries (JJ of every token) are
+  // requested before the first is used, so that the loads of a thread overlap; each entry is counted
+  // for its expert and compared with this cluster's expert.
   const int64_t hi = min(N, (int64_t)(rank + 1) * T);
-  int slot[TPT], home[TPT];
+  const int64_t tok0 = (int64_t)rank * T + (int64_t)(tid >> 5) * (32 * TPT) + lane;   // token of u: tok0 + 32 u
+  int slot[TPT], home_lo[TPT];                      // home_lo: first expert of the token's home device
   uint32_t key[TPT];
   bool dup[TPT];                                    // Expanded Drop: home-device expert that is already a top-k slot
+  {
+    int g = 0;
 #pragma unroll
-  for (int u = 0; u < TPT; ++u) {
-    slot[u] = -1; dup[u] = false;
-    home[u] = (EXPANDED && lo + u < hi) ? home_group(lo + u, N, D, token_group) : -1;
-    if (count_homes && home[u] >= 0) atomicAdd(&homec[home[u]], 1);
+    for (int u = 0; u < TPT; ++u) {
+      const int64_t t = tok0 + 32 * u;
+      slot[u] = -1; dup[u] = false; home_lo[u] = -m;   // (-m for a token past the end: matches no expert)
+      if (EXPANDED && t < hi) {
+        if (token_group) g = token_group[t];
+        else if (u == 0) g = (int)((t * (int64_t)D) / N);
+        else while ((int64_t)(g + 1) * N <= t * (int64_t)D) ++g;        // floor(t * D / N), from the previous token's
+        home_lo[u] = g * m;
+        if (count_homes) atomicAdd(&homec[g], 1);
+      }
+    }
   }
+  // A token's k entries are contiguous and the lanes of a warp hold consecutive tokens; with k a
+  // multiple of 4 (or 2) the entries are fetched four (two) at a time.  (With TPT consecutive tokens
+  // per thread and scalar loads this loop took 7 of the kernel's 18 us at 64 experts and k = 8, 19 of
+  // 42 us at 16384 tokens with k = 6: every load instruction touched up to 32 cache lines.)
   constexpr int JJ = TPT <= 2 ? 8 : 16 / TPT;
+  const int vec = (k & 3) == 0 && JJ >= 4 ? 4 : (k & 1) == 0 ? 2 : 1;
   for (int j0 = 0; j0 < k; j0 += JJ) {
     int32_t v[TPT][JJ];
+    if (vec == 4) {
+      if constexpr (JJ >= 4) {
 #pragma unroll
-    for (int u = 0; u < TPT; ++u)
+        for (int u = 0; u < TPT; ++u)
 #pragma unroll
-      for (int jj = 0; jj < JJ; ++jj)
-        v[u][jj] = (lo + u < hi && j0 + jj < k) ? topk_idx[(lo + u) * k + j0 + jj] : -1;
+          for (int jj = 0; jj < JJ; jj += 4) {
+            int4 q = make_int4(-1, -1, -1, -1);
+            if (tok0 + 32 * u < hi && j0 + jj < k) q = *reinterpret_cast<const int4*>(topk_idx + (tok0 + 32 * u) * k + j0 + jj);
+            v[u][jj] = q.x; v[u][jj + 1] = q.y; v[u][jj + 2] = q.z; v[u][jj + 3] = q.w;
+          }
+      }
+    } else if (vec == 2) {
+#pragma unroll
+      for (int u = 0; u < TPT; ++u)
+#pragma unroll
+        for (int jj = 0; jj < JJ; jj += 2) {
+          int2 q = make_int2(-1, -1);
+          if (tok0 + 32 * u < hi && j0 + jj < k) q = *reinterpret_cast<const int2*>(topk_idx + (tok0 + 32 * u) * k + j0 + jj);
+          v[u][jj] = q.x; v[u][jj + 1] = q.y;
+        }
+    } else {
+#pragma unroll
+      for (int u = 0; u < TPT; ++u)
+#pragma unroll
+        for (int jj = 0; jj < JJ; ++jj)
+          v[u][jj] = (tok0 + 32 * u < hi && j0 + jj < k) ? topk_idx[(tok0 + 32 * u) * k + j0 + jj] : -1;
+    }
 #pragma unroll
     for (int u = 0; u < TPT; ++u)
 #pragma unroll
@@ -121,7 +192,7 @@ k_select_cluster(const float* __restrict__ score_src,   // topk_score [N,k] (Tok
         const int ev = v[u][jj];
         if (ev >= 0) {
           if (!load) atomicAdd(&cnt[ev], 1);          // (aggregating these per warp with match.any measured slower)
-          if (EXPANDED && ev / m == home[u]) atomicAdd(&dupc[ev], 1);
+          if (EXPANDED && (unsigned)(ev - home_lo[u]) < (unsigned)m) atomicAdd(&dupc[ev], 1);
           if (ev == e) slot[u] = j0 + jj;
         }
       }
@@ -129,14 +200,14 @@ k_select_cluster(const float* __restrict__ score_src,   // topk_score [N,k] (Tok
   if (EXPANDED) {
 #pragma unroll
     for (int u = 0; u < TPT; ++u)
-      if (home[u] == e / m) {
+      if (home_lo[u] == e - e % m) {
         if (slot[u] < 0) slot[u] = k + (e % m);
         else dup[u] = true;
       }
   }
 #pragma unroll
   for (int u = 0; u < TPT; ++u) {
-    const int64_t t = lo + u;
+    const int64_t t = tok0 + 32 * u;
     key[u] = 0;
     if (slot[u] >= 0) key[u] = __float_as_uint(EXPANDED ? score_src[t * E + e] : score_src[t * k + slot[u]]);
   }
@@ -236,30 +307,30 @@ k_select_cluster(const float* __restrict__ score_src,   // topk_score [N,k] (Tok
   }
 
   // ranks in token order: kept = above tau, plus the first `need` equal to it
-  uint32_t packed = 0;
+  uint32_t packed[TPT], before[TPT];
 #pragma unroll
-  for (int u = 0; u < TPT; ++u)
+  for (int u = 0; u < TPT; ++u) {
+    packed[u] = 0;
     if (slot[u] >= 0) {
       const bool gt = keep_all || (select && key[u] > tau), eq = select && key[u] == tau;
-      packed += (gt ? 1u : 0u) | (eq ? 0x10000u : 0u);
+      packed[u] = (gt ? 1u : 0u) | (eq ? 0x10000u : 0u);
     }
+  }
   uint32_t tot;
-  const uint32_t before = block_scan1(packed, wt[4], tot);      // a CTA holds at most 8192 tokens: 16 bits each
+  block_scan_tokens<TPT>(packed, before, wt[4], tot);           // a CTA holds at most 8192 tokens: 16 bits each
   if (R > 1) {
     if (tid < R) *cluster.map_shared_rank(&totals[rank], tid) = tot;
     cluster.sync();                                 // last access to another CTA's shared memory is behind us
   }
-  uint32_t gt_before = before & 0xffffu, eq_before = before >> 16;
-  for (int r = 0; r < rank; ++r) { gt_before += totals[r] & 0xffffu; eq_before += totals[r] >> 16; }
+  uint32_t gt_base = 0, eq_base = 0;
+  for (int r = 0; r < rank; ++r) { gt_base += totals[r] & 0xffffu; eq_base += totals[r] >> 16; }
 #pragma unroll
   for (int u = 0; u < TPT; ++u) {
-    const int64_t t = lo + u;
+    const int64_t t = tok0 + 32 * u;
     if (slot[u] >= 0) {
-      const bool gt = keep_all || (select && key[u] > tau), eq = select && key[u] == tau;
-      const bool keep = gt || (eq && eq_before < need);
+      const uint32_t gt_before = gt_base + (before[u] & 0xffffu), eq_before = eq_base + (before[u] >> 16);
+      const bool keep = (packed[u] & 1u) || ((packed[u] >> 16) && eq_before < need);
       slot_row[t * slots + slot[u]] = keep ? (int32_t)(off + gt_before + (eq_before < need ? eq_before : need)) : -1;
-      gt_before += gt ? 1u : 0u;
-      eq_before += eq ? 1u : 0u;
     }
     if (EXPANDED && dup[u]) slot_row[t * slots + k + (e % m)] = -1;   // that slot is the top-k slot's duplicate
   }
