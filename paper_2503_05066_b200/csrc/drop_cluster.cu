@@ -394,15 +394,14 @@ static int cluster_size(int64_t N, int E, bool expanded) {
   return R;
 }
 
-// Whether the cluster select serves this batch (else the token-parallel select of drop_parallel.cu).
-// Every cluster reads all N top-k lists, E times in total, so the cluster select wins while a CTA
-// holds few tokens per thread: measured faster up to 4 per thread (16384 tokens with 64 experts:
-// 27 us against 35 us), and up to 8 with at most 16 experts (65536 tokens, 8 experts: 27 against
-// 48 us), slower beyond (32768 tokens, 60 experts: 54 against 38 us).  Expanded Drop goes up to 8 per
-// thread whatever E: the token-parallel select then walks five radix levels of two launches each
-// (16384 tokens, 64 experts, D = 8: 49 against 57 us; 60 experts, D = 4: 52 against 61 us).
+// Whether the cluster select serves this batch (else the token-parallel select of drop_parallel.cu):
+// while a CTA holds at most 8 tokens per thread.  Every cluster reads all N top-k lists, E times in
+// total, but out of L2 and in one launch; the token-parallel select takes 13.  Measured (stage call
+// replayed from a graph / inside a layer forward): 32768 tokens, 60 experts, Token Drop 28 / 31 us
+// against 42 / 58 us; 64 experts 47 / 46 against 50 / 75 us; 16384 tokens, 64 experts, Expanded Drop
+// 38 / 54 against 57 / 89 us.
 bool drop_cluster_takes(int64_t N, int E, bool expanded) {
-  const int max_tpt = (E <= 16 || expanded) ? 8 : 4;
+  const int max_tpt = 8;
   return N > 0 && ceil_div(N, cluster_size(N, E, expanded)) <= (int64_t)SEL_THREADS * max_tpt;
 }
 
