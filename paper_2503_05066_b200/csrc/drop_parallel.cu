@@ -101,22 +101,31 @@ pk_hist(PArgs a, PWs w, int level, Level lv, int first_level_counts_cand) {
     for (int i = tid; i < a.E; i += PAIR_THREADS) cand_s[i] = 0;
   __syncthreads();
   const int64_t t = (int64_t)blockIdx.x * CHUNK + (tid & (CHUNK - 1));
-  if (t < a.N) {
-    const int32_t* row = a.topk_idx + t * a.k;
-    const int home = a.expanded ? home_group(t, a.N, a.D, a.token_group) : 0;
-    for (int s = tid / CHUNK; s < a.slots; s += TPT) {
-      int e;
-      unsigned long long key;
-      if (!pair_of(a, t, s, row, home, e, key)) continue;
-      if (first_level_counts_cand) atomicAdd(&cand_s[e], 1);
-      const int sg = e / a.seg_m;
-      if (level > 0) {
-        const SegState st = w.seg[sg];
-        if (st.done) continue;
-        const int hi = lv.shift + lv.bits;                       // < 64 for every level after the first
-        if ((key >> hi) != (st.prefix >> hi)) continue;
-      }
-      const uint32_t digit = (uint32_t)(key >> lv.shift) & ((1u << lv.bits) - 1u);
+  const bool tok_ok = t < a.N;
+  const int32_t* row = a.topk_idx + (tok_ok ? t : 0) * a.k;
+  const int home = (a.expanded && tok_ok) ? home_group(t, a.N, a.D, a.token_group) : 0;
+  const int lane = tid & 31;
+  // (the slot index is the same for all lanes of a warp, so the warp stays together in this loop)
+  for (int s = tid / CHUNK; s < a.slots; s += TPT) {
+    int e = 0;
+    unsigned long long key = 0;
+    bool in = tok_ok && pair_of(a, t, s, row, home, e, key);
+    if (in && first_level_counts_cand) atomicAdd(&cand_s[e], 1);
+    const int sg = e / a.seg_m;
+    if (in && level > 0) {
+      const SegState st = w.seg[sg];
+      const int hi = lv.shift + lv.bits;                         // < 64 for every level after the first
+      in = !st.done && (key >> hi) == (st.prefix >> hi);
+    }
+    const uint32_t digit = (uint32_t)(key >> lv.shift) & ((1u << lv.bits) - 1u);
+    if (level == 0) {
+      // Every candidate takes part in the first level, and a warp's lanes hold one slot of 32
+      // consecutive tokens: for a home-device slot that is one expert, whose scores fall into a few
+      // bins.  One atomic per distinct (segment, bin) of the warp instead of one per lane.
+      const uint32_t bin = in ? (uint32_t)sg * BINS + digit : 0xffffffffu - (uint32_t)lane;
+      const unsigned same = __match_any_sync(0xffffffffu, bin);
+      if (in && lane == __ffs(same) - 1) atomicAdd(&w.hist[bin], (uint32_t)__popc(same));
+    } else if (in) {
       atomicAdd(&w.hist[(size_t)sg * BINS + digit], 1u);
     }
   }
