@@ -155,7 +155,8 @@ k_select_cluster(const float* __restrict__ score_src,   // topk_score [N,k] (Tok
   // per thread and scalar loads this loop took 7 of the kernel's 18 us at 64 experts and k = 8, 19 of
   // 42 us at 16384 tokens with k = 6: every load instruction touched up to 32 cache lines.)
   constexpr int JJ = TPT <= 2 ? 8 : 16 / TPT;
-  const int vec = (k & 3) == 0 && JJ >= 4 ? 4 : (k & 1) == 0 ? 2 : 1;
+  const uintptr_t idx_addr = reinterpret_cast<uintptr_t>(topk_idx);
+  const int vec = (k & 3) == 0 && JJ >= 4 && (idx_addr & 15) == 0 ? 4 : (k & 1) == 0 && (idx_addr & 7) == 0 ? 2 : 1;
   for (int j0 = 0; j0 < k; j0 += JJ) {
     int32_t v[TPT][JJ];
     if (vec == 4) {
@@ -350,13 +351,22 @@ k_mask_from_rows(const int32_t* __restrict__ slot_row, const int32_t* __restrict
   const int32_t* sr = slot_row + t * slots;
   const int m = slots > k ? E / D : 0;
   const int g = slots > k ? home_group(t, N, D, token_group) : 0;
-  for (int s = 0; s < slots; ++s)
-    if (sr[s] >= 0) {
+  auto mark = [&](int s, int row) {
+    if (row >= 0) {
       const int e = s < k ? topk_idx[t * k + s] : g * m + (s - k);
 #pragma unroll
       for (int i = 0; i < MAX_E / 64; ++i)
         if (i == (e >> 6)) w[i] |= 1ull << (e & 63);
     }
+  };
+  if ((slots & 3) == 0 && (reinterpret_cast<uintptr_t>(slot_row) & 15) == 0) {   // rows of 16-byte pieces: four entries per load
+    for (int s = 0; s < slots; s += 4) {
+      const int4 q = *reinterpret_cast<const int4*>(sr + s);
+      mark(s, q.x); mark(s + 1, q.y); mark(s + 2, q.z); mark(s + 3, q.w);
+    }
+  } else {
+    for (int s = 0; s < slots; ++s) mark(s, sr[s]);
+  }
 #pragma unroll
   for (int i = 0; i < MAX_E / 64; ++i)
     if (i < W) keep_mask[t * W + i] = w[i];
