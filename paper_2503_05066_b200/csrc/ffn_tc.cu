@@ -315,6 +315,10 @@ k_ffn_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUte
           group_sync(5, 4 * RF_SUBS * 32);                     // the tile of logits is complete
           const int et = tid - 64;                             // 0 .. 511
           const int r = et >> 3, j = et & 7;
+          if (((et >> 5) << 2) >= t.rows) {                    // none of this warp's four tokens exists:
+            group_sync(5, 4 * RF_SUBS * 32);                   // leave the issue slots to the warps that have some
+            continue;
+          }
           const bool tok_ok = r < t.rows;
           const int64_t tok = (int64_t)t.row0 + r;
           const int c0 = j * CS;
