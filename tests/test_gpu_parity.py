@@ -156,6 +156,10 @@ DROP_CASES = [
     (4000, 200, 4, 8, 1.0, 1.0),
     (16000, 60, 4, 4, 1.0, 1.0),     # Expanded Drop: 8 tokens per thread with many experts, heavy ties
     (15000, 64, 8, 8, 0.5, 0.5),
+    # the limits of the interface: 256 experts, 32 experts per token
+    (600, 256, 32, 8, 1.0, 0.0),
+    (300, 256, 32, 256, 1.0, 0.5),
+    (9000, 256, 32, 4, 1.5, 0.0),
     # larger batches take the token-parallel select
     (17001, 60, 4, 4, 0.5, 1.0),     # ties at the threshold resolved by position
     (16400, 130, 6, 10, 1.0, 0.0),
@@ -338,6 +342,14 @@ def _layer_case(cm, cfg, mode, gamma, straggler=False, sample=None, std=0.02, co
 @pytest.mark.parametrize("mode", ["nodrop", "token_drop", "expanded_drop"])
 def test_layer_tiny_fp32(cm, mode):
     _layer_case(cm, synth.CONFIGS["tiny_f32"], mode, 1.0)
+
+
+@pytest.mark.parametrize("mode", ["nodrop", "token_drop", "expanded_drop"])
+@pytest.mark.parametrize("dtype,d,F", [("bf16", 64, 128), ("f32", 24, 20)])
+def test_layer_at_the_expert_and_k_limits(cm, mode, dtype, d, F):
+    """256 experts, 32 per token, 8 devices: 64 slots per token under Expanded Drop."""
+    cfg = synth.CONFIGS["tiny_f32"].with_(N=700, d=d, F=F, E=256, k=32, D=8, dtype=dtype, bias_kind="zipf")
+    _layer_case(cm, cfg, mode, 1.0)
 
 
 @pytest.mark.parametrize("mode", ["nodrop", "token_drop", "expanded_drop"])
