@@ -586,6 +586,8 @@ def main():
         "peak_burst": peaks["bf16_tflops"], "peak_sustained": peaks["bf16_tflops_sustained"],
         # the same throughput scaled to the maximum SM clock (time x median sampled MHz / max MHz)
         "achieved_at_max_clock": (ach1 * sm_max / sm_mhz) if (ach1 and sm_mhz and sm_max) else None,
+        "achieved_at_max_clock_note": "extrapolation from the median of 100 ms nvidia-smi clock samples over the whole timed "
+                                      "region; under the power cap the clock moves within a step, so this can overshoot",
         "flops_per_launch": gemm1_flops,
         "traffic": tr1, "traffic_note": tr_note,
         "algorithmic_bytes": (2 * cfg.E * cfg.F * cfg.d + A * cfg.d + A * cfg.F) * elt,
